@@ -1,0 +1,260 @@
+/*
+ * qe.h -- C ABI of libqe: an FP8 delayed-scaling linear layer run as three checked actions
+ * (forward F, input-gradient dI, deferred weight-gradient dW) on one NVIDIA B200 (sm_100a).
+ *
+ * The operations and their rules follow the QEffect contract:
+ *   Eqs. 1-2      TapeKey(e,s,m,u,i) / TapeRef(p,g_p): retained work is named by a logical key and by a slot
+ *                 plus its generation; a consumer presents both.
+ *   Eqs. 3-5      (Y,S1,T)=F(X,W,S0); (dX,S2,Q)=dI(dY,T,S1); dW=dW(Q).  F and dI advance the effect token and
+ *                 the scaling state once each; dW never touches scaling state.
+ *   Sec. 3.3      weight version e_W and cache version e_C; the first forward after an optimizer step refreshes
+ *                 the quantised-weight cache.
+ *   Sec. 3.4      direct gradient placement: dW accumulates in place into a caller-owned flat FP32 buffer.
+ *   Algorithm 1   every action is check -> run -> commit; a failed check changes nothing.
+ *   Sec. 4.4      capture/replay with a caller->graph wait and a graph->caller completion event on every call.
+ *   Invariants 1-4.
+ *
+ * Conventions
+ *   - Every function returns a qe_status (0 = QE_OK, negative = error).  Nothing throws, aborts or exits.
+ *     qe_last_error() returns a thread-local, human-readable message for the last failure on this thread.
+ *   - "dev" pointers are CUDA device pointers on the context's device; "host" pointers are ordinary host
+ *     memory.  The library never frees caller memory.  All device memory a layer uses lives in the workspace
+ *     the caller passes to qe_layer_create (size from qe_layer_workspace_bytes); the library itself allocates
+ *     no device memory.
+ *   - Tensors are dense row-major.  bf16 = IEEE bfloat16 bit patterns (2 bytes).  Tokens T, in-features K,
+ *     out-features N:  X[T,K], W[N,K], Y[T,N], dY[T,N], dX[T,K]; a gradient slice is [N,K] FP32 at
+ *     grad_buf + offset (offset in ELEMENTS).  T, K, N must be multiples of 128.
+ *   - Streams are cudaStream_t passed as void* (NULL = the legacy default stream).  Work is issued on the
+ *     context's own execution stream; each action first makes that stream wait on the caller's stream and
+ *     finally makes the caller's stream wait on the action's tail, so the caller may use its outputs on
+ *     `caller_stream` without further synchronisation (bidirectional completion).
+ *   - Device-side waits are bounded; if one expires the kernel sets a status word and returns.  The host reads
+ *     that word at qe_optimizer_boundary / qe_get_state and reports QE_ERR_TIMEOUT.
+ */
+#ifndef QE_H_
+#define QE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum qe_status {
+  QE_OK = 0,
+  QE_ERR_BAD_ARG = -1,      /* null pointer, index out of range, unknown enum value                           */
+  QE_ERR_SHAPE = -2,        /* T, K or N not a multiple of 128, zero, or beyond the supported range           */
+  QE_ERR_KEY_LIVE = -3,     /* forward: the same TapeKey already has a live tape (mapping must stay injective)*/
+  QE_ERR_POOL_FULL = -4,    /* forward: no free slot; an occupied slot is never pre-empted                    */
+  QE_ERR_STALE_CACHE = -5,  /* forward: e_C != e_W on a non-first forward ("cache refresh required")          */
+  QE_ERR_ABORTED = -6,      /* the step was aborted; the arena is unusable until qe_arena_rebuild             */
+  QE_ERR_STALE_REF = -7,    /* the reference's generation does not name the slot's live tape                  */
+  QE_ERR_KEY_MISMATCH = -8, /* the slot is live with that generation but under a different key               */
+  QE_ERR_EPOCH = -9,        /* caller's weight version, or the tape's epoch, differs from e_W                 */
+  QE_ERR_DUP_CONSUME = -10, /* dI (or dW) already consumed this tape                                          */
+  QE_ERR_ORDER = -11,       /* dW before dI; or first gradient write of an epoch is not microbatch 0          */
+  QE_ERR_DEST = -12,        /* destination null/misaligned/too small/not the bound one/aliasing another layer */
+  QE_ERR_DUP_WRITE = -13,   /* this microbatch already wrote its gradient in this epoch                       */
+  QE_ERR_PENDING = -14,     /* live tape at a quiescent point (optimizer boundary, checkpoint, rebuild)       */
+  QE_ERR_INCOMPLETE = -15,  /* optimizer boundary: some configured microbatch has not written its gradient    */
+  QE_ERR_CUDA = -16,        /* a CUDA runtime/driver call failed (message has the CUDA error string)          */
+  QE_ERR_TIMEOUT = -17,     /* a bounded device-side wait expired (device status word non-zero)               */
+  QE_ERR_WORKSPACE = -18,   /* workspace null, misaligned (256 B) or smaller than qe_layer_workspace_bytes    */
+  QE_ERR_UNSUPPORTED = -19  /* no sm_100 device, or a size beyond a stated maximum                            */
+} qe_status;
+
+typedef enum qe_exec_mode { QE_EXEC_EAGER = 0, QE_EXEC_GRAPH = 1 } qe_exec_mode;
+typedef enum qe_tensor_class { QE_CLASS_X = 0, QE_CLASS_W = 1, QE_CLASS_G = 2, QE_CLASS_Y = 3 } qe_tensor_class;
+typedef enum qe_fp8_format { QE_E4M3 = 0, QE_E5M2 = 1 } qe_fp8_format;
+
+#define QE_MAX_SLOTS 64u
+#define QE_MAX_MICROBATCHES 64u
+#define QE_MAX_HISTORY 4096u
+#define QE_INVALID_EPOCH UINT64_MAX
+
+/* ---- Eq. 1 / Eq. 2 ------------------------------------------------------------------------------------------- */
+typedef struct qe_tape_key { uint32_t epoch, stage, mb, unit, inv; } qe_tape_key; /* (e, s, m, u, i)              */
+typedef struct qe_tape_ref { uint32_t slot; uint32_t reserved; uint64_t gen; } qe_tape_ref; /* (p, g_p)          */
+/* The (K, R) pair carried on the saved-value edge (Sec. 4.2).  Returned by value, owned by the caller, meaningless
+ * after the slot is released: a later use fails with QE_ERR_STALE_REF and never touches the slot's new occupant. */
+typedef struct qe_tape { qe_tape_key key; uint32_t reserved; qe_tape_ref ref; } qe_tape;
+
+/* ================================================================================================================
+ * Contract core (host only; creates no CUDA context).  The layer calls use it internally with exactly these
+ * check/commit pairs; it is exported so that the contract can be exercised without a GPU (Table 3: the fault
+ * injections run in a process that initialises no CUDA context).
+ * ============================================================================================================== */
+typedef struct qe_contract qe_contract;
+typedef struct qe_registry qe_registry; /* gradient destinations bound this epoch by a group of layers (alias check) */
+
+int32_t qe_registry_create(qe_registry** out);
+int32_t qe_registry_destroy(qe_registry*);
+
+/* slots in [1, QE_MAX_SLOTS]; registry may be NULL (then only this layer's own rules are checked). */
+int32_t qe_contract_create(uint32_t slots, uint32_t stage, uint32_t unit, uint32_t inv, qe_registry* registry,
+                           qe_contract** out);
+int32_t qe_contract_destroy(qe_contract*);
+
+/* Forward (Algorithm 1, lines 2-4).  check: aborted? mb < 64? gen == e_W? cache fresh (or first forward of the
+ * epoch -> *refresh_out = 1)? key not live? free slot (lowest index -> *slot_out)?  commit: occupy the slot,
+ * g_p += 1, e_C <- e_W on refresh, token += 1; writes the tape. */
+int32_t qe_contract_forward_check(const qe_contract*, uint32_t mb, uint64_t gen, int32_t* refresh_out,
+                                  uint32_t* slot_out);
+int32_t qe_contract_forward_commit(qe_contract*, uint32_t mb, qe_tape* tape_out);
+/* Input gradient (lines 5-7).  check: generation, key, epoch, dI bit clear.  commit: set dI bit, token += 1. */
+int32_t qe_contract_dI_check(const qe_contract*, const qe_tape*);
+int32_t qe_contract_dI_commit(qe_contract*, const qe_tape*);
+/* Weight gradient (lines 8-11).  dest_addr = address of element 0 of the flat buffer, as an integer.  check:
+ * resolve; dW bit clear; dI bit set; destination valid (non-null, dest_addr + 4*offset 16-byte aligned,
+ * offset + slice_elems <= dest_elems, equal to the destination bound this epoch, no overlap with another
+ * layer's bound slice); this microbatch has not written; the first write of the epoch is microbatch 0.
+ * *accumulate_out = 0 for the first write of the epoch (overwrite), 1 afterwards.  commit: bind destination, set
+ * mask bit and dW bit, release the slot (generation kept). */
+int32_t qe_contract_dW_check(const qe_contract*, const qe_tape*, uint64_t dest_addr, uint64_t dest_elems,
+                             uint64_t offset, uint64_t slice_elems, int32_t* accumulate_out);
+int32_t qe_contract_dW_commit(qe_contract*, const qe_tape*, uint64_t dest_addr, uint64_t offset,
+                              uint64_t slice_elems);
+/* Optimizer commit (lines 13-14): no live tape (else PENDING), every microbatch in [0, expected) wrote exactly
+ * once (else INCOMPLETE); then e_W += 1, mask cleared, next forward refreshes the cache. */
+int32_t qe_contract_boundary(qe_contract*, uint32_t microbatches_expected);
+/* Failure boundary (Sec. 4.5): purge this epoch's tapes (generations kept), mark the arena unusable. */
+int32_t qe_contract_abort(qe_contract*);
+/* Make the arena usable again after an abort; the epoch restarts with nothing written (PENDING if a tape lives). */
+int32_t qe_contract_rebuild(qe_contract*);
+/* Mark the quantised-weight cache stale (e_C <- invalid). */
+int32_t qe_contract_invalidate_cache(qe_contract*);
+/* Invariant 4: QE_OK only when no tape is live ("checkpoint withheld" otherwise -> PENDING). */
+int32_t qe_contract_checkpoint_check(const qe_contract*);
+
+typedef struct qe_slot_view { uint64_t gen; uint32_t live; uint32_t bits; qe_tape_key key; uint32_t reserved; } qe_slot_view;
+typedef struct qe_contract_view {
+  uint64_t e_W, e_C, token, write_mask;
+  uint32_t fwd_in_epoch, aborted, slots, live_tapes;
+  qe_slot_view slot[QE_MAX_SLOTS];
+} qe_contract_view;
+int32_t qe_contract_get(const qe_contract*, qe_contract_view* out);
+
+/* ================================================================================================================
+ * Layer API (CUDA, sm_100a)
+ * ============================================================================================================== */
+typedef struct qe_ctx qe_ctx;
+typedef struct qe_layer qe_layer;
+
+typedef struct qe_ctx_config {
+  uint32_t exec_mode; /* qe_exec_mode: launch kernels one by one, or replay one prebuilt CUDA graph per (action, slot) */
+  int32_t device;     /* CUDA device ordinal                                                                           */
+  uint32_t reserved[6];
+} qe_ctx_config;
+
+typedef struct qe_layer_config {
+  uint32_t T, K, N;       /* tokens, in-features, out-features: multiples of 128                             */
+  uint32_t history_len;   /* H in [1, QE_MAX_HISTORY]                                                        */
+  int32_t margin;         /* scale = fp8_max / max(history) / 2^margin; margin in [-32, 32]                  */
+  uint32_t slots;         /* tape slots P in [1, QE_MAX_SLOTS]                                               */
+  uint32_t stage, unit, inv; /* s, u, i of Eq. 1                                                             */
+  uint32_t reserved0;
+  const void* weight_dev; /* bf16 W[N,K]; caller-owned; read on the first forward of every epoch             */
+  uint64_t reserved1[4];
+} qe_layer_config;
+
+int32_t qe_ctx_create(const qe_ctx_config*, qe_ctx** out);
+int32_t qe_ctx_destroy(qe_ctx*);
+int32_t qe_layer_workspace_bytes(const qe_layer_config*, uint64_t* bytes_out);
+/* workspace_dev: 256-byte aligned device memory of at least qe_layer_workspace_bytes; owned by the caller, must
+ * outlive the layer.  The call zero-initialises the state in it (histories 0, scales 1) on the execution stream. */
+int32_t qe_layer_create(qe_ctx*, const qe_layer_config*, void* workspace_dev, uint64_t workspace_bytes,
+                        qe_layer** out);
+int32_t qe_layer_destroy(qe_layer*);
+
+/* F (Eq. 3).  x_dev bf16 [T,K] in, y_dev bf16 [T,N] out.  `gen` is the caller's view of the weight version and must
+ * equal e_W.  On the first forward of an epoch the weight is re-quantised (E4M3, plus its transpose) and its amax
+ * committed.  Then: X quantised to E4M3 with the current scale (amax taken in the same pass; the inverse scale is
+ * snapshotted into the tape slot), Y = bf16((Xq Wq^T) * sinv_X * sinv_W) on the tensor cores with max|Y| reduced in
+ * the epilogue, and the X and Y histories/scales updated.  *tape_out names the retained work. */
+int32_t qe_forward(qe_layer*, uint32_t mb, uint64_t gen, const void* x_dev, void* y_dev, void* caller_stream,
+                   qe_tape* tape_out);
+/* dI (Eq. 4).  dy_dev bf16 [T,N] in, dx_dev bf16 [T,K] out.  Quantises dY to E5M2 (and its transpose, retained for
+ * dW), dX = bf16((Gq Wq) * sinv_G * sinv_W), commits the gradient amax/scale once. */
+int32_t qe_backward_dI(qe_layer*, const qe_tape*, const void* dy_dev, void* dx_dev, void* caller_stream);
+/* dW (Eq. 5) with direct gradient placement (Sec. 3.4).  D = (Gq^T Xq) * sinv_G * sinv_X using the inverse scales
+ * snapshotted in the tape; grad_buf_dev[offset + n*K + k] = D (first write of the epoch) or += D (FP32, in place,
+ * one owner thread per element: deterministic).  No staging copy, no scale-state change. */
+int32_t qe_backward_dW(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t grad_buf_elems, uint64_t offset,
+                       void* caller_stream);
+/* The copied-gradient comparison path of Sec. 3.4: same checks and the same final values, but D is first written
+ * to temp_dev (FP32 [N,K], caller-owned scratch) and then added into the destination by a second kernel. */
+int32_t qe_backward_dW_staged(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t grad_buf_elems,
+                              uint64_t offset, float* temp_dev, void* caller_stream);
+/* Optimizer boundary: waits for the execution stream, reads the device status word, then applies
+ * qe_contract_boundary (bumping the weight version so that the next forward refreshes the cache). */
+int32_t qe_optimizer_boundary(qe_layer*, uint32_t microbatches_expected);
+/* The scale update as a standalone call: push *amax_dev (one FP32 on the device) into the class's history ring and
+ * recompute scale = fp8_max / max(history) / 2^margin and its inverse (unchanged if the maximum is 0 or not
+ * finite; +Inf clamps to FLT_MAX).  Same kernel F and dI use.  Does not advance the effect token. */
+int32_t qe_scale_commit(qe_layer*, uint32_t tensor_class, const float* amax_dev, void* caller_stream);
+int32_t qe_abort_step(qe_layer*);
+int32_t qe_arena_rebuild(qe_layer*);
+int32_t qe_invalidate_cache(qe_layer*);
+/* Slot the next successful qe_forward will occupy (lowest free index), or QE_ERR_POOL_FULL. */
+int32_t qe_next_slot(const qe_layer*, uint32_t* slot_out);
+
+typedef struct qe_class_state {
+  float scale, scale_inv;
+  uint32_t count;      /* commits so far */
+  uint32_t reserved;
+} qe_class_state;
+typedef struct qe_state_view {
+  qe_class_state cls[4];       /* indexed by qe_tensor_class                                                   */
+  float cache_sinv_W;          /* inverse weight scale snapshotted when the cache was last refreshed           */
+  uint32_t device_status;      /* 0 = clean                                                                    */
+  uint64_t device_token;       /* effect token as counted on the device (F and dI kernels' commits)            */
+  qe_contract_view contract;   /* host-side bookkeeping (its token must equal device_token)                    */
+} qe_state_view;
+/* Synchronises the execution stream and copies the state out.  window_out (host, may be NULL): 4*H floats, class c's
+ * history at [c*H, (c+1)*H) as a logical window, newest first.  slot_sinv_out (host, may be NULL): 2*P floats,
+ * sinv_X of slot p at [p], sinv_G at [P+p]. */
+int32_t qe_get_state(qe_layer*, qe_state_view* out, float* window_out, float* slot_sinv_out);
+/* Copies a slot's retained FP8 bytes to host memory (testing aid; synchronises).  which: 0 = Xq [T,K],
+ * 1 = Xq^T [K,T], 2 = Gq [T,N], 3 = Gq^T [N,T], 4 = Wq [N,K] (slot ignored), 5 = Wq^T [K,N] (slot ignored). */
+int32_t qe_read_fp8(qe_layer*, uint32_t which, uint32_t slot, void* host_out, uint64_t bytes);
+
+typedef struct qe_stats {
+  uint64_t graphs_built, graph_replays, eager_launches, handoffs, node_param_updates;
+  uint64_t kernels_launched;   /* kernels of this library enqueued (eager launches + kernel nodes replayed)   */
+  double capture_host_ms;      /* host time spent building graphs                                             */
+  uint64_t workspace_bytes;    /* sum over live layers                                                        */
+} qe_stats;
+int32_t qe_get_stats(const qe_ctx*, qe_stats* out);
+
+/* ================================================================================================================
+ * Standalone kernels of the path (no layer state; everything on `stream`)
+ * ============================================================================================================== */
+/* Fused cast: q[r,c] = fp8_rne_satfinite(fp32(x[r,c]) * *scale_dev); optional transposed copy qT[c,r]; optional
+ * amax: *amax_dev = max(*amax_dev, max|x|) (atomic max on the non-negative FP32 bit pattern -- zero it first for a
+ * fresh maximum).  rows and cols multiples of 64.  x bf16; q, qT bytes.  qT_dev and amax_dev may be NULL. */
+int32_t qe_quantize(const void* x_dev, uint32_t rows, uint32_t cols, const float* scale_dev, uint32_t fp8_format,
+                    void* q_dev, void* qT_dev, float* amax_dev, void* stream);
+/* max|x| over n bf16 values, two passes without atomics: per-block partial maxima into partials_dev (FP32, at least
+ * qe_amax_partials() entries, scratch owned by the caller), then a final block writes *amax_dev.  n multiple of 8. */
+int32_t qe_amax(const void* x_dev, uint64_t n, float* partials_dev, float* amax_dev, void* stream);
+uint32_t qe_amax_partials(void);
+/* dst[i] (=|+=) src[i] in FP32 (the second half of the copied-gradient path).  n multiple of 4, 16-byte aligned. */
+int32_t qe_accumulate(float* dst_dev, const float* src_dev, uint64_t n, int32_t accumulate, void* stream);
+/* One FP8 GEMM on the tensor cores: D[m,n] = (sum_k A[m,k] B[n,k]) * *alpha_a_dev * *alpha_b_dev with A [M,Kc] and
+ * B [Nn,Kc] both contraction-major bytes.  out_kind 0: bf16 D (amax_dev optional, as in qe_quantize); 1: FP32
+ * D overwrite; 2: FP32 D accumulate.  M, Nn, Kc multiples of 128.  status_dev: one uint32 the kernel ORs error
+ * bits into (caller zeroes it). */
+int32_t qe_gemm_fp8(const void* a_dev, uint32_t a_format, const void* b_dev, uint32_t b_format, uint32_t M,
+                    uint32_t Nn, uint32_t Kc, const float* alpha_a_dev, const float* alpha_b_dev, void* d_dev,
+                    uint32_t out_kind, float* amax_dev, uint32_t* status_dev, void* stream);
+
+const char* qe_last_error(void);
+const char* qe_status_name(int32_t status);
+/* Version of this ABI (bumped on incompatible change). */
+uint32_t qe_abi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QE_H_ */

@@ -1,0 +1,396 @@
+"""ctypes binding over libqe.so: the same entry points as include/qe.h, argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels.  There is no fallback: if the shared
+library is missing the import fails, and every call raises QEError on a negative status.
+
+torch tensors are accepted wherever the C signature takes a device pointer (their data_ptr() is
+passed); streams default to torch's current CUDA stream.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqe.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} not found: build it with `python -m paper_2609_23536_b200.build` "
+        "(this package has no CPU or PyTorch fallback)"
+    )
+lib = C.CDLL(LIB_PATH)
+
+QE_MAX_SLOTS = 64
+QE_INVALID_EPOCH = (1 << 64) - 1
+EAGER, GRAPH = 0, 1
+CLASS_X, CLASS_W, CLASS_G, CLASS_Y = 0, 1, 2, 3
+CLASS_NAMES = ("X", "W", "G", "Y")
+E4M3, E5M2 = 0, 1
+
+
+class qe_tape_key(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("epoch", "stage", "mb", "unit", "inv")]
+
+
+class qe_tape_ref(C.Structure):
+    _fields_ = [("slot", C.c_uint32), ("reserved", C.c_uint32), ("gen", C.c_uint64)]
+
+
+class qe_tape(C.Structure):
+    _fields_ = [("key", qe_tape_key), ("reserved", C.c_uint32), ("ref", qe_tape_ref)]
+
+    def astuple(self):
+        k, r = self.key, self.ref
+        return ((k.epoch, k.stage, k.mb, k.unit, k.inv), (r.slot, r.gen))
+
+
+class qe_slot_view(C.Structure):
+    _fields_ = [("gen", C.c_uint64), ("live", C.c_uint32), ("bits", C.c_uint32), ("key", qe_tape_key), ("reserved", C.c_uint32)]
+
+
+class qe_contract_view(C.Structure):
+    _fields_ = [
+        ("e_W", C.c_uint64), ("e_C", C.c_uint64), ("token", C.c_uint64), ("write_mask", C.c_uint64),
+        ("fwd_in_epoch", C.c_uint32), ("aborted", C.c_uint32), ("slots", C.c_uint32), ("live_tapes", C.c_uint32),
+        ("slot", qe_slot_view * QE_MAX_SLOTS),
+    ]
+
+
+class qe_ctx_config(C.Structure):
+    _fields_ = [("exec_mode", C.c_uint32), ("device", C.c_int32), ("reserved", C.c_uint32 * 6)]
+
+
+class qe_layer_config(C.Structure):
+    _fields_ = [
+        ("T", C.c_uint32), ("K", C.c_uint32), ("N", C.c_uint32), ("history_len", C.c_uint32), ("margin", C.c_int32),
+        ("slots", C.c_uint32), ("stage", C.c_uint32), ("unit", C.c_uint32), ("inv", C.c_uint32), ("reserved0", C.c_uint32),
+        ("weight_dev", C.c_void_p), ("reserved1", C.c_uint64 * 4),
+    ]
+
+
+class qe_class_state(C.Structure):
+    _fields_ = [("scale", C.c_float), ("scale_inv", C.c_float), ("count", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class qe_state_view(C.Structure):
+    _fields_ = [
+        ("cls", qe_class_state * 4), ("cache_sinv_W", C.c_float), ("device_status", C.c_uint32),
+        ("device_token", C.c_uint64), ("contract", qe_contract_view),
+    ]
+
+
+class qe_stats(C.Structure):
+    _fields_ = [
+        ("graphs_built", C.c_uint64), ("graph_replays", C.c_uint64), ("eager_launches", C.c_uint64),
+        ("handoffs", C.c_uint64), ("node_param_updates", C.c_uint64), ("kernels_launched", C.c_uint64),
+        ("capture_host_ms", C.c_double), ("workspace_bytes", C.c_uint64),
+    ]
+
+    def asdict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+# every symbol include/qe.h declares, with its signature
+_P = C.c_void_p
+_SIGNATURES = {
+    "qe_registry_create": (C.c_int32, [C.POINTER(_P)]),
+    "qe_registry_destroy": (C.c_int32, [_P]),
+    "qe_contract_create": (C.c_int32, [C.c_uint32] * 4 + [_P, C.POINTER(_P)]),
+    "qe_contract_destroy": (C.c_int32, [_P]),
+    "qe_contract_forward_check": (C.c_int32, [_P, C.c_uint32, C.c_uint64, C.POINTER(C.c_int32), C.POINTER(C.c_uint32)]),
+    "qe_contract_forward_commit": (C.c_int32, [_P, C.c_uint32, C.POINTER(qe_tape)]),
+    "qe_contract_dI_check": (C.c_int32, [_P, C.POINTER(qe_tape)]),
+    "qe_contract_dI_commit": (C.c_int32, [_P, C.POINTER(qe_tape)]),
+    "qe_contract_dW_check": (C.c_int32, [_P, C.POINTER(qe_tape), C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64, C.POINTER(C.c_int32)]),
+    "qe_contract_dW_commit": (C.c_int32, [_P, C.POINTER(qe_tape), C.c_uint64, C.c_uint64, C.c_uint64]),
+    "qe_contract_boundary": (C.c_int32, [_P, C.c_uint32]),
+    "qe_contract_abort": (C.c_int32, [_P]),
+    "qe_contract_rebuild": (C.c_int32, [_P]),
+    "qe_contract_invalidate_cache": (C.c_int32, [_P]),
+    "qe_contract_checkpoint_check": (C.c_int32, [_P]),
+    "qe_contract_get": (C.c_int32, [_P, C.POINTER(qe_contract_view)]),
+    "qe_ctx_create": (C.c_int32, [C.POINTER(qe_ctx_config), C.POINTER(_P)]),
+    "qe_ctx_destroy": (C.c_int32, [_P]),
+    "qe_layer_workspace_bytes": (C.c_int32, [C.POINTER(qe_layer_config), C.POINTER(C.c_uint64)]),
+    "qe_layer_create": (C.c_int32, [_P, C.POINTER(qe_layer_config), _P, C.c_uint64, C.POINTER(_P)]),
+    "qe_layer_destroy": (C.c_int32, [_P]),
+    "qe_forward": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
+    "qe_backward_dI": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
+    "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
+    "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
+    "qe_optimizer_boundary": (C.c_int32, [_P, C.c_uint32]),
+    "qe_scale_commit": (C.c_int32, [_P, C.c_uint32, _P, _P]),
+    "qe_abort_step": (C.c_int32, [_P]),
+    "qe_arena_rebuild": (C.c_int32, [_P]),
+    "qe_invalidate_cache": (C.c_int32, [_P]),
+    "qe_next_slot": (C.c_int32, [_P, C.POINTER(C.c_uint32)]),
+    "qe_get_state": (C.c_int32, [_P, C.POINTER(qe_state_view), _P, _P]),
+    "qe_read_fp8": (C.c_int32, [_P, C.c_uint32, C.c_uint32, _P, C.c_uint64]),
+    "qe_get_stats": (C.c_int32, [_P, C.POINTER(qe_stats)]),
+    "qe_quantize": (C.c_int32, [_P, C.c_uint32, C.c_uint32, _P, C.c_uint32, _P, _P, _P, _P]),
+    "qe_amax": (C.c_int32, [_P, C.c_uint64, _P, _P, _P]),
+    "qe_amax_partials": (C.c_uint32, []),
+    "qe_accumulate": (C.c_int32, [_P, _P, C.c_uint64, C.c_int32, _P]),
+    "qe_gemm_fp8": (C.c_int32, [_P, C.c_uint32, _P, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, _P, _P, _P, C.c_uint32, _P, _P, _P]),
+    "qe_last_error": (C.c_char_p, []),
+    "qe_status_name": (C.c_char_p, [C.c_int32]),
+    "qe_abi_version": (C.c_uint32, []),
+}
+for _name, (_res, _args) in _SIGNATURES.items():
+    _fn = getattr(lib, _name)  # AttributeError here = the library does not export what the header declares
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class QEError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        name = lib.qe_status_name(status).decode()
+        self.code = name[len("QE_ERR_"):] if name.startswith("QE_ERR_") else name
+        super().__init__(lib.qe_last_error().decode() or name)
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        raise QEError(status)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream or None
+    return stream or None
+
+
+# ---------------------------------------------------------------------------------------- contract core (host only)
+class Contract:
+    """qe_contract_* with check+commit exposed separately; no CUDA involved."""
+
+    def __init__(self, slots, stage=0, unit=0, inv=0, registry=None):
+        self.h = _P()
+        self.registry = registry
+        _check(lib.qe_contract_create(slots, stage, unit, inv, registry.h if registry else None, C.byref(self.h)))
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            lib.qe_contract_destroy(self.h)
+            self.h = None
+
+    def forward_check(self, mb, gen):
+        r, p = C.c_int32(), C.c_uint32()
+        _check(lib.qe_contract_forward_check(self.h, mb, gen, C.byref(r), C.byref(p)))
+        return bool(r.value), p.value
+
+    def forward_commit(self, mb) -> qe_tape:
+        t = qe_tape()
+        _check(lib.qe_contract_forward_commit(self.h, mb, C.byref(t)))
+        return t
+
+    def dI_check(self, tape):
+        _check(lib.qe_contract_dI_check(self.h, C.byref(tape)))
+
+    def dI_commit(self, tape):
+        _check(lib.qe_contract_dI_commit(self.h, C.byref(tape)))
+
+    def dW_check(self, tape, dest_addr, dest_elems, offset, slice_elems) -> bool:
+        a = C.c_int32()
+        _check(lib.qe_contract_dW_check(self.h, C.byref(tape), dest_addr, dest_elems, offset, slice_elems, C.byref(a)))
+        return bool(a.value)
+
+    def dW_commit(self, tape, dest_addr, offset, slice_elems):
+        _check(lib.qe_contract_dW_commit(self.h, C.byref(tape), dest_addr, offset, slice_elems))
+
+    def boundary(self, expected):
+        _check(lib.qe_contract_boundary(self.h, expected))
+
+    def abort(self):
+        _check(lib.qe_contract_abort(self.h))
+
+    def rebuild(self):
+        _check(lib.qe_contract_rebuild(self.h))
+
+    def invalidate_cache(self):
+        _check(lib.qe_contract_invalidate_cache(self.h))
+
+    def checkpoint_check(self):
+        _check(lib.qe_contract_checkpoint_check(self.h))
+
+    def get(self) -> dict:
+        v = qe_contract_view()
+        _check(lib.qe_contract_get(self.h, C.byref(v)))
+        return contract_view_to_dict(v)
+
+
+class Registry:
+    def __init__(self):
+        self.h = _P()
+        _check(lib.qe_registry_create(C.byref(self.h)))
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            lib.qe_registry_destroy(self.h)
+            self.h = None
+
+
+def contract_view_to_dict(v: qe_contract_view) -> dict:
+    slots = []
+    for p in range(v.slots):
+        s = v.slot[p]
+        k = s.key
+        slots.append({"gen": s.gen, "live": bool(s.live), "bits": s.bits,
+                      "key": (k.epoch, k.stage, k.mb, k.unit, k.inv) if s.live else None})
+    return {"e_W": v.e_W, "e_C": v.e_C, "token": v.token, "write_mask": v.write_mask,
+            "fwd_in_epoch": v.fwd_in_epoch, "aborted": bool(v.aborted), "slots": slots}
+
+
+# ---------------------------------------------------------------------------------------- layer API
+class Context:
+    def __init__(self, exec_mode=EAGER, device=0):
+        cfg = qe_ctx_config(exec_mode=exec_mode, device=device)
+        self.h = _P()
+        _check(lib.qe_ctx_create(C.byref(cfg), C.byref(self.h)))
+        self.exec_mode = exec_mode
+
+    def stats(self) -> dict:
+        s = qe_stats()
+        _check(lib.qe_get_stats(self.h, C.byref(s)))
+        return s.asdict()
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib.qe_ctx_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
+
+
+class Layer:
+    """One FP8 delayed-scaling linear.  Holds the torch-allocated workspace and the weight tensor alive."""
+
+    def __init__(self, ctx: Context, T, K, N, H, margin, slots, weight, stage=0, unit=0, inv=0):
+        import torch
+
+        assert weight.dtype == torch.bfloat16 and weight.is_cuda and weight.is_contiguous() and tuple(weight.shape) == (N, K)
+        self.ctx, self.T, self.K, self.N, self.H, self.P = ctx, T, K, N, H, slots
+        self.weight = weight
+        self.cfg = qe_layer_config(T=T, K=K, N=N, history_len=H, margin=margin, slots=slots, stage=stage, unit=unit,
+                                   inv=inv, weight_dev=weight.data_ptr())
+        nbytes = C.c_uint64()
+        _check(lib.qe_layer_workspace_bytes(C.byref(self.cfg), C.byref(nbytes)))
+        self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=weight.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.h = _P()
+        _check(lib.qe_layer_create(ctx.h, C.byref(self.cfg), base, nbytes.value, C.byref(self.h)))
+
+    # the five calls of the path
+    def forward(self, mb, gen, x, y, stream=None) -> qe_tape:
+        t = qe_tape()
+        _check(lib.qe_forward(self.h, mb, gen, _ptr(x), _ptr(y), _stream(stream), C.byref(t)))
+        return t
+
+    def backward_dI(self, tape, dy, dx, stream=None):
+        _check(lib.qe_backward_dI(self.h, C.byref(tape), _ptr(dy), _ptr(dx), _stream(stream)))
+
+    def backward_dW(self, tape, grad_buf, offset, stream=None):
+        _check(lib.qe_backward_dW(self.h, C.byref(tape), _ptr(grad_buf), grad_buf.numel(), offset, _stream(stream)))
+
+    def backward_dW_staged(self, tape, grad_buf, offset, temp, stream=None):
+        _check(lib.qe_backward_dW_staged(self.h, C.byref(tape), _ptr(grad_buf), grad_buf.numel(), offset, _ptr(temp), _stream(stream)))
+
+    def optimizer_boundary(self, expected):
+        _check(lib.qe_optimizer_boundary(self.h, expected))
+
+    def scale_commit(self, cls, amax_dev, stream=None):
+        _check(lib.qe_scale_commit(self.h, cls, _ptr(amax_dev), _stream(stream)))
+
+    def abort_step(self):
+        _check(lib.qe_abort_step(self.h))
+
+    def arena_rebuild(self):
+        _check(lib.qe_arena_rebuild(self.h))
+
+    def invalidate_cache(self):
+        _check(lib.qe_invalidate_cache(self.h))
+
+    def next_slot(self) -> int:
+        p = C.c_uint32()
+        _check(lib.qe_next_slot(self.h, C.byref(p)))
+        return p.value
+
+    def state(self) -> dict:
+        """Same shape as the oracle's state(): bit-comparable."""
+        v = qe_state_view()
+        win = np.zeros(4 * self.H, np.float32)
+        sinv = np.zeros(2 * self.P, np.float32)
+        _check(lib.qe_get_state(self.h, C.byref(v), win.ctypes.data, sinv.ctypes.data))
+        d = contract_view_to_dict(v.contract)
+        d["classes"] = {
+            CLASS_NAMES[c]: {
+                "window": win[c * self.H:(c + 1) * self.H].copy(),
+                "scale": np.float32(v.cls[c].scale),
+                "scale_inv": np.float32(v.cls[c].scale_inv),
+                "count": v.cls[c].count,
+            }
+            for c in range(4)
+        }
+        d["cache_sinv_W"] = np.float32(v.cache_sinv_W)
+        d["device_status"] = v.device_status
+        d["device_token"] = v.device_token
+        d["slot_sinv_X"] = sinv[: self.P].copy()
+        d["slot_sinv_G"] = sinv[self.P:].copy()
+        return d
+
+    def read_fp8(self, which: int, slot: int = 0) -> np.ndarray:
+        shape = {0: (self.T, self.K), 1: (self.K, self.T), 2: (self.T, self.N), 3: (self.N, self.T),
+                 4: (self.N, self.K), 5: (self.K, self.N)}[which]
+        out = np.empty(shape, np.uint8)
+        _check(lib.qe_read_fp8(self.h, which, slot, out.ctypes.data, out.size))
+        return out
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib.qe_layer_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
+
+
+# ---------------------------------------------------------------------------------------- standalone kernels
+def qe_quantize(x, scale_dev, fmt, q, qT=None, amax_dev=None, stream=None):
+    rows, cols = x.shape
+    _check(lib.qe_quantize(_ptr(x), rows, cols, _ptr(scale_dev), fmt, _ptr(q), _ptr(qT), _ptr(amax_dev), _stream(stream)))
+
+
+def qe_amax_partials() -> int:
+    return lib.qe_amax_partials()
+
+
+def qe_amax(x, partials_dev, amax_dev, stream=None):
+    _check(lib.qe_amax(_ptr(x), x.numel(), _ptr(partials_dev), _ptr(amax_dev), _stream(stream)))
+
+
+def qe_accumulate(dst, src, accumulate: bool, stream=None):
+    _check(lib.qe_accumulate(_ptr(dst), _ptr(src), dst.numel(), int(accumulate), _stream(stream)))
+
+
+def qe_gemm_fp8(a, a_fmt, b, b_fmt, alpha_a_dev, alpha_b_dev, d, out_kind, amax_dev=None, status_dev=None, stream=None):
+    M, Kc = a.shape
+    Nn, Kc2 = b.shape
+    assert Kc == Kc2
+    _check(lib.qe_gemm_fp8(_ptr(a), a_fmt, _ptr(b), b_fmt, M, Nn, Kc, _ptr(alpha_a_dev), _ptr(alpha_b_dev), _ptr(d),
+                           out_kind, _ptr(amax_dev), _ptr(status_dev), _stream(stream)))

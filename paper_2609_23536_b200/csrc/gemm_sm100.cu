@@ -1,0 +1,337 @@
+// FP8 GEMM for sm_100a: D[M,N] = (A[M,Kc] . B[N,Kc]^T) * alpha, A and B contraction-major bytes (E4M3 or E5M2,
+// mixed freely), FP32 accumulation in tensor memory.
+//
+// Structure (one persistent CTA per SM, 192 threads):
+//   warp 0      TMA producer: cp.async.bulk.tensor 2D tiles (128-byte swizzle) into a 4-stage shared-memory ring
+//   warp 1      allocates tensor memory, then one lane issues tcgen05.mma (128 x 256 x 32 per instruction) and
+//               tcgen05.commit to release ring stages / publish a finished accumulator
+//   warps 2-5   epilogue: tcgen05.ld the 128 x 256 FP32 accumulator (each warp its own 32-lane quadrant), scale,
+//               and write bf16 (+ max|D| reduced by warp shuffles, one atomicMax per warp and tile), or FP32
+//               overwrite, or FP32 read-modify-write straight into the destination (direct gradient placement)
+// Two accumulators (2 x 256 tensor-memory columns) let the epilogue of tile i overlap the main loop of tile i+1.
+// Each output element is produced by exactly one thread with a fixed contraction order, so results do not depend
+// on the grid size or on how tiles are scheduled (no split-K, no atomics on data).
+//
+// Every wait on an mbarrier is bounded by a clock budget; on expiry the thread ORs an error bit into the status
+// word, raises a CTA-wide abort flag that all other waits observe, and the CTA falls through to its common exit
+// where tensor memory is released.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+
+namespace qe {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 128;  // BK bytes = FP8 elements per stage along the contraction
+constexpr int STAGES = 4;
+constexpr int UMMA_K = 32;
+constexpr uint32_t A_BYTES = BM * BK, B_BYTES = BN * BK, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr int THREADS = 192;
+constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;  // ~2 s at the maximum SM clock
+
+constexpr uint32_t ERR_PRODUCER = 1u, ERR_MMA = 2u, ERR_EPILOGUE = 4u;
+
+// ------------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the budget ran out or another thread of the CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status, uint32_t err_bit) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
+      *abort_flag = 1u;
+      atomicOr(status, err_bit);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor for a contraction-major tile whose rows are 128 bytes, 128-byte swizzle:
+// start address (>>4) in bits 0-13; leading byte offset (unused for this layout) 1 in bits 16-29; stride byte
+// offset = 1024 (eight 128-byte rows) >>4 in bits 32-45; descriptor version 1 in bits 46-47; swizzle mode 2
+// (128 B) in bits 61-63.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);  // .x = a in the low half
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Tile order: m fastest, so that the CTAs running at the same time share a few B tiles and all of A through L2.
+__device__ __forceinline__ void tile_coords(uint32_t tile, uint32_t tiles_m, uint32_t& m0, uint32_t& n0) {
+  m0 = (tile % tiles_m) * BM;
+  n0 = (tile / tiles_m) * BN;
+}
+
+// ------------------------------------------------------------------------------------------------ kernel
+__global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], then tmem address + abort flag
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tiles_m = p.M / BM, tiles_n = (p.N + BN - 1) / BN;
+  const uint32_t num_tiles = tiles_m * tiles_n;
+  const uint32_t num_kb = p.Kc / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);
+    }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (uint32_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        uint32_t m0, n0;
+        tile_coords(tile, tiles_m, m0, n0);
+        for (uint32_t kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, ERR_PRODUCER))) break;
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_BYTES;
+          tma_load_2d(a_dst, &p.tmA, full_bar(s), (int)(kb * BK), (int)m0);
+          tma_load_2d(b_dst, &p.tmB, full_bar(s), (int)(kb * BK), (int)n0);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // give copies already in flight a bounded chance to land before the CTA's shared memory goes away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) { }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0, acc = 0, acc_ph = 0;
+      bool ok = true;
+      for (uint32_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, ERR_MMA))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
+        for (uint32_t kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, p.status, ERR_MMA))) break;
+          tc_fence_after();
+          const uint32_t a_src = smem_base + s * STAGE_BYTES, b_src = a_src + A_BYTES;
+          const uint64_t adesc = make_desc(a_src), bdesc = make_desc(b_src);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advancing 32 bytes along the contraction inside the 128-byte swizzle row: +2 in the address field
+            tc_mma_f8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | (uint32_t)k) != 0u);
+          }
+          tc_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));  // accumulator complete
+        if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 2..5)
+    const uint32_t quad = (uint32_t)warp & 3u;  // tensor-memory lane quadrant this warp may read
+    const float alpha = __fmul_rn(*p.alpha_a, *p.alpha_b);
+    uint32_t acc = 0, acc_ph = 0;
+    bool ok = true;
+    for (uint32_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      uint32_t m0, n0;
+      tile_coords(tile, tiles_m, m0, n0);
+      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, ERR_EPILOGUE))) break;
+      tc_fence_after();
+      const uint32_t row = m0 + quad * 32u + (uint32_t)lane;
+      const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN;
+      uint32_t amax_bits = 0;
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        const uint32_t col = n0 + ch * 32u;
+        if (col >= p.N) break;  // ragged last column tile (N a multiple of 128 but not of 256); warp-uniform
+        uint32_t r[32];
+        tmem_ld32(t_row + ch * 32u, r);
+        tmem_ld_wait();
+        if (p.epi == 0) {
+          uint32_t o[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float a = __fmul_rn(__uint_as_float(r[2 * j]), alpha);
+            const float b = __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha);
+            o[j] = pack_bf16(a, b);
+            // magnitude of the rounded values actually stored, as FP32 bit patterns (bf16 bits << 16)
+            amax_bits = max(amax_bits, max((o[j] << 16) & 0x7fffffffu, o[j] & 0x7fff0000u));
+          }
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)row * p.ldo + col);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        } else {
+          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + (size_t)row * p.ldo + col);
+          if (p.epi == 2) {
+            float4 old[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) old[j] = dst[j];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float4 v;
+              v.x = __fadd_rn(old[j].x, __fmul_rn(__uint_as_float(r[4 * j]), alpha));
+              v.y = __fadd_rn(old[j].y, __fmul_rn(__uint_as_float(r[4 * j + 1]), alpha));
+              v.z = __fadd_rn(old[j].z, __fmul_rn(__uint_as_float(r[4 * j + 2]), alpha));
+              v.w = __fadd_rn(old[j].w, __fmul_rn(__uint_as_float(r[4 * j + 3]), alpha));
+              dst[j] = v;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float4 v;
+              v.x = __fmul_rn(__uint_as_float(r[4 * j]), alpha);
+              v.y = __fmul_rn(__uint_as_float(r[4 * j + 1]), alpha);
+              v.z = __fmul_rn(__uint_as_float(r[4 * j + 2]), alpha);
+              v.w = __fmul_rn(__uint_as_float(r[4 * j + 3]), alpha);
+              dst[j] = v;
+            }
+          }
+        }
+      }
+      // accumulator drained: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (p.epi == 0 && p.amax_bits) {
+        const uint32_t w = __reduce_max_sync(0xffffffffu, amax_bits);
+        if (lane == 0 && w) atomicMax(p.amax_bits, w);
+      }
+      if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace
+
+uint32_t gemm_idesc(int a_fmt, int b_fmt) {
+  // bits 4-5: accumulator format (1 = FP32); 7-9 / 10-12: A / B format (0 = E4M3, 1 = E5M2); 15 / 16: A / B major
+  // (0 = contraction-major); 17-22: N >> 3; 24-28: M >> 4.
+  return (1u << 4) | ((uint32_t)a_fmt << 7) | ((uint32_t)b_fmt << 10) | ((uint32_t)(BN >> 3) << 17) |
+         ((uint32_t)(BM >> 4) << 24);
+}
+
+cudaError_t gemm_prepare() {
+  return cudaFuncSetAttribute((const void*)gemm_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)SMEM_BYTES);
+}
+
+Launch make_gemm(const GemmParams& p, int num_sms) {
+  Launch l;
+  l.func = (const void*)gemm_fp8_kernel;
+  const uint32_t tiles = (p.M / BM) * ((p.N + BN - 1) / BN);
+  l.grid = dim3(tiles < (uint32_t)num_sms ? tiles : (uint32_t)num_sms, 1, 1);
+  l.block = dim3(THREADS, 1, 1);
+  l.smem = SMEM_BYTES;
+  l.set(p);
+  return l;
+}
+
+}  // namespace qe

@@ -1,0 +1,107 @@
+// Kernel parameter blocks and host-side launch descriptors shared by the execution layer.
+// Every kernel of the library takes exactly one by-value parameter struct, so that a launch is fully
+// described by (function, grid, block, dynamic shared memory, parameter bytes) and the same description
+// serves an eager launch, a CUDA-graph kernel node and a later in-place update of that node.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace qe {
+
+// ---- device-resident layer state (lives at the start of the caller's workspace) -------------------------------
+struct DevState {
+  float scale[4];              // indexed by qe_tensor_class
+  float scale_inv[4];
+  uint32_t count[4];           // commits so far
+  uint32_t pending_amax[4];    // non-negative FP32 bit patterns, accumulated with atomicMax, cleared by commit
+  unsigned long long token;    // effect token as counted on the device
+  float cache_sinv_W;          // inverse weight scale at the last cache refresh
+  uint32_t status;             // error bits ORed in by kernels whose bounded waits expired
+  float slot_sinv_X[64];       // inverse scales snapshotted when X_m / dY_m were quantised (per tape slot)
+  float slot_sinv_G[64];
+  uint32_t pad[44];            // header is 768 bytes; history rings [4][H] follow
+};
+static_assert(sizeof(DevState) == 768, "DevState layout");
+
+struct QuantParams {
+  const uint16_t* x;           // bf16 [rows, cols]
+  uint8_t* q;                  // fp8 [rows, cols]
+  uint8_t* qT;                 // fp8 [cols, rows] or null
+  uint32_t rows, cols;
+  const float* scale;          // device scalar read by every thread
+  const float* sinv_src;       // if non-null, block 0 copies *sinv_src to *sinv_dst (tape snapshot)
+  float* sinv_dst;
+  uint32_t* amax_bits;         // atomicMax target or null
+  int32_t fmt;                 // 0 = E4M3, 1 = E5M2
+};
+
+struct CommitParams {
+  DevState* st;
+  float* hist;                 // [4][H]
+  uint32_t H;
+  uint32_t class_mask;         // bit c set: commit class c from pending_amax[c] (or from amax_override)
+  float pow2_neg_margin;       // 2^-margin
+  const float* amax_override;  // if non-null: value to push for the single class in class_mask
+  uint32_t bump_token;         // 1 for F and dI, 0 for a standalone commit
+  uint32_t pad;
+};
+
+struct AmaxParams {
+  const uint4* x;              // bf16, 8 per vector
+  uint64_t nvec;
+  float* partials;
+  float* out;
+  uint32_t nparts;
+  uint32_t pad;
+};
+
+struct AccumParams {
+  float4* dst;
+  const float4* src;
+  uint64_t nvec;
+  int32_t accumulate;
+  int32_t pad;
+};
+
+struct GemmParams {
+  CUtensorMap tmA;             // A [M, Kc] bytes, box 128 x 128, 128-byte swizzle
+  CUtensorMap tmB;             // B [N, Kc] bytes, box 128 x 256
+  uint32_t M, N, Kc;
+  uint32_t idesc;              // tcgen05 instruction descriptor (formats, 128 x 256 shape)
+  const float* alpha_a;
+  const float* alpha_b;
+  void* out;                   // bf16 or FP32 [M, N], row pitch ldo elements
+  uint32_t ldo;
+  int32_t epi;                 // 0 bf16 (+amax), 1 FP32 overwrite, 2 FP32 accumulate
+  uint32_t* amax_bits;         // or null
+  uint32_t* status;
+};
+
+// One launch, self-contained.
+struct Launch {
+  const void* func = nullptr;
+  dim3 grid{1, 1, 1}, block{1, 1, 1};
+  uint32_t smem = 0;
+  uint32_t nbytes = 0;
+  alignas(64) unsigned char params[384];
+  template <class P>
+  void set(const P& p) {
+    static_assert(sizeof(P) <= sizeof(params), "parameter block too large");
+    nbytes = sizeof(P);
+    __builtin_memcpy(params, &p, sizeof(P));
+  }
+};
+
+Launch make_quantize(const QuantParams& p);
+Launch make_commit(const CommitParams& p);
+Launch make_amax_pass1(const AmaxParams& p);
+Launch make_amax_pass2(const AmaxParams& p);
+Launch make_accumulate(const AccumParams& p);
+Launch make_gemm(const GemmParams& p, int num_sms);
+cudaError_t gemm_prepare();  // opt in to the dynamic shared memory the GEMM needs (once per device)
+uint32_t gemm_idesc(int a_fmt, int b_fmt);
+constexpr uint32_t kAmaxPartials = 2048;
+
+}  // namespace qe

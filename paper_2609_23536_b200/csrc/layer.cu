@@ -1,0 +1,738 @@
+// Host side of the layer API: workspace carve-up, tensor maps, the three checked actions and the execution layer
+// (eager launches or one CUDA graph per (action, slot), both bracketed by the two-way stream handshake).
+#include <chrono>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "contract.h"
+#include "error.h"
+#include "kernels.h"
+#include "qe.h"
+
+using qe::fail;
+
+#define QE_CUDA(expr)                                                                         \
+  do {                                                                                        \
+    cudaError_t e_ = (expr);                                                                  \
+    if (e_ != cudaSuccess) return fail(QE_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceInfo {
+  bool ready = false;
+  int device = -1, num_sms = 0, cc_major = 0;
+  EncodeTiledFn encode = nullptr;
+};
+DeviceInfo g_dev[16];
+
+// Per-device one-time setup: SM count, compute capability, driver entry point for tensor-map encoding, and the
+// GEMM's shared-memory opt-in.  The device must be current.
+int32_t device_info(int device, DeviceInfo** out) {
+  if (device < 0 || device >= 16) return fail(QE_ERR_BAD_ARG, "device %d", device);
+  DeviceInfo& d = g_dev[device];
+  if (!d.ready) {
+    cudaDeviceProp prop;
+    QE_CUDA(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return fail(QE_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library needs sm_100", device, prop.major, prop.minor);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    QE_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return fail(QE_ERR_CUDA, "cuTensorMapEncodeTiled not available");
+    QE_CUDA(qe::gemm_prepare());
+    d.device = device;
+    d.num_sms = prop.multiProcessorCount;
+    d.cc_major = prop.major;
+    d.encode = (EncodeTiledFn)fn;
+    d.ready = true;
+  }
+  *out = &d;
+  return QE_OK;
+}
+
+// Tensor map over a contraction-major byte matrix [rows, inner]: box = 128 bytes x box_rows, 128-byte swizzle.
+int32_t make_map(const DeviceInfo* d, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t inner,
+                 uint32_t box_rows) {
+  cuuint64_t gdim[2] = {inner, rows};
+  cuuint64_t gstride[1] = {inner};
+  cuuint32_t box[2] = {128u, box_rows};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = d->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(QE_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
+  return QE_OK;
+}
+
+uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+bool shape_ok(uint32_t v) { return v >= 256 && v % 128 == 0 && v <= (1u << 20); }
+
+}  // namespace
+
+// ================================================================================================ execution layer
+struct ActionGraph {
+  bool built = false;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  std::vector<cudaGraphNode_t> nodes;
+  std::vector<qe::Launch> launches;
+};
+
+struct qe_ctx {
+  DeviceInfo* dev = nullptr;
+  uint32_t exec_mode = QE_EXEC_EAGER;
+  cudaStream_t exec_stream = nullptr;
+  cudaEvent_t ev_in = nullptr, ev_out = nullptr;
+  qe_registry* registry = nullptr;
+  qe_stats stats{};
+};
+
+struct qe_layer {
+  qe_ctx* ctx = nullptr;
+  qe_layer_config cfg{};
+  qe_contract* contract = nullptr;
+  uint64_t ws_bytes = 0;
+  qe::DevState* st = nullptr;
+  float* hist = nullptr;
+  uint8_t *Wq = nullptr, *WqT = nullptr;
+  uint8_t *Xq[QE_MAX_SLOTS], *XqT[QE_MAX_SLOTS], *Gq[QE_MAX_SLOTS], *GqT[QE_MAX_SLOTS];
+  // tensor maps: A-role boxes are 128 rows, B-role boxes 256 rows
+  CUtensorMap tmXq_A[QE_MAX_SLOTS], tmGq_A[QE_MAX_SLOTS], tmGqT_A[QE_MAX_SLOTS], tmXqT_B[QE_MAX_SLOTS];
+  CUtensorMap tmWq_B, tmWqT_B;
+  ActionGraph gF[QE_MAX_SLOTS], gDI[QE_MAX_SLOTS], gDW[QE_MAX_SLOTS], gDWs[QE_MAX_SLOTS], gRefresh, gCommit;
+};
+
+namespace {
+
+int32_t launch_eager(qe_ctx* ctx, const qe::Launch& l) {
+  void* args[1] = {const_cast<unsigned char*>(l.params)};
+  QE_CUDA(cudaLaunchKernel(l.func, l.grid, l.block, args, l.smem, ctx->exec_stream));
+  ctx->stats.eager_launches += 1;
+  ctx->stats.kernels_launched += 1;
+  return QE_OK;
+}
+
+// Capture the launches on the execution stream into a graph, instantiate it, and recover the kernel nodes in
+// launch order by walking the (linear) dependency chain from the root.
+int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls) {
+  const auto t0 = std::chrono::steady_clock::now();
+  QE_CUDA(cudaStreamBeginCapture(ctx->exec_stream, cudaStreamCaptureModeThreadLocal));
+  cudaError_t err = cudaSuccess;
+  for (const qe::Launch& l : ls) {
+    void* args[1] = {const_cast<unsigned char*>(l.params)};
+    err = cudaLaunchKernel(l.func, l.grid, l.block, args, l.smem, ctx->exec_stream);
+    if (err != cudaSuccess) break;
+  }
+  cudaGraph_t graph = nullptr;
+  cudaError_t end = cudaStreamEndCapture(ctx->exec_stream, &graph);
+  if (err != cudaSuccess) {
+    if (graph) cudaGraphDestroy(graph);
+    return fail(QE_ERR_CUDA, "launch during capture: %s", cudaGetErrorString(err));
+  }
+  QE_CUDA(end);
+  size_t n = 0;
+  QE_CUDA(cudaGraphGetNodes(graph, nullptr, &n));
+  if (n != ls.size()) {
+    cudaGraphDestroy(graph);
+    return fail(QE_ERR_CUDA, "captured %zu nodes for %zu launches", n, ls.size());
+  }
+  std::vector<cudaGraphNode_t> chain;
+  size_t nroot = 1;
+  cudaGraphNode_t cur = nullptr;
+  QE_CUDA(cudaGraphGetRootNodes(graph, &cur, &nroot));
+  if (nroot != 1) return fail(QE_ERR_CUDA, "captured graph has %zu roots", nroot);
+  while (cur) {
+    chain.push_back(cur);
+    size_t nd = 0;
+    QE_CUDA(cudaGraphNodeGetDependentNodes(cur, nullptr, &nd));
+    if (nd == 0) break;
+    if (nd != 1) return fail(QE_ERR_CUDA, "captured graph is not a chain");
+    cudaGraphNode_t next = nullptr;
+    QE_CUDA(cudaGraphNodeGetDependentNodes(cur, &next, &nd));
+    cur = next;
+  }
+  if (chain.size() != ls.size()) return fail(QE_ERR_CUDA, "chain of %zu nodes for %zu launches", chain.size(), ls.size());
+  cudaGraphExec_t exec = nullptr;
+  QE_CUDA(cudaGraphInstantiate(&exec, graph, 0));
+  g->graph = graph;
+  g->exec = exec;
+  g->nodes = chain;
+  g->launches = ls;
+  g->built = true;
+  ctx->stats.graphs_built += 1;
+  ctx->stats.capture_host_ms += std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
+  return QE_OK;
+}
+
+int32_t replay_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls) {
+  if (ls.size() != g->launches.size()) return fail(QE_ERR_CUDA, "graph shape changed");
+  for (size_t i = 0; i < ls.size(); ++i) {
+    const qe::Launch& now = ls[i];
+    qe::Launch& was = g->launches[i];
+    const bool same = now.func == was.func && now.nbytes == was.nbytes && now.smem == was.smem &&
+                      now.grid.x == was.grid.x && now.grid.y == was.grid.y && now.block.x == was.block.x &&
+                      std::memcmp(now.params, was.params, now.nbytes) == 0;
+    if (same) continue;
+    // caller-visible pointers (x, y, gradient destination) or the accumulate flag changed: patch the node in place
+    cudaKernelNodeParams np{};
+    void* args[1] = {const_cast<unsigned char*>(now.params)};
+    np.func = const_cast<void*>(now.func);
+    np.gridDim = now.grid;
+    np.blockDim = now.block;
+    np.sharedMemBytes = now.smem;
+    np.kernelParams = args;
+    np.extra = nullptr;
+    QE_CUDA(cudaGraphExecKernelNodeSetParams(g->exec, g->nodes[i], &np));
+    was = now;
+    ctx->stats.node_param_updates += 1;
+  }
+  QE_CUDA(cudaGraphLaunch(g->exec, ctx->exec_stream));
+  ctx->stats.graph_replays += 1;
+  ctx->stats.kernels_launched += ls.size();
+  return QE_OK;
+}
+
+// Sec. 4.4: the execution stream waits on the caller's stream before the action...
+int32_t handoff_in(qe_ctx* ctx, cudaStream_t caller) {
+  if (caller == ctx->exec_stream) return QE_OK;
+  QE_CUDA(cudaEventRecord(ctx->ev_in, caller));
+  QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_in, 0));
+  ctx->stats.handoffs += 1;
+  return QE_OK;
+}
+// ...and the caller's stream waits on the action's tail before it may consume anything.
+int32_t handoff_out(qe_ctx* ctx, cudaStream_t caller) {
+  if (caller == ctx->exec_stream) return QE_OK;
+  QE_CUDA(cudaEventRecord(ctx->ev_out, ctx->exec_stream));
+  QE_CUDA(cudaStreamWaitEvent(caller, ctx->ev_out, 0));
+  ctx->stats.handoffs += 1;
+  return QE_OK;
+}
+
+int32_t run_action(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls) {
+  if (ctx->exec_mode == QE_EXEC_GRAPH) {
+    if (!g->built) {
+      int32_t st = build_graph(ctx, g, ls);
+      if (st != QE_OK) return st;
+    }
+    return replay_graph(ctx, g, ls);
+  }
+  for (const qe::Launch& l : ls) {
+    int32_t st = launch_eager(ctx, l);
+    if (st != QE_OK) return st;
+  }
+  return QE_OK;
+}
+
+void destroy_graph(ActionGraph* g) {
+  if (g->exec) cudaGraphExecDestroy(g->exec);
+  if (g->graph) cudaGraphDestroy(g->graph);
+  g->exec = nullptr;
+  g->graph = nullptr;
+  g->built = false;
+}
+
+struct Carve {
+  uint64_t hist, Wq, WqT, slot0, per_slot, xq, xqT, gq, gqT, total;
+};
+Carve carve(const qe_layer_config& c) {
+  Carve k{};
+  uint64_t o = sizeof(qe::DevState);
+  k.hist = o;
+  o = align_up(o + 4ull * c.history_len * sizeof(float), 1024);
+  const uint64_t nk = (uint64_t)c.N * c.K, tk = (uint64_t)c.T * c.K, tn = (uint64_t)c.T * c.N;
+  k.Wq = o;
+  o += align_up(nk, 1024);
+  k.WqT = o;
+  o += align_up(nk, 1024);
+  k.slot0 = o;
+  k.xq = 0;
+  k.xqT = align_up(tk, 1024);
+  k.gq = k.xqT + align_up(tk, 1024);
+  k.gqT = k.gq + align_up(tn, 1024);
+  k.per_slot = k.gqT + align_up(tn, 1024);
+  k.total = o + k.per_slot * c.slots;
+  return k;
+}
+
+int32_t check_config(const qe_layer_config* c) {
+  if (!c) return fail(QE_ERR_BAD_ARG, "config is null");
+  if (!shape_ok(c->T) || !shape_ok(c->K) || !shape_ok(c->N))
+    return fail(QE_ERR_SHAPE, "T=%u K=%u N=%u: each must be a multiple of 128 in [256, 2^20]", c->T, c->K, c->N);
+  if (c->history_len < 1 || c->history_len > QE_MAX_HISTORY) return fail(QE_ERR_BAD_ARG, "history_len %u", c->history_len);
+  if (c->margin < -32 || c->margin > 32) return fail(QE_ERR_BAD_ARG, "margin %d", c->margin);
+  if (c->slots < 1 || c->slots > QE_MAX_SLOTS) return fail(QE_ERR_BAD_ARG, "slots %u", c->slots);
+  return QE_OK;
+}
+
+qe::Launch commit_launch(qe_layer* L, uint32_t mask, uint32_t bump, const float* override_amax) {
+  qe::CommitParams cp{};
+  cp.st = L->st;
+  cp.hist = L->hist;
+  cp.H = L->cfg.history_len;
+  cp.class_mask = mask;
+  cp.pow2_neg_margin = std::ldexp(1.0f, -L->cfg.margin);
+  cp.amax_override = override_amax;
+  cp.bump_token = bump;
+  return qe::make_commit(cp);
+}
+
+qe::Launch quant_launch(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uint32_t rows, uint32_t cols, int cls,
+                        float* sinv_dst, int fmt) {
+  qe::QuantParams qp{};
+  qp.x = (const uint16_t*)x;
+  qp.q = q;
+  qp.qT = qT;
+  qp.rows = rows;
+  qp.cols = cols;
+  qp.scale = &L->st->scale[cls];
+  qp.sinv_src = &L->st->scale_inv[cls];
+  qp.sinv_dst = sinv_dst;
+  qp.amax_bits = &L->st->pending_amax[cls];
+  qp.fmt = fmt;
+  return qe::make_quantize(qp);
+}
+
+}  // namespace
+
+// ================================================================================================ C ABI
+extern "C" {
+
+int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
+  if (!cfg || !out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (cfg->exec_mode > QE_EXEC_GRAPH) return fail(QE_ERR_BAD_ARG, "exec_mode %u", cfg->exec_mode);
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess || ndev == 0) return fail(QE_ERR_UNSUPPORTED, "no CUDA device: %s", cudaGetErrorString(e));
+  QE_CUDA(cudaSetDevice(cfg->device));
+  DeviceInfo* d = nullptr;
+  int32_t st = device_info(cfg->device, &d);
+  if (st != QE_OK) return st;
+  qe_ctx* c = new (std::nothrow) qe_ctx();
+  if (!c) return fail(QE_ERR_BAD_ARG, "out of host memory");
+  c->dev = d;
+  c->exec_mode = cfg->exec_mode;
+  QE_CUDA(cudaStreamCreateWithFlags(&c->exec_stream, cudaStreamNonBlocking));
+  QE_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
+  QE_CUDA(cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming));
+  st = qe_registry_create(&c->registry);
+  if (st != QE_OK) return st;
+  *out = c;
+  return QE_OK;
+}
+
+int32_t qe_ctx_destroy(qe_ctx* c) {
+  if (!c) return QE_OK;
+  cudaStreamSynchronize(c->exec_stream);
+  cudaEventDestroy(c->ev_in);
+  cudaEventDestroy(c->ev_out);
+  cudaStreamDestroy(c->exec_stream);
+  qe_registry_destroy(c->registry);
+  delete c;
+  return QE_OK;
+}
+
+int32_t qe_layer_workspace_bytes(const qe_layer_config* cfg, uint64_t* bytes_out) {
+  int32_t st = check_config(cfg);
+  if (st != QE_OK) return st;
+  if (!bytes_out) return fail(QE_ERR_BAD_ARG, "bytes_out is null");
+  *bytes_out = carve(*cfg).total;
+  return QE_OK;
+}
+
+int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint64_t ws_bytes, qe_layer** out) {
+  if (!ctx || !out) return fail(QE_ERR_BAD_ARG, "null argument");
+  int32_t st = check_config(cfg);
+  if (st != QE_OK) return st;
+  if (!cfg->weight_dev) return fail(QE_ERR_BAD_ARG, "weight_dev is null");
+  const Carve k = carve(*cfg);
+  if (!ws || ((uintptr_t)ws & 255u) || ws_bytes < k.total)
+    return fail(QE_ERR_WORKSPACE, "workspace %p of %llu bytes; need %llu bytes, 256-byte aligned", ws,
+                (unsigned long long)ws_bytes, (unsigned long long)k.total);
+  qe_layer* L = new (std::nothrow) qe_layer();
+  if (!L) return fail(QE_ERR_BAD_ARG, "out of host memory");
+  L->ctx = ctx;
+  L->cfg = *cfg;
+  L->ws_bytes = k.total;
+  st = qe_contract_create(cfg->slots, cfg->stage, cfg->unit, cfg->inv, ctx->registry, &L->contract);
+  if (st != QE_OK) { delete L; return st; }
+  uint8_t* base = (uint8_t*)ws;
+  L->st = (qe::DevState*)base;
+  L->hist = (float*)(base + k.hist);
+  L->Wq = base + k.Wq;
+  L->WqT = base + k.WqT;
+  const DeviceInfo* d = ctx->dev;
+  const uint32_t T = cfg->T, K = cfg->K, N = cfg->N;
+  for (uint32_t p = 0; p < cfg->slots; ++p) {
+    uint8_t* s = base + k.slot0 + k.per_slot * p;
+    L->Xq[p] = s + k.xq;
+    L->XqT[p] = s + k.xqT;
+    L->Gq[p] = s + k.gq;
+    L->GqT[p] = s + k.gqT;
+    if ((st = make_map(d, &L->tmXq_A[p], L->Xq[p], T, K, 128)) != QE_OK) break;   // F:  A = Xq  [T,K]
+    if ((st = make_map(d, &L->tmGq_A[p], L->Gq[p], T, N, 128)) != QE_OK) break;   // dI: A = Gq  [T,N]
+    if ((st = make_map(d, &L->tmGqT_A[p], L->GqT[p], N, T, 128)) != QE_OK) break; // dW: A = Gq^T [N,T]
+    if ((st = make_map(d, &L->tmXqT_B[p], L->XqT[p], K, T, 256)) != QE_OK) break; // dW: B = Xq^T [K,T]
+  }
+  if (st == QE_OK) st = make_map(d, &L->tmWq_B, L->Wq, N, K, 256);    // F:  B = Wq   [N,K]
+  if (st == QE_OK) st = make_map(d, &L->tmWqT_B, L->WqT, K, N, 256);  // dI: B = Wq^T [K,N]
+  if (st != QE_OK) { qe_contract_destroy(L->contract); delete L; return st; }
+  // state: histories 0, scales 1, everything else 0
+  qe::DevState init{};
+  for (int c = 0; c < 4; ++c) init.scale[c] = init.scale_inv[c] = 1.0f;
+  cudaError_t e = cudaMemsetAsync(base, 0, k.Wq, ctx->exec_stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(base, &init, sizeof(init), cudaMemcpyHostToDevice, ctx->exec_stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->exec_stream);
+  if (e != cudaSuccess) {
+    qe_contract_destroy(L->contract);
+    delete L;
+    return fail(QE_ERR_CUDA, "state initialisation: %s", cudaGetErrorString(e));
+  }
+  ctx->stats.workspace_bytes += k.total;
+  *out = L;
+  return QE_OK;
+}
+
+int32_t qe_layer_destroy(qe_layer* L) {
+  if (!L) return QE_OK;
+  cudaStreamSynchronize(L->ctx->exec_stream);
+  for (uint32_t p = 0; p < L->cfg.slots; ++p) {
+    destroy_graph(&L->gF[p]);
+    destroy_graph(&L->gDI[p]);
+    destroy_graph(&L->gDW[p]);
+    destroy_graph(&L->gDWs[p]);
+  }
+  destroy_graph(&L->gRefresh);
+  destroy_graph(&L->gCommit);
+  L->ctx->stats.workspace_bytes -= L->ws_bytes;
+  qe_contract_destroy(L->contract);
+  delete L;
+  return QE_OK;
+}
+
+int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* y, void* caller_stream,
+                   qe_tape* tape_out) {
+  if (!L || !x || !y || !tape_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (((uintptr_t)x | (uintptr_t)y) & 15u) return fail(QE_ERR_BAD_ARG, "x and y must be 16-byte aligned");
+  int32_t refresh = 0;
+  uint32_t p = 0;
+  int32_t st = qe_contract_forward_check(L->contract, mb, gen, &refresh, &p);  // check ...
+  if (st != QE_OK) return st;
+  qe_ctx* ctx = L->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (refresh) {  // Invariant 3: first forward of the epoch re-quantises the weight and commits its amax
+    std::vector<qe::Launch> ls;
+    ls.push_back(quant_launch(L, L->cfg.weight_dev, L->Wq, L->WqT, N, K, QE_CLASS_W, &L->st->cache_sinv_W, QE_E4M3));
+    ls.push_back(commit_launch(L, 1u << QE_CLASS_W, 0, nullptr));
+    if ((st = run_action(ctx, &L->gRefresh, ls)) != QE_OK) return st;
+  }
+  std::vector<qe::Launch> ls;
+  ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
+  qe::GemmParams gp{};
+  gp.tmA = L->tmXq_A[p];
+  gp.tmB = L->tmWq_B;
+  gp.M = T;
+  gp.N = N;
+  gp.Kc = K;
+  gp.idesc = qe::gemm_idesc(QE_E4M3, QE_E4M3);
+  gp.alpha_a = &L->st->slot_sinv_X[p];
+  gp.alpha_b = &L->st->cache_sinv_W;
+  gp.out = y;
+  gp.ldo = N;
+  gp.epi = 0;
+  gp.amax_bits = &L->st->pending_amax[QE_CLASS_Y];
+  gp.status = &L->st->status;
+  ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
+  ls.push_back(commit_launch(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr));
+  if ((st = run_action(ctx, &L->gF[p], ls)) != QE_OK) return st;  // ... run ...
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  return qe_contract_forward_commit(L->contract, mb, tape_out);  // ... commit
+}
+
+int32_t qe_backward_dI(qe_layer* L, const qe_tape* tape, const void* dy, void* dx, void* caller_stream) {
+  if (!L || !tape || !dy || !dx) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (((uintptr_t)dy | (uintptr_t)dx) & 15u) return fail(QE_ERR_BAD_ARG, "dy and dx must be 16-byte aligned");
+  int32_t st = qe_contract_dI_check(L->contract, tape);
+  if (st != QE_OK) return st;
+  qe_ctx* ctx = L->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  const uint32_t p = tape->ref.slot, T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  std::vector<qe::Launch> ls;
+  ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
+  qe::GemmParams gp{};
+  gp.tmA = L->tmGq_A[p];
+  gp.tmB = L->tmWqT_B;
+  gp.M = T;
+  gp.N = K;
+  gp.Kc = N;
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3);
+  gp.alpha_a = &L->st->slot_sinv_G[p];
+  gp.alpha_b = &L->st->cache_sinv_W;
+  gp.out = dx;
+  gp.ldo = K;
+  gp.epi = 0;
+  gp.amax_bits = nullptr;
+  gp.status = &L->st->status;
+  ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
+  ls.push_back(commit_launch(L, 1u << QE_CLASS_G, 1, nullptr));  // backward amax/scale updated exactly once, here
+  if ((st = run_action(ctx, &L->gDI[p], ls)) != QE_OK) return st;
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  return qe_contract_dI_commit(L->contract, tape);
+}
+
+static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, uint64_t elems, uint64_t off,
+                                float* temp, void* caller_stream) {
+  if (!L || !tape) return fail(QE_ERR_BAD_ARG, "null argument");
+  const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
+  const uint64_t slice = (uint64_t)N * K;
+  int32_t acc = 0;
+  int32_t st = qe_contract_dW_check(L->contract, tape, (uint64_t)(uintptr_t)grad, elems, off, slice, &acc);
+  if (st != QE_OK) return st;
+  qe_ctx* ctx = L->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  const uint32_t p = tape->ref.slot;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  qe::GemmParams gp{};
+  gp.tmA = L->tmGqT_A[p];
+  gp.tmB = L->tmXqT_B[p];
+  gp.M = N;
+  gp.N = K;
+  gp.Kc = T;
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3);
+  gp.alpha_a = &L->st->slot_sinv_G[p];  // snapshots taken when dY_m and X_m were quantised, never the current state
+  gp.alpha_b = &L->st->slot_sinv_X[p];
+  gp.ldo = K;
+  gp.amax_bits = nullptr;
+  gp.status = &L->st->status;
+  std::vector<qe::Launch> ls;
+  if (!temp) {
+    gp.out = grad + off;  // direct placement: the epilogue reads, adds and writes the destination itself
+    gp.epi = acc ? 2 : 1;
+    ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
+    st = run_action(ctx, &L->gDW[p], ls);
+  } else {
+    gp.out = temp;
+    gp.epi = 1;
+    ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
+    qe::AccumParams ap{};
+    ap.dst = (float4*)(grad + off);
+    ap.src = (const float4*)temp;
+    ap.nvec = slice / 4;
+    ap.accumulate = acc;
+    ls.push_back(qe::make_accumulate(ap));
+    st = run_action(ctx, &L->gDWs[p], ls);
+  }
+  if (st != QE_OK) return st;
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  return qe_contract_dW_commit(L->contract, tape, (uint64_t)(uintptr_t)grad, off, slice);
+}
+
+int32_t qe_backward_dW(qe_layer* L, const qe_tape* tape, float* grad, uint64_t elems, uint64_t off, void* stream) {
+  return backward_dW_impl(L, tape, grad, elems, off, nullptr, stream);
+}
+
+int32_t qe_backward_dW_staged(qe_layer* L, const qe_tape* tape, float* grad, uint64_t elems, uint64_t off,
+                              float* temp, void* stream) {
+  if (!temp || ((uintptr_t)temp & 15u)) return fail(QE_ERR_BAD_ARG, "temp_dev must be non-null and 16-byte aligned");
+  return backward_dW_impl(L, tape, grad, elems, off, temp, stream);
+}
+
+static int32_t read_status(qe_layer* L, uint32_t* status) {
+  QE_CUDA(cudaStreamSynchronize(L->ctx->exec_stream));
+  QE_CUDA(cudaMemcpy(status, &L->st->status, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+  return QE_OK;
+}
+
+int32_t qe_optimizer_boundary(qe_layer* L, uint32_t expected) {
+  if (!L) return fail(QE_ERR_BAD_ARG, "layer is null");
+  uint32_t status = 0;
+  int32_t st = read_status(L, &status);
+  if (st != QE_OK) return st;
+  if (status) return fail(QE_ERR_TIMEOUT, "device status word %#x: a bounded wait expired in a GEMM", status);
+  return qe_contract_boundary(L->contract, expected);
+}
+
+int32_t qe_scale_commit(qe_layer* L, uint32_t cls, const float* amax_dev, void* caller_stream) {
+  if (!L) return fail(QE_ERR_BAD_ARG, "layer is null");
+  if (cls > QE_CLASS_Y) return fail(QE_ERR_BAD_ARG, "tensor_class %u", cls);
+  qe_ctx* ctx = L->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  int32_t st;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  std::vector<qe::Launch> ls;
+  ls.push_back(commit_launch(L, 1u << cls, 0, amax_dev));
+  if ((st = run_action(ctx, &L->gCommit, ls)) != QE_OK) return st;
+  return handoff_out(ctx, caller);
+}
+
+int32_t qe_abort_step(qe_layer* L) {
+  if (!L) return fail(QE_ERR_BAD_ARG, "layer is null");
+  return qe_contract_abort(L->contract);
+}
+int32_t qe_arena_rebuild(qe_layer* L) {
+  if (!L) return fail(QE_ERR_BAD_ARG, "layer is null");
+  return qe_contract_rebuild(L->contract);
+}
+int32_t qe_invalidate_cache(qe_layer* L) {
+  if (!L) return fail(QE_ERR_BAD_ARG, "layer is null");
+  return qe_contract_invalidate_cache(L->contract);
+}
+int32_t qe_next_slot(const qe_layer* L, uint32_t* slot_out) {
+  if (!L || !slot_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  const int p = L->contract->lowest_free();
+  if (p < 0) return fail(QE_ERR_POOL_FULL, "all slots occupied");
+  *slot_out = (uint32_t)p;
+  return QE_OK;
+}
+
+int32_t qe_get_state(qe_layer* L, qe_state_view* out, float* window_out, float* slot_sinv_out) {
+  if (!L || !out) return fail(QE_ERR_BAD_ARG, "null argument");
+  QE_CUDA(cudaStreamSynchronize(L->ctx->exec_stream));
+  qe::DevState h;
+  QE_CUDA(cudaMemcpy(&h, L->st, sizeof(h), cudaMemcpyDeviceToHost));
+  std::memset(out, 0, sizeof(*out));
+  for (int c = 0; c < 4; ++c) {
+    out->cls[c].scale = h.scale[c];
+    out->cls[c].scale_inv = h.scale_inv[c];
+    out->cls[c].count = h.count[c];
+  }
+  out->cache_sinv_W = h.cache_sinv_W;
+  out->device_status = h.status;
+  out->device_token = h.token;
+  int32_t st = qe_contract_get(L->contract, &out->contract);
+  if (st != QE_OK) return st;
+  const uint32_t H = L->cfg.history_len, P = L->cfg.slots;
+  if (window_out) {
+    std::vector<float> ring(4ull * H);
+    QE_CUDA(cudaMemcpy(ring.data(), L->hist, ring.size() * sizeof(float), cudaMemcpyDeviceToHost));
+    for (int c = 0; c < 4; ++c)
+      for (uint32_t j = 0; j < H; ++j) {
+        const uint64_t idx = ((uint64_t)h.count[c] + (uint64_t)H * 2 - 1 - j) % H;  // newest first
+        window_out[(size_t)c * H + j] = ring[(size_t)c * H + idx];
+      }
+  }
+  if (slot_sinv_out)
+    for (uint32_t p = 0; p < P; ++p) {
+      slot_sinv_out[p] = h.slot_sinv_X[p];
+      slot_sinv_out[P + p] = h.slot_sinv_G[p];
+    }
+  return QE_OK;
+}
+
+int32_t qe_read_fp8(qe_layer* L, uint32_t which, uint32_t slot, void* host_out, uint64_t bytes) {
+  if (!L || !host_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  const uint64_t tk = (uint64_t)L->cfg.T * L->cfg.K, tn = (uint64_t)L->cfg.T * L->cfg.N, nk = (uint64_t)L->cfg.N * L->cfg.K;
+  if (which > 5 || (which < 4 && slot >= L->cfg.slots)) return fail(QE_ERR_BAD_ARG, "which %u slot %u", which, slot);
+  const uint8_t* src = which == 0 ? L->Xq[slot] : which == 1 ? L->XqT[slot] : which == 2 ? L->Gq[slot]
+                     : which == 3 ? L->GqT[slot] : which == 4 ? L->Wq : L->WqT;
+  const uint64_t need = which < 2 ? tk : which < 4 ? tn : nk;
+  if (bytes != need) return fail(QE_ERR_BAD_ARG, "bytes %llu, tensor has %llu", (unsigned long long)bytes, (unsigned long long)need);
+  QE_CUDA(cudaStreamSynchronize(L->ctx->exec_stream));
+  QE_CUDA(cudaMemcpy(host_out, src, need, cudaMemcpyDeviceToHost));
+  return QE_OK;
+}
+
+int32_t qe_get_stats(const qe_ctx* ctx, qe_stats* out) {
+  if (!ctx || !out) return fail(QE_ERR_BAD_ARG, "null argument");
+  *out = ctx->stats;
+  return QE_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ standalone kernels
+static int32_t current_device_info(DeviceInfo** d) {
+  int dev = 0;
+  QE_CUDA(cudaGetDevice(&dev));
+  return device_info(dev, d);
+}
+
+static int32_t launch_on(const qe::Launch& l, cudaStream_t s) {
+  void* args[1] = {const_cast<unsigned char*>(l.params)};
+  QE_CUDA(cudaLaunchKernel(l.func, l.grid, l.block, args, l.smem, s));
+  return QE_OK;
+}
+
+int32_t qe_quantize(const void* x, uint32_t rows, uint32_t cols, const float* scale_dev, uint32_t fmt, void* q,
+                    void* qT, float* amax_dev, void* stream) {
+  if (!x || !scale_dev || !q) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (fmt > QE_E5M2) return fail(QE_ERR_BAD_ARG, "fp8_format %u", fmt);
+  if (rows == 0 || cols == 0 || rows % 64 || cols % 64) return fail(QE_ERR_SHAPE, "rows %u cols %u must be multiples of 64", rows, cols);
+  if (((uintptr_t)x & 15u) || ((uintptr_t)q & 7u) || ((uintptr_t)qT & 7u)) return fail(QE_ERR_BAD_ARG, "misaligned pointer");
+  qe::QuantParams qp{};
+  qp.x = (const uint16_t*)x;
+  qp.q = (uint8_t*)q;
+  qp.qT = (uint8_t*)qT;
+  qp.rows = rows;
+  qp.cols = cols;
+  qp.scale = scale_dev;
+  qp.amax_bits = (uint32_t*)amax_dev;
+  qp.fmt = (int32_t)fmt;
+  return launch_on(qe::make_quantize(qp), (cudaStream_t)stream);
+}
+
+uint32_t qe_amax_partials(void) { return qe::kAmaxPartials; }
+
+int32_t qe_amax(const void* x, uint64_t n, float* partials, float* amax_dev, void* stream) {
+  if (!x || !partials || !amax_dev) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (n % 8 || ((uintptr_t)x & 15u)) return fail(QE_ERR_SHAPE, "n must be a multiple of 8 and x 16-byte aligned");
+  qe::AmaxParams ap{};
+  ap.x = (const uint4*)x;
+  ap.nvec = n / 8;
+  ap.partials = partials;
+  ap.out = amax_dev;
+  const uint64_t blocks = (ap.nvec + 1023) / 1024;  // 4 vectors per thread per trip
+  ap.nparts = (uint32_t)(blocks < 1 ? 1 : blocks > qe::kAmaxPartials ? qe::kAmaxPartials : blocks);
+  int32_t st = launch_on(qe::make_amax_pass1(ap), (cudaStream_t)stream);
+  if (st != QE_OK) return st;
+  return launch_on(qe::make_amax_pass2(ap), (cudaStream_t)stream);
+}
+
+int32_t qe_accumulate(float* dst, const float* src, uint64_t n, int32_t accumulate, void* stream) {
+  if (!dst || !src) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (n % 4 || (((uintptr_t)dst | (uintptr_t)src) & 15u)) return fail(QE_ERR_SHAPE, "n must be a multiple of 4, pointers 16-byte aligned");
+  qe::AccumParams ap{};
+  ap.dst = (float4*)dst;
+  ap.src = (const float4*)src;
+  ap.nvec = n / 4;
+  ap.accumulate = accumulate;
+  return launch_on(qe::make_accumulate(ap), (cudaStream_t)stream);
+}
+
+int32_t qe_gemm_fp8(const void* a, uint32_t a_fmt, const void* b, uint32_t b_fmt, uint32_t M, uint32_t Nn, uint32_t Kc,
+                    const float* alpha_a, const float* alpha_b, void* d, uint32_t out_kind, float* amax_dev,
+                    uint32_t* status_dev, void* stream) {
+  if (!a || !b || !alpha_a || !alpha_b || !d || !status_dev) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (a_fmt > QE_E5M2 || b_fmt > QE_E5M2 || out_kind > 2) return fail(QE_ERR_BAD_ARG, "bad enum");
+  if (!shape_ok(M) && M != 128) return fail(QE_ERR_SHAPE, "M=%u", M);
+  if (!shape_ok(Nn) || !shape_ok(Kc) && Kc != 128) return fail(QE_ERR_SHAPE, "N=%u Kc=%u", Nn, Kc);
+  if ((((uintptr_t)a | (uintptr_t)b | (uintptr_t)d) & 15u)) return fail(QE_ERR_BAD_ARG, "misaligned pointer");
+  DeviceInfo* dev = nullptr;
+  int32_t st = current_device_info(&dev);
+  if (st != QE_OK) return st;
+  qe::GemmParams gp{};
+  if ((st = make_map(dev, &gp.tmA, a, M, Kc, 128)) != QE_OK) return st;
+  if ((st = make_map(dev, &gp.tmB, b, Nn, Kc, 256)) != QE_OK) return st;
+  gp.M = M;
+  gp.N = Nn;
+  gp.Kc = Kc;
+  gp.idesc = qe::gemm_idesc((int)a_fmt, (int)b_fmt);
+  gp.alpha_a = alpha_a;
+  gp.alpha_b = alpha_b;
+  gp.out = d;
+  gp.ldo = Nn;
+  gp.epi = (int32_t)out_kind;
+  gp.amax_bits = (uint32_t*)amax_dev;
+  gp.status = status_dev;
+  return launch_on(qe::make_gemm(gp, dev->num_sms), (cudaStream_t)stream);
+}
+
+}  // extern "C"
