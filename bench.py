@@ -1,0 +1,432 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 delayed-scaling linear-layer hot path (F + dI + dW, split-backward schedule).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--mode graph|eager] [--impl ours|reference]
+
+One "step" is one optimizer step of the configuration: every microbatch's F, dI and dW for every linear
+of the block in zero-bubble order (dW deferred), all weight gradients accumulated in place in one flat
+FP32 buffer, then the optimizer boundary of every layer (which makes the next step re-quantise the
+weights).  Prints ONE JSON line.  N > 1 runs N independent replicas (the path does not shard).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_23536_b200 import inputs  # noqa: E402
+from paper_2609_23536_b200.schedules import peak_live, sched  # noqa: E402
+
+METRIC = "fp8_linear_layer_F_dI_dW_tflops"
+UNIT = "TFLOP/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+def step_flops(cfg) -> float:
+    per_mb = 6.0 * cfg["T"] * sum(K * N for _, K, N in cfg["linears"])
+    return per_mb * cfg["M"] * cfg["layers"]
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+class Stage:
+    """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
+
+    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False):
+        import torch
+
+        self.qe, self.cfg, self.dev = qe, cfg, device
+        self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0)
+        self.schedule = sched(cfg["M"], *cfg["sched"])
+        P = peak_live(self.schedule)
+        T, M = cfg["T"], cfg["M"]
+        self.layers, self.offsets = [], []
+        lin = cfg["linears"]
+        offs, per_layer = inputs.grad_offsets(lin)
+        self.grad = torch.zeros(per_layer * cfg["layers"], dtype=torch.float32, device=device)
+        for l in range(cfg["layers"]):
+            for j, (_, K, N) in enumerate(lin):
+                w = inputs.weights(cfg_name, l, j, N, K).to(device)
+                self.layers.append(qe.Layer(self.ctx, T, K, N, cfg["H"], cfg["margin"], P, w, stage=0, unit=l * len(lin) + j))
+                self.offsets.append(l * per_layer + offs[j])
+        # distinct synthetic tensors per (microbatch, linear); drawn on the host once, outside any timed region
+        g = torch.Generator(device="cpu")
+        g.manual_seed(inputs.seed_for(cfg_name, "bench"))
+        self.X, self.dY, self.Y, self.dX, self.Xh, self.dYh = [], [], [], [], [], []
+        for m in range(M):
+            xs, gs, ys, dxs, xh, gh = [], [], [], [], [], []
+            for L in self.layers:
+                x = torch.randn((T, L.K), generator=g, dtype=torch.float32).to(torch.bfloat16)
+                dy = (torch.randn((T, L.N), generator=g, dtype=torch.float32) * 1e-3).to(torch.bfloat16)
+                if host_io:
+                    xh.append(x.pin_memory())
+                    gh.append(dy.pin_memory())
+                xs.append(x.to(device))
+                gs.append(dy.to(device))
+                ys.append(torch.empty((T, L.N), dtype=torch.bfloat16, device=device))
+                dxs.append(torch.empty((T, L.K), dtype=torch.bfloat16, device=device))
+            self.X.append(xs); self.dY.append(gs); self.Y.append(ys); self.dX.append(dxs)
+            self.Xh.append(xh); self.dYh.append(gh)
+        self.grad_host = torch.empty(self.grad.shape, dtype=torch.float32).pin_memory() if host_io else None
+        self.epoch = 0
+        self.h2d = self.d2h = 0
+
+    def step(self, host_io=False):
+        tapes = {}
+        n = len(self.layers)
+        for a, m in self.schedule:
+            order = range(n) if a == "F" else range(n - 1, -1, -1)
+            for i in order:
+                L = self.layers[i]
+                if a == "F":
+                    if host_io:
+                        self.X[m][i].copy_(self.Xh[m][i], non_blocking=True)
+                        self.h2d += self.Xh[m][i].numel() * 2
+                    tapes[(m, i)] = L.forward(m, self.epoch, self.X[m][i], self.Y[m][i])
+                elif a == "dI":
+                    if host_io:
+                        self.dY[m][i].copy_(self.dYh[m][i], non_blocking=True)
+                        self.h2d += self.dYh[m][i].numel() * 2
+                    L.backward_dI(tapes[(m, i)], self.dY[m][i], self.dX[m][i])
+                else:
+                    L.backward_dW(tapes[(m, i)], self.grad, self.offsets[i])
+        if host_io:
+            self.grad_host.copy_(self.grad, non_blocking=True)
+            self.d2h += self.grad.numel() * 4
+        for L in self.layers:
+            L.optimizer_boundary(self.cfg["M"])
+        self.epoch += 1
+
+
+def time_steps(stage, steps, warmup, host_io, dist):
+    import torch
+
+    for _ in range(warmup):
+        stage.step(host_io)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    stage.h2d = stage.d2h = 0
+    k0 = stage.ctx.stats()["kernels_launched"]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        stage.step(host_io)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    return ms, stage.ctx.stats()["kernels_launched"] - k0
+
+
+def gemm_roofline(qe, cfg, peaks, device):
+    """Times the dominant kernel (the tcgen05 FP8 GEMM) alone, live: every GEMM shape of one microbatch, launched
+    back to back through the C-ABI on the current stream over rotating operand sets larger than L2, CUDA events
+    around the loop.  achieved = algorithmic flops / average launch duration."""
+    import torch
+
+    T = cfg["T"]
+    shapes = []
+    for _, K, N in cfg["linears"]:
+        shapes += [("F", T, N, K, 0, 0, 0), ("dI", T, K, N, 1, 0, 0), ("dW", N, K, T, 1, 0, 2)]
+    one = torch.ones(1, dtype=torch.float32, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    tot_flops = tot_ms = 0.0
+    per = {}
+    for name, M_, N_, Kc, af, bf, kind in shapes:
+        nset = max(2, int(160e6 // (M_ * Kc + N_ * Kc + M_ * N_ * (2 if kind == 0 else 8))) + 1)
+        nset = min(nset, 24)
+        A = [torch.randint(0, 120, (M_, Kc), dtype=torch.uint8, device=device) for _ in range(nset)]
+        B = [torch.randint(0, 120, (N_, Kc), dtype=torch.uint8, device=device) for _ in range(nset)]
+        D = [torch.zeros((M_, N_), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=device) for _ in range(nset)]
+        reps = 3 * nset
+        for i in range(nset):
+            qe.qe_gemm_fp8(A[i], af, B[i], bf, one, one, D[i], kind, None, status)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for r in range(reps):
+            i = r % nset
+            qe.qe_gemm_fp8(A[i], af, B[i], bf, one, one, D[i], kind, None, status)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        fl = 2.0 * M_ * N_ * Kc
+        tot_flops += fl
+        tot_ms += ms
+        per.setdefault(name, [0.0, 0.0])
+        per[name][0] += fl
+        per[name][1] += ms
+        del A, B, D
+    assert status.item() == 0
+    achieved = tot_flops / (tot_ms * 1e-3) / 1e12
+    peak = 2.0 * peaks["bf16_burst"]  # FP8 dense = 2 x the bf16 peak (nominal ratio), kernels timed alone -> burst figure
+    return {
+        "bound": "tensor", "kernel": "gemm_fp8_kernel", "achieved": round(achieved, 1), "peak": round(peak, 1),
+        "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": None, "peak_source": peaks["source"] + " bf16 burst x2",
+        "frac_of_nominal_4500": round(achieved / 4500.0, 4),
+        "per_action_tflops": {k: round(v[0] / (v[1] * 1e-3) / 1e12, 1) for k, v in per.items()},
+        "gemm_ms_per_microbatch": round(tot_ms, 4),
+    }
+
+
+def hbm_kernels(qe, cfg, peaks, device):
+    """Quantise(+transpose+amax) and standalone amax on tensors larger than L2: achieved algorithmic GB/s."""
+    import torch
+
+    rows, cols = 8192, 16384  # 268 MB bf16 in: larger than L2
+    x = (torch.randn((rows, cols), device=device) * 1.0).to(torch.bfloat16)
+    s = torch.ones(1, device=device)
+    q = torch.empty((rows, cols), dtype=torch.uint8, device=device)
+    qT = torch.empty((cols, rows), dtype=torch.uint8, device=device)
+    amax = torch.zeros(1, device=device)
+    part = torch.empty(qe.qe_amax_partials(), device=device)
+    out = {}
+
+    def timeit(fn, nbytes, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        gbs = nbytes / (e0.elapsed_time(e1) / reps * 1e-3) / 1e9
+        return {"GB/s": round(gbs, 1), "frac": round(gbs / peaks["hbm_gbs"], 4)}
+
+    n = rows * cols
+    out["quantize_transpose_amax_4B_per_elt"] = timeit(lambda: qe.qe_quantize(x, s, 0, q, qT, amax), 4 * n)
+    out["quantize_amax_3B_per_elt"] = timeit(lambda: qe.qe_quantize(x, s, 0, q, None, amax), 3 * n)
+    out["amax_2B_per_elt"] = timeit(lambda: qe.qe_amax(x, part, amax), 2 * n)
+    g = torch.zeros(n // 2, device=device)
+    t = torch.ones(n // 2, device=device)
+    out["accumulate_12B_per_elt"] = timeit(lambda: qe.qe_accumulate(g, t, True), 12 * (n // 2))
+    out["peak_GB/s"] = peaks["hbm_gbs"]
+    out["peak_source"] = peaks["source"]
+    return out
+
+
+# ------------------------------------------------------------------------------------------------ oracle legs
+def oracle_sample(cfg_name, cfg):
+    """One microbatch of every linear of the block (F + dI + dW) through the CPU oracle, as it stands."""
+    from oracle.layer import OracleLinear
+
+    T = cfg["T"]
+    t_total, flops = 0.0, 0.0
+    for j, (_, K, N) in enumerate(cfg["linears"]):
+        L = OracleLinear(T, K, N, cfg["H"], cfg["margin"], 1)
+        L.set_weight(inputs.bits(inputs.weights(cfg_name, 0, j, N, K)))
+        X = inputs.bits(inputs.activations(cfg_name, 0, 0, j, 0, T, K))
+        dY = inputs.bits(inputs.upstream_grads(cfg_name, 0, 0, j, 0, T, N))
+        buf = np.zeros(N * K, np.float32)
+        t0 = time.perf_counter()
+        tape, _ = L.forward(0, 0, X)
+        L.backward_dI(tape, dY)
+        L.backward_dW(tape, buf, 0)
+        t_total += time.perf_counter() - t0
+        flops += 6.0 * T * K * N
+    return t_total, flops
+
+
+def _threads():
+    try:
+        from threadpoolctl import threadpool_info
+
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def run_reference(args, cfg_name, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = "one microbatch of all %d linears of %s (F+dI+dW), 1/%d of a step" % (len(cfg["linears"]), cfg_name, cfg["M"] * cfg["layers"])
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(cfg_name, cfg)
+    t0 = time.perf_counter()
+    tot_s = tot_f = 0.0
+    for _ in range(args.steps):
+        s, f = oracle_sample(cfg_name, cfg)
+        tot_s += s
+        tot_f += f
+    val = tot_f / tot_s / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": tot_s / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg_name, "note": "CPU oracle on the host cores; each step is a bounded sample: " + sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": _threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "wall_s": time.perf_counter() - t0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="C2")
+    ap.add_argument("--mode", default="graph", choices=["graph", "eager"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the e2e, roofline, HBM-kernel and CPU-baseline legs")
+    args = ap.parse_args()
+    cfg_name, cfg = args.config, inputs.CONFIGS[args.config]
+    if args.impl == "reference":
+        return run_reference(args, cfg_name, cfg)
+
+    import torch
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle arm")
+    from paper_2609_23536_b200 import build
+
+    build.build()
+    from paper_2609_23536_b200 import binding as qe
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    device = torch.device("cuda", local)
+    peaks = _peaks()
+    args.warmup = max(args.warmup, 3)
+
+    stage = Stage(qe, cfg_name, cfg, args.mode, device)
+    with ClockSampler(local) as clk:
+        ms, launches = time_steps(stage, args.steps, args.warmup, False, dist)
+    clocks = clk.summary()
+    flops = step_flops(cfg) * args.steps * world
+    value = flops / (ms * 1e-3) / 1e12
+    stats = stage.ctx.stats()
+    status = max(L.state()["device_status"] for L in stage.layers[:1])
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp8_e4m3_e5m2_fp32acc", "data": "synthetic",
+        "config": {
+            "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
+            "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
+            "history_len": cfg["H"], "exec": args.mode, "parallelism": "replicas x%d (path does not shard)" % world,
+            "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
+                sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
+            "flop_per_step": step_flops(cfg),
+        },
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "frac_of_fp8_peak": {"of_measured_bf16_sustained_x2": round(value / world / (2 * peaks["bf16_sustained"]), 4),
+                             "of_nominal_4500": round(value / world / 4500.0, 4)},
+        "stats": {k: (round(v, 3) if isinstance(v, float) else v) for k, v in stats.items()},
+        "device_status": int(status),
+    }
+    del stage
+    torch.cuda.empty_cache()
+
+    if not args.no_extras:
+        stage = Stage(qe, cfg_name, cfg, args.mode, device, host_io=True)
+        ms2, _ = time_steps(stage, max(2, args.steps // 2), 3, True, dist)
+        n2 = max(2, args.steps // 2)
+        line["e2e"] = {"value": round(step_flops(cfg) * n2 * world / (ms2 * 1e-3) / 1e12, 2), "unit": UNIT,
+                       "h2d_bytes_per_step": stage.h2d // n2, "d2h_bytes_per_step": stage.d2h // n2,
+                       "ms_per_step": round(ms2 / n2, 3),
+                       "what": "X and dY of every microbatch copied from pinned host memory, gradient buffer read back, each step"}
+        del stage
+        torch.cuda.empty_cache()
+        if rank == 0:
+            line["roofline"] = gemm_roofline(qe, cfg, peaks, device)
+            line["roofline"]["gemm_share_of_step"] = round(line["roofline"]["gemm_ms_per_microbatch"] * cfg["M"] * cfg["layers"] / (ms / args.steps), 3)
+            line["hbm_kernels"] = hbm_kernels(qe, cfg, peaks, device)
+            if world == 1:
+                s, f = oracle_sample(cfg_name, cfg)
+                line["cpu_baseline"] = {"value": round(f / s / 1e12, 5), "unit": UNIT, "cores": _threads(), "kind": "oracle",
+                                        "sample": "one microbatch of all %d linears (F+dI+dW), 1/%d of a step, %.1f s" % (len(cfg["linears"]), cfg["M"] * cfg["layers"], s)}
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

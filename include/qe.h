@@ -89,6 +89,7 @@ typedef struct qe_contract qe_contract;
 typedef struct qe_registry qe_registry; /* gradient destinations bound this epoch by a group of layers (alias check) */
 
 int32_t qe_registry_create(qe_registry** out);
+/* Contracts created with a registry share ownership of it; the handle may be destroyed before or after them. */
 int32_t qe_registry_destroy(qe_registry*);
 
 /* slots in [1, QE_MAX_SLOTS]; registry may be NULL (then only this layer's own rules are checked). */
@@ -96,16 +97,16 @@ int32_t qe_contract_create(uint32_t slots, uint32_t stage, uint32_t unit, uint32
                            qe_contract** out);
 int32_t qe_contract_destroy(qe_contract*);
 
-/* Forward (Algorithm 1, lines 2-4).  check: aborted? mb < 64? gen == e_W? cache fresh (or first forward of the
+/* Forward (Algorithm 1, forward branch).  check: aborted? mb < 64? gen == e_W? cache fresh (or first forward of the
  * epoch -> *refresh_out = 1)? key not live? free slot (lowest index -> *slot_out)?  commit: occupy the slot,
  * g_p += 1, e_C <- e_W on refresh, token += 1; writes the tape. */
 int32_t qe_contract_forward_check(const qe_contract*, uint32_t mb, uint64_t gen, int32_t* refresh_out,
                                   uint32_t* slot_out);
 int32_t qe_contract_forward_commit(qe_contract*, uint32_t mb, qe_tape* tape_out);
-/* Input gradient (lines 5-7).  check: generation, key, epoch, dI bit clear.  commit: set dI bit, token += 1. */
+/* Input gradient (Algorithm 1, input-grad branch).  check: generation, key, epoch, dI bit clear.  commit: set dI bit, token += 1. */
 int32_t qe_contract_dI_check(const qe_contract*, const qe_tape*);
 int32_t qe_contract_dI_commit(qe_contract*, const qe_tape*);
-/* Weight gradient (lines 8-11).  dest_addr = address of element 0 of the flat buffer, as an integer.  check:
+/* Weight gradient (Algorithm 1, weight-grad branch).  dest_addr = address of element 0 of the flat buffer, as an integer.  check:
  * resolve; dW bit clear; dI bit set; destination valid (non-null, dest_addr + 4*offset 16-byte aligned,
  * offset + slice_elems <= dest_elems, equal to the destination bound this epoch, no overlap with another
  * layer's bound slice); this microbatch has not written; the first write of the epoch is microbatch 0.
@@ -115,7 +116,7 @@ int32_t qe_contract_dW_check(const qe_contract*, const qe_tape*, uint64_t dest_a
                              uint64_t offset, uint64_t slice_elems, int32_t* accumulate_out);
 int32_t qe_contract_dW_commit(qe_contract*, const qe_tape*, uint64_t dest_addr, uint64_t offset,
                               uint64_t slice_elems);
-/* Optimizer commit (lines 13-14): no live tape (else PENDING), every microbatch in [0, expected) wrote exactly
+/* Optimizer commit (Algorithm 1, after the loop): no live tape (else PENDING), every microbatch in [0, expected) wrote exactly
  * once (else INCOMPLETE); then e_W += 1, mask cleared, next forward refreshes the cache. */
 int32_t qe_contract_boundary(qe_contract*, uint32_t microbatches_expected);
 /* Failure boundary (Sec. 4.5): purge this epoch's tapes (generations kept), mark the arena unusable. */
@@ -159,6 +160,7 @@ typedef struct qe_layer_config {
 } qe_layer_config;
 
 int32_t qe_ctx_create(const qe_ctx_config*, qe_ctx** out);
+/* A context stays alive until it has been destroyed AND its last layer has been destroyed (either order). */
 int32_t qe_ctx_destroy(qe_ctx*);
 int32_t qe_layer_workspace_bytes(const qe_layer_config*, uint64_t* bytes_out);
 /* workspace_dev: 256-byte aligned device memory of at least qe_layer_workspace_bytes; owned by the caller, must

@@ -190,7 +190,7 @@ int32_t qe_contract_dW_commit(qe_contract* c, const qe_tape* t, uint64_t dest_ad
   return QE_OK;
 }
 
-// Algorithm 1, lines 13-14.
+// Algorithm 1, after the action loop.
 int32_t qe_contract_boundary(qe_contract* c, uint32_t expected) {
   if (!c) return fail(QE_ERR_BAD_ARG, "contract is null");
   if (c->aborted) return fail(QE_ERR_ABORTED, "step aborted");

@@ -92,7 +92,21 @@ struct qe_ctx {
   cudaEvent_t ev_in = nullptr, ev_out = nullptr;
   qe_registry* registry = nullptr;
   qe_stats stats{};
+  // Layers keep their context alive: it is released when the caller has destroyed it AND its last layer is gone,
+  // so the two destroy calls may come in either order.
+  uint32_t layers = 0;
+  bool closed = false;
 };
+
+static void ctx_release(qe_ctx* c) {
+  if (!c->closed || c->layers) return;
+  cudaStreamSynchronize(c->exec_stream);
+  cudaEventDestroy(c->ev_in);
+  cudaEventDestroy(c->ev_out);
+  cudaStreamDestroy(c->exec_stream);
+  qe_registry_destroy(c->registry);
+  delete c;
+}
 
 struct qe_layer {
   qe_ctx* ctx = nullptr;
@@ -329,13 +343,9 @@ int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
 }
 
 int32_t qe_ctx_destroy(qe_ctx* c) {
-  if (!c) return QE_OK;
-  cudaStreamSynchronize(c->exec_stream);
-  cudaEventDestroy(c->ev_in);
-  cudaEventDestroy(c->ev_out);
-  cudaStreamDestroy(c->exec_stream);
-  qe_registry_destroy(c->registry);
-  delete c;
+  if (!c || c->closed) return QE_OK;
+  c->closed = true;
+  ctx_release(c);
   return QE_OK;
 }
 
@@ -349,6 +359,7 @@ int32_t qe_layer_workspace_bytes(const qe_layer_config* cfg, uint64_t* bytes_out
 
 int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint64_t ws_bytes, qe_layer** out) {
   if (!ctx || !out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (ctx->closed) return fail(QE_ERR_BAD_ARG, "context already destroyed");
   int32_t st = check_config(cfg);
   if (st != QE_OK) return st;
   if (!cfg->weight_dev) return fail(QE_ERR_BAD_ARG, "weight_dev is null");
@@ -396,6 +407,7 @@ int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint6
     return fail(QE_ERR_CUDA, "state initialisation: %s", cudaGetErrorString(e));
   }
   ctx->stats.workspace_bytes += k.total;
+  ctx->layers += 1;
   *out = L;
   return QE_OK;
 }
@@ -411,9 +423,12 @@ int32_t qe_layer_destroy(qe_layer* L) {
   }
   destroy_graph(&L->gRefresh);
   destroy_graph(&L->gCommit);
-  L->ctx->stats.workspace_bytes -= L->ws_bytes;
+  qe_ctx* ctx = L->ctx;
+  ctx->stats.workspace_bytes -= L->ws_bytes;
   qe_contract_destroy(L->contract);
   delete L;
+  ctx->layers -= 1;
+  ctx_release(ctx);
   return QE_OK;
 }
 

@@ -1,0 +1,176 @@
+"""GPU parity of the standalone kernels against the oracle (through the C-ABI)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import bf16, fp8
+from oracle.layer import gemm_dI, gemm_dW, gemm_fwd
+from oracle.scaling import amax_bf16
+from paper_2609_23536_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+FMT = {0: fp8.E4M3, 1: fp8.E5M2}
+
+
+@pytest.fixture(scope="module")
+def qe():
+    from paper_2609_23536_b200 import build
+
+    build.build()
+    from paper_2609_23536_b200 import binding
+
+    return binding
+
+
+def _dev(bits_np):
+    return inputs.from_bits(bits_np).to(DEV)
+
+
+def _special_values(n):
+    """bf16 patterns that exercise saturation, subnormals, ties, signed zero and infinities."""
+    vals = [0.0, -0.0, 1.0, -1.0, 448.0, 464.0, -480.0, 57344.0, 61440.0, 1e30, -1e30, float("inf"), -float("inf"),
+            2.0**-9, 2.0**-10, 1.5 * 2.0**-10, 2.0**-16, 2.0**-17, 1.0625, 1.1875, 1.125, 1.375, 2.0**-126, 2.0**-133]
+    t = torch.tensor(vals, dtype=torch.float32).to(torch.bfloat16)
+    return t.repeat((n + len(vals) - 1) // len(vals))[:n]
+
+
+@pytest.mark.parametrize("rows,cols", [(64, 64), (320, 192), (2048, 1024), (4096 + 64, 2048 + 64)])
+@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("scale", [1.0, 448.0 / 3.3, 2.0**-3, 3.1e4])
+def test_quantize_bytes_transposed_copy_and_amax_bit_exact(qe, rows, cols, fmt, scale):
+    if rows > 4096 and scale != 1.0:
+        pytest.skip("large case once per format")
+    x = inputs.normal_bf16((rows, cols), 1.0 if fmt == 0 else 1e-3, "q", rows, cols, fmt)
+    x.view(-1)[: min(4096, x.numel())] = _special_values(min(4096, x.numel()))
+    xb = inputs.bits(x)
+    xd = x.to(DEV)
+    s = torch.tensor([scale], dtype=torch.float32, device=DEV)
+    q = torch.empty((rows, cols), dtype=torch.uint8, device=DEV)
+    qT = torch.empty((cols, rows), dtype=torch.uint8, device=DEV)
+    amax = torch.zeros(1, dtype=torch.float32, device=DEV)
+    qe.qe_quantize(xd, s, fmt, q, qT, amax)
+    torch.cuda.synchronize()
+    want = fp8.quantize(bf16.decode(xb), np.float32(s.item()), FMT[fmt])
+    got = q.cpu().numpy()
+    assert np.array_equal(got, want), np.argwhere(got != want)[:5]
+    assert np.array_equal(qT.cpu().numpy(), want.T)
+    a = amax_bf16(bf16.decode(xb))
+    assert amax.cpu().numpy().view(np.uint32)[0] == np.float32(a).view(np.uint32)
+    # without the optional outputs
+    q2 = torch.zeros_like(q)
+    qe.qe_quantize(xd, s, fmt, q2)
+    assert torch.equal(q2, q)
+
+
+def test_quantize_rejects_bad_shapes(qe):
+    x = torch.zeros((64, 96), dtype=torch.bfloat16, device=DEV)
+    s = torch.ones(1, device=DEV)
+    q = torch.empty((64, 96), dtype=torch.uint8, device=DEV)
+    with pytest.raises(qe.QEError) as e:
+        qe.qe_quantize(x, s, 0, q)
+    assert e.value.code == "SHAPE"
+    with pytest.raises(qe.QEError) as e:
+        qe.qe_quantize(x[:, :64].contiguous(), s, 7, q)
+    assert e.value.code == "BAD_ARG"
+
+
+@pytest.mark.parametrize("n", [8, 8 * 1000 + 8, 1 << 20, (1 << 24) + 4096])
+def test_standalone_amax(qe, n):
+    x = inputs.normal_bf16((n,), 3.0, "amax", n)
+    x[n // 3] = 1234.0
+    x[-1] = -4321.0 if n > 8 else x[-1]
+    xd = x.to(DEV)
+    part = torch.full((qe.qe_amax_partials(),), 7e9, dtype=torch.float32, device=DEV)  # stale contents must not matter
+    out = torch.zeros(1, dtype=torch.float32, device=DEV)
+    for _ in range(2):
+        qe.qe_amax(xd, part, out)
+    assert out.item() == float(amax_bf16(bf16.decode(inputs.bits(x))))
+
+
+@pytest.mark.parametrize("n", [4, 4 * 257, 1 << 22])
+def test_accumulate(qe, n):
+    a = torch.randn(n, device=DEV)
+    b = torch.randn(n, device=DEV) * 1e-3
+    d = a.clone()
+    qe.qe_accumulate(d, b, True)
+    assert torch.equal(d, a + b)  # one IEEE add per element
+    qe.qe_accumulate(d, b, False)
+    assert torch.equal(d, b)
+
+
+# ------------------------------------------------------------------------------------------ GEMM
+def _run_gemm(qe, A, afmt, B, bfmt, sa, sb, kind, init=None):
+    M, Nn = A.shape[0], B.shape[0]
+    Ad, Bd = torch.from_numpy(A).to(DEV), torch.from_numpy(B).to(DEV)
+    sad = torch.tensor([sa], dtype=torch.float32, device=DEV)
+    sbd = torch.tensor([sb], dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    amax = torch.zeros(1, dtype=torch.float32, device=DEV)
+    if kind == 0:
+        D = torch.empty((M, Nn), dtype=torch.bfloat16, device=DEV)
+    else:
+        D = init.clone().to(DEV) if init is not None else torch.full((M, Nn), float("nan"), device=DEV)
+    qe.qe_gemm_fp8(Ad, afmt, Bd, bfmt, sad, sbd, D, kind, amax if kind == 0 else None, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    return D.cpu(), amax.item()
+
+
+def _int_codes(rng, shape, lim, fmt):
+    v = rng.integers(-lim, lim + 1, shape).astype(np.float32)
+    q = fp8.encode(v, fmt)
+    assert np.array_equal(fp8.decode(q, fmt), v)
+    return q, v
+
+
+@pytest.mark.parametrize("M,Nn,Kc", [(128, 256, 128), (256, 256, 256), (384, 384, 512), (128 * 5, 256 * 3, 4096), (128 * 30, 256 * 11, 256)])
+def test_gemm_integer_inputs_are_bit_exact(qe, M, Nn, Kc):
+    # every partial sum is an integer below 2^24: exact in FP32 in any order, so layout or descriptor
+    # mistakes cannot hide behind a tolerance
+    rng = np.random.default_rng(M + Nn + Kc)
+    A, Av = _int_codes(rng, (M, Kc), 8, fp8.E4M3)
+    B, Bv = _int_codes(rng, (Nn, Kc), 4, fp8.E4M3)
+    want = Av.astype(np.float64) @ Bv.astype(np.float64).T
+    assert np.abs(want).max() < 2**24
+    D32, _ = _run_gemm(qe, A, 0, B, 0, 1.0, 1.0, 1)
+    assert np.array_equal(D32.numpy(), want.astype(np.float32))
+    Dbf, amax = _run_gemm(qe, A, 0, B, 0, 1.0, 1.0, 0)
+    wb = bf16.round_from_f64(want)
+    assert np.array_equal(inputs.bits(Dbf), wb)
+    assert amax == float(np.abs(bf16.decode(wb)).max())
+    init = torch.randint(-1000, 1000, (M, Nn)).float()
+    Dacc, _ = _run_gemm(qe, A, 0, B, 0, 1.0, 1.0, 2, init)
+    assert np.array_equal(Dacc.numpy(), init.numpy() + want.astype(np.float32))
+
+
+def test_gemm_permutation_weight_moves_columns(qe):
+    rng = np.random.default_rng(1)
+    M, K = 256, 512
+    A, Av = _int_codes(rng, (M, K), 8, fp8.E4M3)
+    perm = rng.permutation(K)
+    Bv = np.zeros((K, K), np.float32)
+    Bv[np.arange(K), perm] = 1.0
+    B = fp8.encode(Bv, fp8.E4M3)
+    D, _ = _run_gemm(qe, A, 0, B, 0, 1.0, 1.0, 1)
+    assert np.array_equal(D.numpy(), Av[:, perm])
+
+
+@pytest.mark.parametrize("afmt,bfmt", [(0, 0), (1, 0), (1, 1)])
+@pytest.mark.parametrize("M,Nn,Kc", [(256, 256, 256), (512, 640, 1024), (2048, 2048, 2048)])
+def test_gemm_random_bytes_within_tolerance(qe, afmt, bfmt, M, Nn, Kc):
+    rng = np.random.default_rng(afmt * 7 + bfmt + M)
+    A = fp8.quantize(rng.standard_normal((M, Kc)).astype(np.float32), np.float32(20.0), FMT[afmt])
+    B = fp8.quantize(rng.standard_normal((Nn, Kc)).astype(np.float32), np.float32(20.0), FMT[bfmt])
+    sa, sb = np.float32(1 / 20.0), np.float32(0.049)
+    acc = fp8.decode(A, FMT[afmt]) @ fp8.decode(B, FMT[bfmt]).T * np.float64(sa) * np.float64(sb)
+    D32, _ = _run_gemm(qe, A, afmt, B, bfmt, float(sa), float(sb), 1)
+    rel = np.linalg.norm(D32.numpy().astype(np.float64) - acc) / np.linalg.norm(acc)
+    assert rel < 1e-5, rel
+    Dbf, amax = _run_gemm(qe, A, afmt, B, bfmt, float(sa), float(sb), 0)
+    got = bf16.decode(inputs.bits(Dbf)).astype(np.float64)
+    want = bf16.decode(bf16.round_from_f64(acc)).astype(np.float64)
+    assert np.linalg.norm(got - acc) / np.linalg.norm(acc) < 1e-3 * 3
+    floor = 2.0**-6 * np.sqrt(np.mean(acc**2))
+    assert np.all(np.abs(got - want) <= 4 * bf16.ulp(np.maximum(np.abs(want), floor)))
+    assert amax == float(np.abs(got).max())  # self-consistent with what was stored

@@ -1,0 +1,229 @@
+"""GPU parity of the layer (F / dI / dW through the C-ABI) against the oracle, action by action."""
+import numpy as np
+import pytest
+import torch
+
+from harness import (assert_gemm_close, assert_grad_close, c1_inputs, run_gpu_steps, run_oracle_steps, state_equal,
+                     state_equal_except_Y)
+from oracle import bf16, fp8
+from oracle.layer import ContractError, OracleLinear
+from paper_2609_23536_b200 import inputs
+from paper_2609_23536_b200.schedules import full_backward, peak_live, sched
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def qe():
+    from paper_2609_23536_b200 import build
+
+    build.build()
+    from paper_2609_23536_b200 import binding
+
+    return binding
+
+
+def _weights(cfg, N, K, steps):
+    ws = [inputs.weights(cfg, 0, 0, N, K)]
+    for e in range(1, steps):
+        ws.append(inputs.optimizer_perturbation(ws[-1], cfg, e, 0, 0))
+    return [inputs.bits(w) for w in ws]
+
+
+def _mk_layer(qe, mode, T, K, N, H, margin, P):
+    ctx = qe.Context(mode)
+    w = torch.zeros((N, K), dtype=torch.bfloat16, device=DEV)
+    return ctx, qe.Layer(ctx, T, K, N, H, margin, P, w)
+
+
+def _scale_from_window(window, fp8_max, margin, prev):
+    m = np.float32(window.max())
+    if not (np.isfinite(m) and m > 0):
+        return prev
+    return np.float32(np.float32(np.float32(fp8_max) / m) * np.float32(2.0**-margin))
+
+
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_config1_every_action_against_oracle(qe, mode):
+    # Single linear 256^3, history 4, margin 0, 4 microbatches x 3 steps in 1F1B order: the history rolls over.
+    T = K = N = 256
+    M, steps, H = 4, 3, 4
+    s = sched(M, 1, 0)
+    P = peak_live(s)
+    W = _weights("C1", N, K, steps)
+    get = lambda step, mb: c1_inputs(step, mb, T, K, N, "C1")
+    O = OracleLinear(T, K, N, H, 0, P)
+    obuf = np.zeros(N * K + 64, np.float32)
+    otrace = []
+    oouts = run_oracle_steps(O, s, steps, M, obuf, 64, get, lambda e: W[e],
+                             on_action=lambda st, a, m, L: otrace.append((st, a, m, L.state(),
+                                       {p: (sl.Xq, sl.Gq, sl.sinv_X, sl.sinv_G) for p, sl in enumerate(L.slots) if sl.live},
+                                       L.Wq.copy(), L.cache_sinv_W)))
+    ctx, L = _mk_layer(qe, mode, T, K, N, H, 0, P)
+    gbuf = torch.full((N * K + 64,), 7.0, device=DEV)  # garbage: the first write of an epoch must overwrite
+    it = iter(otrace)
+    prevY = [np.float32(1.0)]
+
+    def check(step, a, m, layer, tape):
+        ost, oa, om, ostate, oslots, oWq, osinvW = next(it)
+        assert (ost, oa, om) == (step, a, m)
+        g = layer.state()
+        assert g["device_status"] == 0 and g["device_token"] == g["token"]
+        assert state_equal_except_Y(g, ostate), (step, a, m)
+        assert np.float32(g["cache_sinv_W"]).view(np.uint32) == np.float32(osinvW).view(np.uint32)
+        assert np.array_equal(layer.read_fp8(4), oWq) and np.array_equal(layer.read_fp8(5), oWq.T)
+        for p, (Xq, Gq, sX, sG) in oslots.items():
+            assert np.array_equal(layer.read_fp8(0, p), Xq) and np.array_equal(layer.read_fp8(1, p), Xq.T)
+            assert g["slot_sinv_X"][p].view(np.uint32) == np.float32(sX).view(np.uint32)
+            if Gq is not None:
+                assert np.array_equal(layer.read_fp8(2, p), Gq) and np.array_equal(layer.read_fp8(3, p), Gq.T)
+                assert g["slot_sinv_G"][p].view(np.uint32) == np.float32(sG).view(np.uint32)
+        # class Y: newest entry is max|Y_gpu| exactly; its scale is the closed form of the GPU's own window
+        gy = g["classes"]["Y"]
+        assert gy["count"] == ostate["classes"]["Y"]["count"]
+        want = _scale_from_window(gy["window"], 448.0, 0, prevY[0])
+        assert gy["scale"].view(np.uint32) == want.view(np.uint32)
+        assert gy["scale_inv"].view(np.uint32) == np.float32(np.float32(1.0) / want).view(np.uint32)
+        prevY[0] = want
+        oy = ostate["classes"]["Y"]["window"]
+        assert np.all(np.abs(gy["window"].astype(np.float64) - oy) <= 4 * bf16.ulp(oy))
+
+    gouts = run_gpu_steps(qe, L, s, steps, M, gbuf, 64, get, lambda e: W[e], on_action=check)
+    assert set(gouts) == set(oouts)
+    for k in oouts:
+        if k[1] == "mg":
+            assert np.array_equal(gouts[k][:64], np.full(64, 7.0, np.float32))  # nothing outside the slice
+            rel = assert_grad_close(gouts[k][64:], oouts[k][64:], k)
+            assert rel < 1e-5, rel
+        else:
+            assert_gemm_close(gouts[k], oouts[k], k)
+    # newest Y amax equals max|Y| of the last forward, exactly
+    lastY = bf16.decode(gouts[(steps - 1, "Y", M - 1)])
+    assert L.state()["classes"]["Y"]["window"][0] == np.abs(lastY).max()
+    st = ctx.stats()
+    n_actions = steps * 3 * M
+    assert st["handoffs"] == 2 * n_actions
+    if mode == 1:
+        assert st["graphs_built"] == 3 * P + 1  # one F/dI/dW triple per slot + the cache refresh
+        assert st["graph_replays"] == n_actions + steps and st["eager_launches"] == 0
+    else:
+        assert st["graphs_built"] == 0 and st["eager_launches"] == st["kernels_launched"]
+    assert st["kernels_launched"] == steps * (M * (3 + 3 + 1) + 2)
+
+
+def _run_variant(qe, mode, schedule, staged=False, T=256, K=384, N=512, M=4, steps=2, H=4):
+    P = max(peak_live(schedule), 2)
+    W = _weights("V", N, K, steps)
+    get = lambda step, mb: c1_inputs(step, mb, T, K, N, "V")
+    ctx, L = _mk_layer(qe, mode, T, K, N, H, 1, P)
+    gbuf = torch.zeros(N * K, device=DEV)
+    temp = torch.empty(N * K, device=DEV) if staged else None
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        outs = run_gpu_steps(qe, L, schedule, steps, M, gbuf, 0, get, lambda e: W[e], staged_temp=temp)
+    st = L.state()
+    return outs, {**st, "slots": [], "slot_sinv_X": 0, "slot_sinv_G": 0}
+
+
+def _same(a, b):
+    (oa, sa), (ob, sb) = a, b
+    assert oa.keys() == ob.keys()
+    for k in oa:
+        assert np.array_equal(oa[k].view(np.uint8), ob[k].view(np.uint8)), k
+    assert state_equal(sa, sb) and sa["device_token"] == sb["device_token"]
+
+
+def test_split_equals_full_backward_bitwise(qe):
+    s = sched(4, 2, 1)
+    _same(_run_variant(qe, 0, s), _run_variant(qe, 0, full_backward(s)))
+
+
+def test_graph_replay_equals_eager_bitwise(qe):
+    s = sched(4, 2, 1)
+    _same(_run_variant(qe, 0, s), _run_variant(qe, 1, s))
+    _same(_run_variant(qe, 0, full_backward(s)), _run_variant(qe, 1, s))
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_staged_copy_path_equals_direct_placement_bitwise(qe, mode):
+    s = sched(4, 2, 1)
+    _same(_run_variant(qe, mode, s), _run_variant(qe, mode, s, staged=True))
+
+
+def test_scale_commit_standalone_matches_hand_worked_rollover(qe):
+    ctx, L = _mk_layer(qe, 0, 256, 256, 256, 4, 0, 1)
+    seq = [1, 8, 2, 2, 2, 2, 0.5, 0, 0, 0, 0, 3]
+    want = [448, 56, 56, 56, 56, 224, 224, 224, 224, 896, 896, None]
+    for a, w in zip(seq, want):
+        L.scale_commit(qe.CLASS_X, torch.tensor([a], dtype=torch.float32, device=DEV))
+        s = L.state()["classes"]["X"]
+        if w is not None:
+            assert s["scale"] == np.float32(w)
+    assert s["scale"].view(np.uint32) == 0x43155555 and s["scale_inv"].view(np.uint32) == 0x3BDB6DB7
+    assert list(s["window"]) == [3.0, 0.0, 0.0, 0.0] and s["count"] == 12
+    assert L.state()["device_token"] == 0  # a standalone commit does not advance the effect token
+    # E5M2 class with margin handled by the same kernel
+    ctx2, L2 = _mk_layer(qe, 1, 256, 256, 256, 4, 1, 1)
+    for a, w in zip([1, 8, 2, 2, 2, 2], [28672, 3584, 3584, 3584, 3584, 14336]):
+        L2.scale_commit(qe.CLASS_G, torch.tensor([a], dtype=torch.float32, device=DEV))
+        assert L2.state()["classes"]["G"]["scale"] == np.float32(w)
+
+
+def test_contract_violations_through_the_layer_leave_state_untouched(qe):
+    T = K = N = 256
+    ctx, L = _mk_layer(qe, 0, T, K, N, 4, 0, 2)
+    L.weight.copy_(inputs.weights("E", 0, 0, N, K).to(DEV))
+    x = inputs.activations("E", 0, 0, 0, 0, T, K).to(DEV)
+    dy = inputs.upstream_grads("E", 0, 0, 0, 0, T, N).to(DEV)
+    y, dx = torch.empty((T, N), dtype=torch.bfloat16, device=DEV), torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+    buf = torch.zeros(N * K + 4, device=DEV)
+
+    def expect(code, fn, *a):
+        before = L.state()
+        with pytest.raises(qe.QEError) as e:
+            fn(*a)
+        assert e.value.code == code, e.value
+        after = L.state()
+        assert state_equal(before, after) and before["device_token"] == after["device_token"]
+
+    expect("EPOCH", L.forward, 0, 3, x, y)
+    t0 = L.forward(0, 0, x, y)
+    expect("KEY_LIVE", L.forward, 0, 0, x, y)
+    expect("ORDER", L.backward_dW, t0, buf, 0)
+    L.backward_dI(t0, dy, dx)
+    expect("DUP_CONSUME", L.backward_dI, t0, dy, dx)
+    expect("DEST", L.backward_dW, t0, buf, 2)
+    expect("DEST", L.backward_dW, t0, buf, 8)
+    L.backward_dW(t0, buf, 0)
+    expect("STALE_REF", L.backward_dW, t0, buf, 0)
+    t1 = L.forward(1, 0, x, y)
+    assert (t1.ref.slot, t1.ref.gen) == (0, 2)
+    expect("STALE_REF", L.backward_dI, t0, dy, dx)
+    expect("PENDING", L.optimizer_boundary, 2)
+    L.invalidate_cache()
+    expect("STALE_CACHE", L.forward, 2, 0, x, y)
+    L.abort_step()
+    expect("ABORTED", L.backward_dI, t1, dy, dx)
+    L.arena_rebuild()
+    t = L.forward(0, 0, x, y)
+    L.backward_dI(t, dy, dx)
+    L.backward_dW(t, buf, 4)
+    expect("INCOMPLETE", L.optimizer_boundary, 2)
+    L.optimizer_boundary(1)
+    assert L.state()["e_W"] == 1
+
+
+def test_bad_configs_are_rejected(qe):
+    ctx = qe.Context(0)
+    w = torch.zeros((256, 256), dtype=torch.bfloat16, device=DEV)
+    for T, K, N, code in [(200, 256, 256, "SHAPE"), (256, 0, 256, "SHAPE"), (256, 256, 128, "SHAPE")]:
+        with pytest.raises(qe.QEError) as e:
+            qe.Layer(ctx, T, K, N, 4, 0, 2, torch.zeros((N, max(K, 1)), dtype=torch.bfloat16, device=DEV)) if K else \
+                qe.lib.qe_layer_workspace_bytes and qe._check(qe.lib.qe_layer_workspace_bytes(
+                    __import__("ctypes").byref(qe.qe_layer_config(T=T, K=K, N=N, history_len=4, slots=2)),
+                    __import__("ctypes").byref(__import__("ctypes").c_uint64())))
+        assert e.value.code == code
+    with pytest.raises(qe.QEError) as e:
+        qe.Layer(ctx, 256, 256, 256, 0, 0, 2, w)
+    assert e.value.code == "BAD_ARG"
