@@ -1,0 +1,80 @@
+"""Small single-kernel cases for profiling (ncu) and quick timing.
+
+    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|quantize|quantize_t|amax|accumulate [--reps N]
+
+Each case holds well under 2 GB on the device, uses operands larger than the 126 MB L2 where DRAM traffic is
+the question, does 2 warm-up launches and then `reps` launches, and prints the CUDA-event time per launch.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import build
+
+build.build()
+from . import binding as qe  # noqa: E402
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case")
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--small", action="store_true", help="Llama-block (hidden 2048) shapes instead of Llama-3-8B ones")
+    a = ap.parse_args()
+    dev = torch.device("cuda", 0)
+    one = torch.ones(1, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    T, H, F = (2048, 2048, 11264) if a.small else (4096, 4096, 28672)
+    work = None
+    if a.case.startswith("gemm"):
+        # gate/up projection: F: [T,H]x[F,H]^T ; dI: [T,F]x[H,F]^T ; dW: [F,T]x[H,T]^T (FP32 read-modify-write)
+        M, N, Kc, af, kind = {"gemm_f": (T, F, H, 0, 0), "gemm_di": (T, H, F, 1, 0), "gemm_dw": (F, H, T, 1, 2)}[a.case]
+        A = torch.randint(0, 120, (M, Kc), dtype=torch.uint8, device=dev)
+        B = torch.randint(0, 120, (N, Kc), dtype=torch.uint8, device=dev)
+        D = torch.zeros((M, N), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=dev)
+        fn = lambda: qe.qe_gemm_fp8(A, af, B, 0, one, one, D, kind, None, status)
+        work = {"flop": 2.0 * M * N * Kc, "bytes": M * Kc + N * Kc + M * N * (2 if kind == 0 else 8)}
+    else:
+        rows, cols = 8192, 16384
+        x = torch.randn((rows, cols), device=dev).to(torch.bfloat16)
+        n = rows * cols
+        if a.case in ("quantize", "quantize_t"):
+            q = torch.empty((rows, cols), dtype=torch.uint8, device=dev)
+            qT = torch.empty((cols, rows), dtype=torch.uint8, device=dev) if a.case == "quantize_t" else None
+            amax = torch.zeros(1, device=dev)
+            fn = lambda: qe.qe_quantize(x, one, 0, q, qT, amax)
+            work = {"bytes": n * (4 if qT is not None else 3)}
+        elif a.case == "amax":
+            part = torch.empty(qe.qe_amax_partials(), device=dev)
+            out = torch.zeros(1, device=dev)
+            fn = lambda: qe.qe_amax(x, part, out)
+            work = {"bytes": 2 * n}
+        elif a.case == "accumulate":
+            g = torch.zeros(n // 2, device=dev)
+            t = torch.ones(n // 2, device=dev)
+            fn = lambda: qe.qe_accumulate(g, t, True)
+            work = {"bytes": 12 * (n // 2)}
+        else:
+            raise SystemExit("unknown case " + a.case)
+    for _ in range(2):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / a.reps
+    out = {"case": a.case, "ms": round(ms, 4), "status": int(status.item())}
+    if "flop" in work:
+        out["TFLOP/s"] = round(work["flop"] / ms / 1e9, 1)
+    out["GB/s_algorithmic"] = round(work["bytes"] / ms / 1e6, 1)
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()
