@@ -251,6 +251,26 @@ int32_t qe_gemm_fp8(const void* a_dev, uint32_t a_format, const void* b_dev, uin
                     uint32_t Nn, uint32_t Kc, const float* alpha_a_dev, const float* alpha_b_dev, void* d_dev,
                     uint32_t out_kind, float* amax_dev, uint32_t* status_dev, void* stream);
 
+/* (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
+ * The copied-gradient step without any allocation: D = (A . B^T) * *alpha_a_dev * *alpha_b_dev is written to a
+ * staging area that is built into the library (a fixed device array of qe_noalloc_staging_elems() = 2^20 FP32
+ * elements, 4 MiB, resident on every GPU that loads the library until the process exits), then
+ * dst_dev[i] = staging[i] (accumulate = 0) or dst_dev[i] += staging[i] (accumulate != 0).  Intended for code that
+ * runs where cudaMalloc is off limits: inside another framework's allocator lock, on a thread or in a callback that
+ * must not allocate, or in a process whose device memory was handed out completely at start-up.  The caller still
+ * passes every input and the output; this call and everything under it call no cudaMalloc/cudaFree and no allocating
+ * library routine.  A, B, shapes, formats, alphas and status_dev are as in qe_gemm_fp8; dst_dev is FP32 [M,Nn],
+ * 16-byte aligned.  M*Nn above 2^20 is rejected with QE_ERR_UNSUPPORTED.  The first call on each device looks up
+ * the staging area's device address (with that device current); make that first call outside any stream capture.
+ * All calls share the one staging area and it keeps the previous call's contents: every call overwrites the part
+ * it uses before reading it, so nothing needs clearing, but two calls whose work overlaps on the GPU (different
+ * streams without an ordering between them) race on it -- keep them on one stream or order them with events. */
+int32_t qe_gemm_fp8_staged_noalloc(const void* a_dev, uint32_t a_format, const void* b_dev, uint32_t b_format,
+                                   uint32_t M, uint32_t Nn, uint32_t Kc, const float* alpha_a_dev,
+                                   const float* alpha_b_dev, float* dst_dev, int32_t accumulate, uint32_t* status_dev,
+                                   void* stream);
+uint64_t qe_noalloc_staging_elems(void);
+
 const char* qe_last_error(void);
 const char* qe_status_name(int32_t status);
 /* Version of this ABI (bumped on incompatible change). */

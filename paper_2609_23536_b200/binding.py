@@ -136,6 +136,8 @@ _SIGNATURES = {
     "qe_amax_partials": (C.c_uint32, []),
     "qe_accumulate": (C.c_int32, [_P, _P, C.c_uint64, C.c_int32, _P]),
     "qe_gemm_fp8": (C.c_int32, [_P, C.c_uint32, _P, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, _P, _P, _P, C.c_uint32, _P, _P, _P]),
+    "qe_gemm_fp8_staged_noalloc": (C.c_int32, [_P, C.c_uint32, _P, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, _P, _P, _P, C.c_int32, _P, _P]),
+    "qe_noalloc_staging_elems": (C.c_uint64, []),
     "qe_last_error": (C.c_char_p, []),
     "qe_status_name": (C.c_char_p, [C.c_int32]),
     "qe_abi_version": (C.c_uint32, []),
@@ -394,3 +396,17 @@ def qe_gemm_fp8(a, a_fmt, b, b_fmt, alpha_a_dev, alpha_b_dev, d, out_kind, amax_
     assert Kc == Kc2
     _check(lib.qe_gemm_fp8(_ptr(a), a_fmt, _ptr(b), b_fmt, M, Nn, Kc, _ptr(alpha_a_dev), _ptr(alpha_b_dev), _ptr(d),
                            out_kind, _ptr(amax_dev), _ptr(status_dev), _stream(stream)))
+
+
+def qe_gemm_fp8_staged_noalloc(a, a_fmt, b, b_fmt, alpha_a_dev, alpha_b_dev, dst, accumulate: bool, status_dev, stream=None):
+    """Copied-gradient step with the library's built-in staging area (no device allocation anywhere underneath):
+    for callers that may not allocate where they run.  dst is FP32 [M, Nn] with M*Nn <= qe_noalloc_staging_elems()."""
+    M, Kc = a.shape
+    Nn, Kc2 = b.shape
+    assert Kc == Kc2
+    _check(lib.qe_gemm_fp8_staged_noalloc(_ptr(a), a_fmt, _ptr(b), b_fmt, M, Nn, Kc, _ptr(alpha_a_dev), _ptr(alpha_b_dev),
+                                          _ptr(dst), int(accumulate), _ptr(status_dev), _stream(stream)))
+
+
+def qe_noalloc_staging_elems() -> int:
+    return lib.qe_noalloc_staging_elems()
