@@ -1,0 +1,66 @@
+// Amax-history reduction and scale update as a device function, shared by the standalone commit kernel and by the
+// tails of the quantise and GEMM kernels (where the last block to finish performs it, saving a launch).
+//   hist[c][count mod H] = amax;  scale_c = fp8_max / max(hist[c]) / 2^margin;  scale_inv_c = 1 / scale_c
+// 256 threads take part: 64 per tensor class, all four classes in parallel, one barrier.  The maximum is taken on
+// the bit patterns of the non-negative FP32 entries, which orders them like their values and lets a NaN or Inf
+// entry surface as "not finite" (scale then stays as it was, like for an all-zero window).
+#pragma once
+#include <cfloat>
+
+#include "kernels.h"
+
+namespace qe {
+
+template <class Sync>
+__device__ __forceinline__ void commit_classes(const CommitParams& p, int tid, uint32_t* red /* shared, 8 words */,
+                                               Sync sync) {
+  DevState* st = p.st;
+  const int c = tid >> 6, g = tid & 63;
+  const bool active = (p.class_mask >> c) & 1u;
+  uint32_t m = 0, newest = 0, cnt = 0, pos = 0;
+  uint32_t* h = reinterpret_cast<uint32_t*>(p.hist + (size_t)c * p.H);
+  if (active) {
+    cnt = __ldcg(&st->count[c]);
+    newest = p.amax_override ? (__float_as_uint(__ldcg(p.amax_override)) & 0x7fffffffu) : __ldcg(&st->pending_amax[c]);
+    pos = cnt % p.H;
+    for (uint32_t i = g; i < p.H; i += 64) m = max(m, i == pos ? newest : __ldcg(h + i));
+  }
+  m = __reduce_max_sync(0xffffffffu, m);
+  if ((tid & 31) == 0) red[tid >> 5] = m;
+  sync();
+  if (active && g == 0) {
+    m = max(red[2 * c], red[2 * c + 1]);
+    h[pos] = newest;
+    st->count[c] = cnt + 1;
+    st->pending_amax[c] = 0;
+    if (m != 0 && m < 0x7f800000u) {
+      const float fp8_max = c == 2 ? 57344.0f : 448.0f;  // class 2 = gradients (E5M2), others E4M3
+      float s = __fmul_rn(__fdiv_rn(fp8_max, __uint_as_float(m)), p.pow2_neg_margin);
+      if (isinf(s)) s = FLT_MAX;
+      st->scale[c] = s;
+      st->scale_inv[c] = __fdiv_rn(1.0f, s);
+    }
+  }
+  if (tid == 0 && p.bump_token) st->token += 1ull;
+}
+
+// Returns true in every thread of exactly one block of the grid: the last one to get here.  Stores and atomics the
+// grid made before this call are visible to that block afterwards.
+template <class Sync>
+__device__ __forceinline__ bool last_block(uint32_t* ticket, uint32_t nblocks, int tid, uint32_t* flag /* shared */,
+                                           Sync sync) {
+  __threadfence();
+  sync();
+  if (tid == 0) {
+    const uint32_t t = atomicAdd(ticket, 1u);
+    const bool last = t == nblocks - 1;
+    if (last) atomicExch(ticket, 0u);  // ready for the next kernel that uses it
+    *flag = last ? 1u : 0u;
+  }
+  sync();
+  const bool last = *flag != 0u;
+  if (last) __threadfence();
+  return last;
+}
+
+}  // namespace qe

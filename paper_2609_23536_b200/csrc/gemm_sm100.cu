@@ -1,14 +1,24 @@
 // FP8 GEMM for sm_100a: D[M,N] = (A[M,Kc] . B[N,Kc]^T) * alpha, A and B contraction-major bytes (E4M3 or E5M2,
 // mixed freely), FP32 accumulation in tensor memory.
 //
-// Structure (one persistent CTA per SM, 192 threads):
+// Structure (one persistent CTA per SM, 320 threads):
 //   warp 0      TMA producer: cp.async.bulk.tensor 2D tiles (128-byte swizzle) into a 4-stage shared-memory ring
 //   warp 1      allocates tensor memory, then one lane issues tcgen05.mma (128 x 256 x 32 per instruction) and
 //               tcgen05.commit to release ring stages / publish a finished accumulator
-//   warps 2-5   epilogue: tcgen05.ld the 128 x 256 FP32 accumulator (each warp its own 32-lane quadrant), scale,
-//               and write bf16 (+ max|D| reduced by warp shuffles, one atomicMax per warp and tile), or FP32
-//               overwrite, or FP32 read-modify-write straight into the destination (direct gradient placement)
+//   warps 2-9   epilogue: tcgen05.ld the 128 x 256 FP32 accumulator (two warps per 32-lane quadrant, 128 columns
+//               each), scale, and write bf16 (+ max|D| reduced by warp shuffles, one atomicMax per warp and tile),
+//               or FP32 overwrite, or FP32 read-modify-write straight into the destination (direct gradient
+//               placement; the destination tile is prefetched into L2 while the main loop of the tile still runs)
+// When asked to, the last CTA to finish folds the pending amax values into their histories and updates the scales
+// (the commit that ends F and dI), so that no extra launch is needed for it.
 // Two accumulators (2 x 256 tensor-memory columns) let the epilogue of tile i overlap the main loop of tile i+1.
+//
+// Two variants share the code below.  The single-CTA one computes 128 x 256 tiles.  The paired one (used whenever M
+// is a multiple of 256) runs as clusters of two CTAs on neighbouring SMs that compute one 256 x 256 tile together
+// with tcgen05.mma.cta_group::2: each CTA loads its own 128 rows of A and its own 128 rows of B (32 KB per stage
+// instead of 48 KB, six stages), the even CTA issues the MMAs for the pair, tcgen05.commit multicasts stage-free and
+// accumulator-ready arrivals to both CTAs, and each CTA drains its own 128 accumulator rows.  That halves the
+// B-operand shared-memory traffic per SM, which is what bounds the single-CTA variant.  No TMA multicast is used.
 // Each output element is produced by exactly one thread with a fixed contraction order, so results do not depend
 // on the grid size or on how tiles are scheduled (no split-K, no atomics on data).
 //
@@ -17,18 +27,29 @@
 // where tensor memory is released.
 #include <cuda_bf16.h>
 
+#include "commit.cuh"
 #include "kernels.h"
 
 namespace qe {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 128;  // BK bytes = FP8 elements per stage along the contraction
-constexpr int STAGES = 4;
+constexpr int BM = 128, BN = 256, BK = 128;  // per-CTA rows, tile columns, bytes (= FP8 elements) per stage along K
 constexpr int UMMA_K = 32;
-constexpr uint32_t A_BYTES = BM * BK, B_BYTES = BN * BK, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t A_BYTES = BM * BK;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int THREADS = 192;
-constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int MAX_STAGES = 6;
+template <bool TWO>
+struct Cfg {
+  static constexpr int STAGES = TWO ? 6 : 4;
+  static constexpr uint32_t B_ROWS = TWO ? 128 : 256;  // rows of B this CTA loads per stage
+  static constexpr uint32_t B_BYTES = B_ROWS * BK;
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr uint32_t TILE_M = TWO ? 256 : 128;  // rows of D per tile (per cluster)
+  static constexpr uint32_t CTAS = TWO ? 2 : 1;
+};
+constexpr int THREADS = 320;
+constexpr int EPI_WARPS = 8, EPI_THREADS = EPI_WARPS * 32;
+constexpr uint32_t SMEM_BYTES = 4 * (A_BYTES + 256 * BK) + 1024 /*alignment slack*/ + 256 /*barriers, flags*/;  // both variants: 192 KB of stages
 constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;  // ~2 s at the maximum SM clock
 
 constexpr uint32_t ERR_PRODUCER = 1u, ERR_MMA = 2u, ERR_EPILOGUE = 4u;
@@ -72,6 +93,46 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       return false;
     }
   }
+}
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {  // barrier may live in the peer CTA
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster (shared::cluster window).
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load whose completion is credited to a barrier that may live in the peer CTA of the pair.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {  // arrives on `bar` in both CTAs of the pair
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3)
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -126,30 +187,49 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Tile order: m fastest, so that the CTAs running at the same time share a few B tiles and all of A through L2.
-__device__ __forceinline__ void tile_coords(uint32_t tile, uint32_t tiles_m, uint32_t& m0, uint32_t& n0) {
-  m0 = (tile % tiles_m) * BM;
-  n0 = (tile / tiles_m) * BN;
+// Tile order.  The CTAs running at the same time take consecutive tiles.  Walking the dimension of the SMALLER
+// operand fastest means that operand is swept again and again (from L2, where it fits) while the larger one is
+// streamed from HBM once.
+__device__ __forceinline__ void tile_coords(uint32_t tile, uint32_t tiles_m, uint32_t tiles_n, bool m_fastest,
+                                            uint32_t tile_m, uint32_t& m0, uint32_t& n0) {
+  if (m_fastest) {
+    m0 = (tile % tiles_m) * tile_m;
+    n0 = (tile / tiles_m) * BN;
+  } else {
+    n0 = (tile % tiles_n) * BN;
+    m0 = (tile / tiles_n) * tile_m;
+  }
 }
 
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory"); }
+
 // ------------------------------------------------------------------------------------------------ kernel
-__global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_constant__ GemmParams p) {
+template <bool TWO>
+__device__ __forceinline__ void gemm_body(const GemmParams& p) {
+  using C = Cfg<TWO>;
+  constexpr int STAGES = C::STAGES;
+  constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
   // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], then tmem address + abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * MAX_STAGES + 4));
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  uint32_t* last_flag = tmem_slot + 2;
+  uint32_t* red = tmem_slot + 4;  // 8 words for the commit's reduction
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t tiles_m = p.M / BM, tiles_n = (p.N + BN - 1) / BN;
+  const uint32_t rank = TWO ? cluster_ctarank() : 0u;  // position in the CTA pair; rank 0 issues the MMAs
+  const uint32_t tiles_m = p.M / C::TILE_M, tiles_n = (p.N + BN - 1) / BN;
   const uint32_t num_tiles = tiles_m * tiles_n;
+  const uint32_t first_tile = blockIdx.x / C::CTAS, tile_step = gridDim.x / C::CTAS;
   const uint32_t num_kb = p.Kc / BK;
+  const bool m_fastest = p.M <= p.N;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -158,20 +238,28 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_const
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);
+      mbar_init(tempty_bar(a), EPI_WARPS * C::CTAS);  // the epilogue warps of every CTA of the pair
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (TWO) {  // same warp in both CTAs of the pair
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (TWO) cluster_sync_all();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -181,15 +269,23 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_const
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (uint32_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
         uint32_t m0, n0;
-        tile_coords(tile, tiles_m, m0, n0);
+        tile_coords(tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
         for (uint32_t kb = 0; kb < num_kb; ++kb) {
           if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, ERR_PRODUCER))) break;
-          mbar_expect_tx(full_bar(s), STAGE_BYTES);
           const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_BYTES;
-          tma_load_2d(a_dst, &p.tmA, full_bar(s), (int)(kb * BK), (int)m0);
-          tma_load_2d(b_dst, &p.tmB, full_bar(s), (int)(kb * BK), (int)n0);
+          if (TWO) {
+            // both CTAs credit the even CTA's barrier, which expects the bytes of the whole pair
+            if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+            const uint32_t bar = map_to_cta(full_bar(s), 0);
+            tma_load_2d_pair(a_dst, &p.tmA, bar, (int)(kb * BK), (int)(m0 + rank * BM));
+            tma_load_2d_pair(b_dst, &p.tmB, bar, (int)(kb * BK), (int)(n0 + rank * C::B_ROWS));
+          } else {
+            mbar_expect_tx(full_bar(s), STAGE_BYTES);
+            tma_load_2d(a_dst, &p.tmA, full_bar(s), (int)(kb * BK), (int)m0);
+            tma_load_2d(b_dst, &p.tmB, full_bar(s), (int)(kb * BK), (int)n0);
+          }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
       }
@@ -201,11 +297,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_const
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       int s = 0;
       uint32_t ph = 0, acc = 0, acc_ph = 0;
       bool ok = true;
-      for (uint32_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
         if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, ERR_MMA))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
@@ -217,38 +313,52 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_const
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 32 bytes along the contraction inside the 128-byte swizzle row: +2 in the address field
-            tc_mma_f8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | (uint32_t)k) != 0u);
+            if (TWO) tc_mma_f8_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | (uint32_t)k) != 0u);
+            else tc_mma_f8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | (uint32_t)k) != 0u);
           }
-          tc_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+          if (TWO) tc_commit_pair(empty_bar(s));  // stage reusable (in both CTAs) once these MMAs have read it
+          else tc_commit(empty_bar(s));
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(tfull_bar(acc));  // accumulator complete
+        if (TWO) tc_commit_pair(tfull_bar(acc));  // accumulator complete (each CTA holds its 128 rows)
+        else tc_commit(tfull_bar(acc));
         if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
       }
     }
   } else {
-    // ---------------------------------------------------------------- epilogue (warps 2..5)
-    const uint32_t quad = (uint32_t)warp & 3u;  // tensor-memory lane quadrant this warp may read
+    // ---------------------------------------------------------------- epilogue (warps 2..9)
+    const uint32_t quad = (uint32_t)warp & 3u;          // tensor-memory lane quadrant this warp may read
+    const uint32_t half = ((uint32_t)warp - 2u) >> 2;   // which 128 of the tile's 256 columns
+    const int etid = (int)threadIdx.x - 64;
     const float alpha = __fmul_rn(*p.alpha_a, *p.alpha_b);
     uint32_t acc = 0, acc_ph = 0;
     bool ok = true;
-    for (uint32_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+    const uint32_t tempty_leader0 = TWO ? map_to_cta(tempty_bar(0), 0) : tempty_bar(0);
+    const uint32_t tempty_leader1 = TWO ? map_to_cta(tempty_bar(1), 0) : tempty_bar(1);
+    for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
       uint32_t m0, n0;
-      tile_coords(tile, tiles_m, m0, n0);
+      tile_coords(tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
+      const uint32_t row = m0 + rank * BM + quad * 32u + (uint32_t)lane;
+      const uint32_t col0 = n0 + half * 128u;
+      if (p.epi == 2 && col0 < p.N) {
+        // read-modify-write: pull this thread's 512 destination bytes towards L2 while the MMAs of the tile run
+        const char* d = reinterpret_cast<const char*>(reinterpret_cast<const float*>(p.out) + (size_t)row * p.ldo + col0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) asm volatile("prefetch.global.L2 [%0];" ::"l"(d + 128 * j));
+      }
       if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, ERR_EPILOGUE))) break;
       tc_fence_after();
-      const uint32_t row = m0 + quad * 32u + (uint32_t)lane;
-      const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN;
+      const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN + half * 128u;
       uint32_t amax_bits = 0;
 #pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        const uint32_t col = n0 + ch * 32u;
+      for (int ch = 0; ch < 4; ++ch) {
+        const uint32_t col = col0 + ch * 32u;
         if (col >= p.N) break;  // ragged last column tile (N a multiple of 128 but not of 256); warp-uniform
         uint32_t r[32];
         tmem_ld32(t_row + ch * 32u, r);
-        tmem_ld_wait();
         if (p.epi == 0) {
+          tmem_ld_wait();
           uint32_t o[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
@@ -266,7 +376,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_const
           if (p.epi == 2) {
             float4 old[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) old[j] = dst[j];
+            for (int j = 0; j < 8; ++j) old[j] = dst[j];  // in flight together with the tensor-memory load
+            tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               float4 v;
@@ -277,6 +388,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_const
               dst[j] = v;
             }
           } else {
+            tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               float4 v;
@@ -292,39 +404,76 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_const
       // accumulator drained: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {
+        if (TWO) mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);  // the MMA issuer waits in the even CTA
+        else mbar_arrive(tempty_bar(acc));
+      }
       if (p.epi == 0 && p.amax_bits) {
         const uint32_t w = __reduce_max_sync(0xffffffffu, amax_bits);
         if (lane == 0 && w) atomicMax(p.amax_bits, w);
       }
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
+    if (p.commit.st) {
+      // every epilogue thread of every CTA gets here (also after a timeout); the last CTA commits the scale state
+      if (last_block(&p.commit.st->ticket, gridDim.x, etid, last_flag, epi_bar_sync))
+        commit_classes(p.commit, etid, red, epi_bar_sync);
+    }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (TWO) cluster_sync_all();  // no arrival may still be on its way to a CTA that has left
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (TWO)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+}
+
+__global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_constant__ GemmParams p) { gemm_body<false>(p); }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+    gemm_fp8_pair_kernel(const __grid_constant__ GemmParams p) {
+  gemm_body<true>(p);
 }
 
 }  // namespace
 
-uint32_t gemm_idesc(int a_fmt, int b_fmt) {
+bool gemm_uses_pair(uint32_t M) { return M % 256 == 0; }
+
+uint32_t gemm_b_box_rows(uint32_t M) { return gemm_uses_pair(M) ? 128u : 256u; }
+
+uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M) {
   // bits 4-5: accumulator format (1 = FP32); 7-9 / 10-12: A / B format (0 = E4M3, 1 = E5M2); 15 / 16: A / B major
-  // (0 = contraction-major); 17-22: N >> 3; 24-28: M >> 4.
+  // (0 = contraction-major); 17-22: N >> 3; 24-28: M >> 4 (128 per CTA, 256 for a CTA pair).
+  const uint32_t mma_m = gemm_uses_pair(M) ? 256u : 128u;
   return (1u << 4) | ((uint32_t)a_fmt << 7) | ((uint32_t)b_fmt << 10) | ((uint32_t)(BN >> 3) << 17) |
-         ((uint32_t)(BM >> 4) << 24);
+         ((mma_m >> 4) << 24);
 }
 
 cudaError_t gemm_prepare() {
-  return cudaFuncSetAttribute((const void*)gemm_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute((const void*)gemm_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute((const void*)gemm_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)SMEM_BYTES);
 }
 
 Launch make_gemm(const GemmParams& p, int num_sms) {
   Launch l;
+  if (gemm_uses_pair(p.M)) {
+    l.func = (const void*)gemm_fp8_pair_kernel;
+    const uint32_t ctas = 2u * (p.M / 256u) * ((p.N + BN - 1) / BN);
+    const uint32_t cap = (uint32_t)num_sms & ~1u;
+    l.grid = dim3(ctas < cap ? ctas : cap, 1, 1);
+    l.block = dim3(THREADS, 1, 1);
+    l.smem = SMEM_BYTES;
+    l.set(p);
+    return l;
+  }
   l.func = (const void*)gemm_fp8_kernel;
   const uint32_t tiles = (p.M / BM) * ((p.N + BN - 1) / BN);
   l.grid = dim3(tiles < (uint32_t)num_sms ? tiles : (uint32_t)num_sms, 1, 1);

@@ -21,9 +21,20 @@ struct DevState {
   uint32_t status;             // error bits ORed in by kernels whose bounded waits expired
   float slot_sinv_X[64];       // inverse scales snapshotted when X_m / dY_m were quantised (per tape slot)
   float slot_sinv_G[64];
-  uint32_t pad[44];            // header is 768 bytes; history rings [4][H] follow
+  uint32_t ticket;             // "last CTA" counter of the kernel whose tail performs the commit; self-resetting
+  uint32_t pad[43];            // header is 768 bytes; history rings [4][H] follow
 };
 static_assert(sizeof(DevState) == 768, "DevState layout");
+
+struct CommitParams {
+  DevState* st;                // null: nothing to commit
+  float* hist;                 // [4][H]
+  uint32_t H;
+  uint32_t class_mask;         // bit c set: commit class c from pending_amax[c] (or from amax_override)
+  float pow2_neg_margin;       // 2^-margin
+  uint32_t bump_token;         // 1 for F and dI, 0 otherwise
+  const float* amax_override;  // if non-null: value to push for the single class in class_mask
+};
 
 struct QuantParams {
   const uint16_t* x;           // bf16 [rows, cols]
@@ -35,18 +46,9 @@ struct QuantParams {
   float* sinv_dst;
   uint32_t* amax_bits;         // atomicMax target or null
   int32_t fmt;                 // 0 = E4M3, 1 = E5M2
+  CommitParams commit;         // performed by the last block to finish (commit.st != null)
 };
 
-struct CommitParams {
-  DevState* st;
-  float* hist;                 // [4][H]
-  uint32_t H;
-  uint32_t class_mask;         // bit c set: commit class c from pending_amax[c] (or from amax_override)
-  float pow2_neg_margin;       // 2^-margin
-  const float* amax_override;  // if non-null: value to push for the single class in class_mask
-  uint32_t bump_token;         // 1 for F and dI, 0 for a standalone commit
-  uint32_t pad;
-};
 
 struct AmaxParams {
   const uint4* x;              // bf16, 8 per vector
@@ -67,7 +69,7 @@ struct AccumParams {
 
 struct GemmParams {
   CUtensorMap tmA;             // A [M, Kc] bytes, box 128 x 128, 128-byte swizzle
-  CUtensorMap tmB;             // B [N, Kc] bytes, box 128 x 256
+  CUtensorMap tmB;             // B [N, Kc] bytes, box 128 x gemm_b_box_rows(M)
   uint32_t M, N, Kc;
   uint32_t idesc;              // tcgen05 instruction descriptor (formats, 128 x 256 shape)
   const float* alpha_a;
@@ -77,6 +79,7 @@ struct GemmParams {
   int32_t epi;                 // 0 bf16 (+amax), 1 FP32 overwrite, 2 FP32 accumulate
   uint32_t* amax_bits;         // or null
   uint32_t* status;
+  CommitParams commit;         // performed by the last CTA to finish (commit.st != null)
 };
 
 // One launch, self-contained.
@@ -101,7 +104,8 @@ Launch make_amax_pass2(const AmaxParams& p);
 Launch make_accumulate(const AccumParams& p);
 Launch make_gemm(const GemmParams& p, int num_sms);
 cudaError_t gemm_prepare();  // opt in to the dynamic shared memory the GEMM needs (once per device)
-uint32_t gemm_idesc(int a_fmt, int b_fmt);
+uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M);
+uint32_t gemm_b_box_rows(uint32_t M);  // rows of the B operand's TMA box for a GEMM with M rows (128 paired, 256 single)
 constexpr uint32_t kAmaxPartials = 2048;
 
 }  // namespace qe

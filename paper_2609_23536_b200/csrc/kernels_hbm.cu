@@ -6,6 +6,7 @@
 
 #include <cfloat>
 
+#include "commit.cuh"
 #include "kernels.h"
 
 namespace qe {
@@ -95,8 +96,9 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_co
       }
     }
   }
+  __shared__ uint32_t wmax[kQuantThreads / 32];
+  __shared__ uint32_t last_flag;
   if (p.amax_bits) {
-    __shared__ uint32_t wmax[kQuantThreads / 32];
     const uint32_t w = warp_max_u32(packed_to_f32bits(m));
     if (lane == 0) wmax[warp] = w;
     __syncthreads();
@@ -106,6 +108,11 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_co
       for (int i = 1; i < kQuantThreads / 32; ++i) b = max(b, wmax[i]);
       if (b) atomicMax(p.amax_bits, b);
     }
+  }
+  if (p.commit.st) {  // the last block to finish folds the new amax into the history and updates the scale
+    auto sync = [] { __syncthreads(); };
+    if (last_block(&p.commit.st->ticket, gridDim.x * gridDim.y, threadIdx.x, &last_flag, sync))
+      commit_classes(p.commit, threadIdx.x, wmax, sync);
   }
 }
 
@@ -119,40 +126,10 @@ Launch make_quantize(const QuantParams& p) {
 }
 
 // ------------------------------------------------------------------------------------------------ commit
-// Amax-history reduction and scale update: hist[c][count mod H] = amax; scale = fp8_max / max(hist) / 2^margin.
-// One block; latency-bound (at most 16 KB read).  The maximum is taken on the bit patterns of the non-negative
-// FP32 entries, which orders them like their values and lets a NaN or Inf entry surface as "not finite".
+// The scale update as a kernel of its own (one block; latency-bound: at most 16 KB read).
 __global__ void __launch_bounds__(256) commit_kernel(const __grid_constant__ CommitParams p) {
   __shared__ uint32_t red[8];
-  DevState* st = p.st;
-  for (int c = 0; c < 4; ++c) {
-    if (!((p.class_mask >> c) & 1u)) continue;
-    const uint32_t cnt = st->count[c];
-    uint32_t* h = reinterpret_cast<uint32_t*>(p.hist + (size_t)c * p.H);
-    const uint32_t newest =
-        p.amax_override ? (__float_as_uint(*p.amax_override) & 0x7fffffffu) : st->pending_amax[c];
-    const uint32_t pos = cnt % p.H;
-    uint32_t m = 0;
-    for (uint32_t i = threadIdx.x; i < p.H; i += blockDim.x) m = max(m, i == pos ? newest : h[i]);
-    m = warp_max_u32(m);
-    __syncthreads();  // previous class's reads of red[] are done
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int i = 1; i < 8; ++i) m = max(m, red[i]);
-      h[pos] = newest;
-      st->count[c] = cnt + 1;
-      st->pending_amax[c] = 0;
-      if (m != 0 && m < 0x7f800000u) {
-        const float fp8_max = c == 2 ? 57344.0f : 448.0f;
-        float s = __fmul_rn(__fdiv_rn(fp8_max, __uint_as_float(m)), p.pow2_neg_margin);
-        if (isinf(s)) s = FLT_MAX;
-        st->scale[c] = s;
-        st->scale_inv[c] = __fdiv_rn(1.0f, s);
-      }
-    }
-  }
-  if (threadIdx.x == 0 && p.bump_token) st->token += 1ull;
+  commit_classes(p, threadIdx.x, red, [] { __syncthreads(); });
 }
 
 Launch make_commit(const CommitParams& p) {

@@ -286,7 +286,7 @@ int32_t check_config(const qe_layer_config* c) {
   return QE_OK;
 }
 
-qe::Launch commit_launch(qe_layer* L, uint32_t mask, uint32_t bump, const float* override_amax) {
+qe::CommitParams commit_params(qe_layer* L, uint32_t mask, uint32_t bump, const float* override_amax) {
   qe::CommitParams cp{};
   cp.st = L->st;
   cp.hist = L->hist;
@@ -295,11 +295,12 @@ qe::Launch commit_launch(qe_layer* L, uint32_t mask, uint32_t bump, const float*
   cp.pow2_neg_margin = std::ldexp(1.0f, -L->cfg.margin);
   cp.amax_override = override_amax;
   cp.bump_token = bump;
-  return qe::make_commit(cp);
+  return cp;
 }
 
+// commit_mask != 0: the kernel's last block also commits those classes (used for the weight refresh)
 qe::Launch quant_launch(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uint32_t rows, uint32_t cols, int cls,
-                        float* sinv_dst, int fmt) {
+                        float* sinv_dst, int fmt, uint32_t commit_mask = 0) {
   qe::QuantParams qp{};
   qp.x = (const uint16_t*)x;
   qp.q = q;
@@ -311,6 +312,7 @@ qe::Launch quant_launch(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uin
   qp.sinv_dst = sinv_dst;
   qp.amax_bits = &L->st->pending_amax[cls];
   qp.fmt = fmt;
+  if (commit_mask) qp.commit = commit_params(L, commit_mask, 0, nullptr);
   return qe::make_quantize(qp);
 }
 
@@ -390,10 +392,10 @@ int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint6
     if ((st = make_map(d, &L->tmXq_A[p], L->Xq[p], T, K, 128)) != QE_OK) break;   // F:  A = Xq  [T,K]
     if ((st = make_map(d, &L->tmGq_A[p], L->Gq[p], T, N, 128)) != QE_OK) break;   // dI: A = Gq  [T,N]
     if ((st = make_map(d, &L->tmGqT_A[p], L->GqT[p], N, T, 128)) != QE_OK) break; // dW: A = Gq^T [N,T]
-    if ((st = make_map(d, &L->tmXqT_B[p], L->XqT[p], K, T, 256)) != QE_OK) break; // dW: B = Xq^T [K,T]
+    if ((st = make_map(d, &L->tmXqT_B[p], L->XqT[p], K, T, qe::gemm_b_box_rows(N))) != QE_OK) break; // dW: B = Xq^T [K,T]
   }
-  if (st == QE_OK) st = make_map(d, &L->tmWq_B, L->Wq, N, K, 256);    // F:  B = Wq   [N,K]
-  if (st == QE_OK) st = make_map(d, &L->tmWqT_B, L->WqT, K, N, 256);  // dI: B = Wq^T [K,N]
+  if (st == QE_OK) st = make_map(d, &L->tmWq_B, L->Wq, N, K, qe::gemm_b_box_rows(T));    // F:  B = Wq   [N,K]
+  if (st == QE_OK) st = make_map(d, &L->tmWqT_B, L->WqT, K, N, qe::gemm_b_box_rows(T));  // dI: B = Wq^T [K,N]
   if (st != QE_OK) { qe_contract_destroy(L->contract); delete L; return st; }
   // state: histories 0, scales 1, everything else 0
   qe::DevState init{};
@@ -446,8 +448,8 @@ int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* 
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
   if (refresh) {  // Invariant 3: first forward of the epoch re-quantises the weight and commits its amax
     std::vector<qe::Launch> ls;
-    ls.push_back(quant_launch(L, L->cfg.weight_dev, L->Wq, L->WqT, N, K, QE_CLASS_W, &L->st->cache_sinv_W, QE_E4M3));
-    ls.push_back(commit_launch(L, 1u << QE_CLASS_W, 0, nullptr));
+    ls.push_back(quant_launch(L, L->cfg.weight_dev, L->Wq, L->WqT, N, K, QE_CLASS_W, &L->st->cache_sinv_W, QE_E4M3,
+                              1u << QE_CLASS_W));
     if ((st = run_action(ctx, &L->gRefresh, ls)) != QE_OK) return st;
   }
   std::vector<qe::Launch> ls;
@@ -458,7 +460,7 @@ int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* 
   gp.M = T;
   gp.N = N;
   gp.Kc = K;
-  gp.idesc = qe::gemm_idesc(QE_E4M3, QE_E4M3);
+  gp.idesc = qe::gemm_idesc(QE_E4M3, QE_E4M3, T);
   gp.alpha_a = &L->st->slot_sinv_X[p];
   gp.alpha_b = &L->st->cache_sinv_W;
   gp.out = y;
@@ -466,8 +468,8 @@ int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* 
   gp.epi = 0;
   gp.amax_bits = &L->st->pending_amax[QE_CLASS_Y];
   gp.status = &L->st->status;
+  gp.commit = commit_params(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr);  // done by the GEMM's last CTA
   ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
-  ls.push_back(commit_launch(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr));
   if ((st = run_action(ctx, &L->gF[p], ls)) != QE_OK) return st;  // ... run ...
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
   return qe_contract_forward_commit(L->contract, mb, tape_out);  // ... commit
@@ -490,7 +492,7 @@ int32_t qe_backward_dI(qe_layer* L, const qe_tape* tape, const void* dy, void* d
   gp.M = T;
   gp.N = K;
   gp.Kc = N;
-  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3);
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, T);
   gp.alpha_a = &L->st->slot_sinv_G[p];
   gp.alpha_b = &L->st->cache_sinv_W;
   gp.out = dx;
@@ -498,8 +500,8 @@ int32_t qe_backward_dI(qe_layer* L, const qe_tape* tape, const void* dy, void* d
   gp.epi = 0;
   gp.amax_bits = nullptr;
   gp.status = &L->st->status;
+  gp.commit = commit_params(L, 1u << QE_CLASS_G, 1, nullptr);  // backward amax/scale updated exactly once, here
   ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
-  ls.push_back(commit_launch(L, 1u << QE_CLASS_G, 1, nullptr));  // backward amax/scale updated exactly once, here
   if ((st = run_action(ctx, &L->gDI[p], ls)) != QE_OK) return st;
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
   return qe_contract_dI_commit(L->contract, tape);
@@ -523,7 +525,7 @@ static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, u
   gp.M = N;
   gp.N = K;
   gp.Kc = T;
-  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3);
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, N);
   gp.alpha_a = &L->st->slot_sinv_G[p];  // snapshots taken when dY_m and X_m were quantised, never the current state
   gp.alpha_b = &L->st->slot_sinv_X[p];
   gp.ldo = K;
@@ -585,7 +587,7 @@ int32_t qe_scale_commit(qe_layer* L, uint32_t cls, const float* amax_dev, void* 
   int32_t st;
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
   std::vector<qe::Launch> ls;
-  ls.push_back(commit_launch(L, 1u << cls, 0, amax_dev));
+  ls.push_back(qe::make_commit(commit_params(L, 1u << cls, 0, amax_dev)));
   if ((st = run_action(ctx, &L->gCommit, ls)) != QE_OK) return st;
   return handoff_out(ctx, caller);
 }
@@ -735,11 +737,11 @@ int32_t qe_gemm_fp8(const void* a, uint32_t a_fmt, const void* b, uint32_t b_fmt
   if (st != QE_OK) return st;
   qe::GemmParams gp{};
   if ((st = make_map(dev, &gp.tmA, a, M, Kc, 128)) != QE_OK) return st;
-  if ((st = make_map(dev, &gp.tmB, b, Nn, Kc, 256)) != QE_OK) return st;
+  if ((st = make_map(dev, &gp.tmB, b, Nn, Kc, qe::gemm_b_box_rows(M))) != QE_OK) return st;
   gp.M = M;
   gp.N = Nn;
   gp.Kc = Kc;
-  gp.idesc = qe::gemm_idesc((int)a_fmt, (int)b_fmt);
+  gp.idesc = qe::gemm_idesc((int)a_fmt, (int)b_fmt, M);
   gp.alpha_a = alpha_a;
   gp.alpha_b = alpha_b;
   gp.out = d;
