@@ -6,9 +6,11 @@
 //   warp 1      allocates tensor memory, then one lane issues tcgen05.mma (128 x 256 x 32 per instruction) and
 //               tcgen05.commit to release ring stages / publish a finished accumulator
 //   warps 2-9   epilogue: tcgen05.ld the 128 x 256 FP32 accumulator (two warps per 32-lane quadrant, 128 columns
-//               each), scale, and write bf16 (+ max|D| reduced by warp shuffles, one atomicMax per warp and tile),
-//               or FP32 overwrite, or FP32 read-modify-write straight into the destination (direct gradient
-//               placement; the destination tile is prefetched into L2 while the main loop of the tile still runs)
+//               each) in 32 x 32 blocks, scale, turn each block through a padded per-warp shared-memory buffer so
+//               that global accesses are coalesced (a lane owns 4 consecutive columns, a warp instruction covers
+//               four 128-byte row segments), and write bf16 (+ max|D| reduced by warp shuffles, one atomicMax per
+//               warp and tile), or FP32 overwrite, or FP32 read-modify-write straight into the destination (direct
+//               gradient placement; the destination tile is prefetched into L2 while the tile's main loop runs)
 // When asked to, the last CTA to finish folds the pending amax values into their histories and updates the scales
 // (the commit that ends F and dI), so that no extra launch is needed for it.
 // Two accumulators (2 x 256 tensor-memory columns) let the epilogue of tile i overlap the main loop of tile i+1.
@@ -38,9 +40,11 @@ constexpr int UMMA_K = 32;
 constexpr uint32_t A_BYTES = BM * BK;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int MAX_STAGES = 6;
+constexpr uint32_t EPI_ROW_WORDS = 36;                       // 32 columns + 4 words of padding: conflict-free both ways
+constexpr uint32_t EPI_BUF_BYTES = 32 * EPI_ROW_WORDS * 4;    // per epilogue warp
 template <bool TWO>
 struct Cfg {
-  static constexpr int STAGES = TWO ? 6 : 4;
+  static constexpr int STAGES = TWO ? 5 : 3;
   static constexpr uint32_t B_ROWS = TWO ? 128 : 256;  // rows of B this CTA loads per stage
   static constexpr uint32_t B_BYTES = B_ROWS * BK;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
@@ -49,7 +53,9 @@ struct Cfg {
 };
 constexpr int THREADS = 320;
 constexpr int EPI_WARPS = 8, EPI_THREADS = EPI_WARPS * 32;
-constexpr uint32_t SMEM_BYTES = 4 * (A_BYTES + 256 * BK) + 1024 /*alignment slack*/ + 256 /*barriers, flags*/;  // both variants: 192 KB of stages
+static_assert(EPI_WARPS == 8, "shared-memory budget below assumes 8 epilogue warps");
+constexpr uint32_t SMEM_BYTES = 5 * (A_BYTES + 128 * BK) + 1024 /*alignment slack*/ + 256 /*barriers, flags*/ +
+                                8 * EPI_BUF_BYTES;  // 160 KB of stages (144 KB for the single-CTA variant)
 constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;  // ~2 s at the maximum SM clock
 
 constexpr uint32_t ERR_PRODUCER = 1u, ERR_MMA = 2u, ERR_EPILOGUE = 4u;
@@ -331,6 +337,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
     const uint32_t quad = (uint32_t)warp & 3u;          // tensor-memory lane quadrant this warp may read
     const uint32_t half = ((uint32_t)warp - 2u) >> 2;   // which 128 of the tile's 256 columns
     const int etid = (int)threadIdx.x - 64;
+    float* epi_buf = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + 256 + (uint32_t)(warp - 2) * EPI_BUF_BYTES);
     const float alpha = __fmul_rn(*p.alpha_a, *p.alpha_b);
     uint32_t acc = 0, acc_ph = 0;
     bool ok = true;
@@ -351,55 +358,61 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN + half * 128u;
       uint32_t amax_bits = 0;
+      // coalesced view of a 32 x 32 block: this lane owns columns 4*(lane%8)..+3 of rows it*4 + lane/8, it = 0..7
+      const uint32_t blk_row0 = m0 + rank * BM + quad * 32u, sub_row = (uint32_t)lane >> 3, sub_col = ((uint32_t)lane & 7u) * 4u;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {
         const uint32_t col = col0 + ch * 32u;
         if (col >= p.N) break;  // ragged last column tile (N a multiple of 128 but not of 256); warp-uniform
         uint32_t r[32];
         tmem_ld32(t_row + ch * 32u, r);
+        float4 old[8];
+        if (p.epi == 2) {
+          const float* src = reinterpret_cast<const float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
+#pragma unroll
+          for (int it = 0; it < 8; ++it)  // in flight together with the tensor-memory load
+            old[it] = *reinterpret_cast<const float4*>(src + (size_t)(it * 4) * p.ldo);
+        }
+        tmem_ld_wait();
+        // row-wise (lane = row) into the padded buffer
+        float4* wr = reinterpret_cast<float4*>(epi_buf + (uint32_t)lane * EPI_ROW_WORDS);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float4 v;
+          v.x = __fmul_rn(__uint_as_float(r[4 * j]), alpha);
+          v.y = __fmul_rn(__uint_as_float(r[4 * j + 1]), alpha);
+          v.z = __fmul_rn(__uint_as_float(r[4 * j + 2]), alpha);
+          v.w = __fmul_rn(__uint_as_float(r[4 * j + 3]), alpha);
+          wr[j] = v;
+        }
+        __syncwarp();
+        const float* rd = epi_buf + sub_row * EPI_ROW_WORDS + sub_col;
         if (p.epi == 0) {
-          tmem_ld_wait();
-          uint32_t o[16];
+          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float a = __fmul_rn(__uint_as_float(r[2 * j]), alpha);
-            const float b = __fmul_rn(__uint_as_float(r[2 * j + 1]), alpha);
-            o[j] = pack_bf16(a, b);
+          for (int it = 0; it < 8; ++it) {
+            const float4 v = *reinterpret_cast<const float4*>(rd + it * 4 * EPI_ROW_WORDS);
+            const uint32_t o0 = pack_bf16(v.x, v.y), o1 = pack_bf16(v.z, v.w);
             // magnitude of the rounded values actually stored, as FP32 bit patterns (bf16 bits << 16)
-            amax_bits = max(amax_bits, max((o[j] << 16) & 0x7fffffffu, o[j] & 0x7fff0000u));
+            amax_bits = max(amax_bits, max(max((o0 << 16) & 0x7fffffffu, o0 & 0x7fff0000u),
+                                           max((o1 << 16) & 0x7fffffffu, o1 & 0x7fff0000u)));
+            *reinterpret_cast<uint2*>(dst + (size_t)(it * 4) * p.ldo) = make_uint2(o0, o1);
           }
-          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)row * p.ldo + col);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
         } else {
-          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + (size_t)row * p.ldo + col);
-          if (p.epi == 2) {
-            float4 old[8];
+          float* dst = reinterpret_cast<float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) old[j] = dst[j];  // in flight together with the tensor-memory load
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              float4 v;
-              v.x = __fadd_rn(old[j].x, __fmul_rn(__uint_as_float(r[4 * j]), alpha));
-              v.y = __fadd_rn(old[j].y, __fmul_rn(__uint_as_float(r[4 * j + 1]), alpha));
-              v.z = __fadd_rn(old[j].z, __fmul_rn(__uint_as_float(r[4 * j + 2]), alpha));
-              v.w = __fadd_rn(old[j].w, __fmul_rn(__uint_as_float(r[4 * j + 3]), alpha));
-              dst[j] = v;
+          for (int it = 0; it < 8; ++it) {
+            float4 v = *reinterpret_cast<const float4*>(rd + it * 4 * EPI_ROW_WORDS);
+            if (p.epi == 2) {
+              v.x = __fadd_rn(old[it].x, v.x);
+              v.y = __fadd_rn(old[it].y, v.y);
+              v.z = __fadd_rn(old[it].z, v.z);
+              v.w = __fadd_rn(old[it].w, v.w);
             }
-          } else {
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              float4 v;
-              v.x = __fmul_rn(__uint_as_float(r[4 * j]), alpha);
-              v.y = __fmul_rn(__uint_as_float(r[4 * j + 1]), alpha);
-              v.z = __fmul_rn(__uint_as_float(r[4 * j + 2]), alpha);
-              v.w = __fmul_rn(__uint_as_float(r[4 * j + 3]), alpha);
-              dst[j] = v;
-            }
+            *reinterpret_cast<float4*>(dst + (size_t)(it * 4) * p.ldo) = v;
           }
         }
+        __syncwarp();  // the buffer is rewritten by the next block
       }
       // accumulator drained: hand it back to the MMA warp
       tc_fence_before();
