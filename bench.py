@@ -97,11 +97,13 @@ class ClockSampler:
 class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
-    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False):
+    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
-        self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0)
+        # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
+        self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
+                              exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None)
         self.schedule = sched(cfg["M"], *cfg["sched"])
         P = peak_live(self.schedule)
         T, M = cfg["T"], cfg["M"]
@@ -135,10 +137,12 @@ class Stage:
         self.grad_host = torch.empty(self.grad.shape, dtype=torch.float32).pin_memory() if host_io else None
         self.epoch = 0
         self.h2d = self.d2h = 0
+        self.issue_s = 0.0
 
     def step(self, host_io=False):
         tapes = {}
         n = len(self.layers)
+        t_issue = time.perf_counter()
         for a, m in self.schedule:
             order = range(n) if a == "F" else range(n - 1, -1, -1)
             for i in order:
@@ -158,6 +162,7 @@ class Stage:
         if host_io:
             self.grad_host.copy_(self.grad, non_blocking=True)
             self.d2h += self.grad.numel() * 4
+        self.issue_s += time.perf_counter() - t_issue  # host time to enqueue the step (before the boundary's sync)
         for L in self.layers:
             L.optimizer_boundary(self.cfg["M"])
         self.epoch += 1
@@ -172,6 +177,7 @@ def time_steps(stage, steps, warmup, host_io, dist):
     if dist is not None:
         dist.barrier()
     stage.h2d = stage.d2h = 0
+    stage.issue_s = 0.0
     k0 = stage.ctx.stats()["kernels_launched"]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -346,6 +352,7 @@ def main():
     ap.add_argument("--mode", default="graph", choices=["graph", "eager"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, roofline, HBM-kernel and CPU-baseline legs")
+    ap.add_argument("--own-stream", action="store_true", help="let the context create its own execution stream (event handoff on every action)")
     args = ap.parse_args()
     cfg_name, cfg = args.config, inputs.CONFIGS[args.config]
     if args.impl == "reference":
@@ -370,10 +377,11 @@ def main():
 
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     device = torch.device("cuda", local)
+    torch.cuda.set_stream(torch.cuda.Stream(device))  # everything below is issued on this (non-default) stream
     peaks = _peaks()
     args.warmup = max(args.warmup, 3)
 
-    stage = Stage(qe, cfg_name, cfg, args.mode, device)
+    stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream)
     with ClockSampler(local) as clk:
         ms, launches = time_steps(stage, args.steps, args.warmup, False, dist)
     clocks = clk.summary()
@@ -388,12 +396,13 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),
         },
         "gpu_launches": int(launches),
+        "host_issue_ms_per_step": round(stage.issue_s / args.steps * 1e3, 3),
         "clocks": clocks,
         "frac_of_fp8_peak": {"of_measured_bf16_sustained_x2": round(value / world / (2 * peaks["bf16_sustained"]), 4),
                              "of_nominal_4500": round(value / world / 4500.0, 4)},
@@ -404,7 +413,7 @@ def main():
     torch.cuda.empty_cache()
 
     if not args.no_extras:
-        stage = Stage(qe, cfg_name, cfg, args.mode, device, host_io=True)
+        stage = Stage(qe, cfg_name, cfg, args.mode, device, host_io=True, same_stream=not args.own_stream)
         ms2, _ = time_steps(stage, max(2, args.steps // 2), 3, True, dist)
         n2 = max(2, args.steps // 2)
         line["e2e"] = {"value": round(step_flops(cfg) * n2 * world / (ms2 * 1e-3) / 1e12, 2), "unit": UNIT,

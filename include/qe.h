@@ -145,7 +145,11 @@ typedef struct qe_layer qe_layer;
 typedef struct qe_ctx_config {
   uint32_t exec_mode; /* qe_exec_mode: launch kernels one by one, or replay one prebuilt CUDA graph per (action, slot) */
   int32_t device;     /* CUDA device ordinal                                                                           */
-  uint32_t reserved[6];
+  void* exec_stream;  /* NULL: the context creates and owns its execution stream (actions then hand off to and from
+                         the caller's stream with events).  Non-NULL: a caller-owned cudaStream_t the context executes
+                         on; an action called with that same stream as caller_stream needs no event handoff, stream
+                         order gives both directions of the completion guarantee.                                     */
+  uint32_t reserved[4];
 } qe_ctx_config;
 
 typedef struct qe_layer_config {

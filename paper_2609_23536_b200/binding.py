@@ -61,7 +61,7 @@ class qe_contract_view(C.Structure):
 
 
 class qe_ctx_config(C.Structure):
-    _fields_ = [("exec_mode", C.c_uint32), ("device", C.c_int32), ("reserved", C.c_uint32 * 6)]
+    _fields_ = [("exec_mode", C.c_uint32), ("device", C.c_int32), ("exec_stream", C.c_void_p), ("reserved", C.c_uint32 * 4)]
 
 
 class qe_layer_config(C.Structure):
@@ -260,8 +260,9 @@ def contract_view_to_dict(v: qe_contract_view) -> dict:
 
 # ---------------------------------------------------------------------------------------- layer API
 class Context:
-    def __init__(self, exec_mode=EAGER, device=0):
-        cfg = qe_ctx_config(exec_mode=exec_mode, device=device)
+    def __init__(self, exec_mode=EAGER, device=0, exec_stream=None):
+        """exec_stream: a cudaStream_t (int) the context should execute on, or None for a context-owned stream."""
+        cfg = qe_ctx_config(exec_mode=exec_mode, device=device, exec_stream=exec_stream)
         self.h = _P()
         _check(lib.qe_ctx_create(C.byref(cfg), C.byref(self.h)))
         self.exec_mode = exec_mode

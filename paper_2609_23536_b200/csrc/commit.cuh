@@ -11,6 +11,13 @@
 
 namespace qe {
 
+// Programmatic dependent launch.  Every kernel of the library is launched with programmatic stream serialization, so
+// the next kernel in the stream may be scheduled while this one drains.  grid_dep_wait() returns once every kernel
+// this one depends on has completed and its writes are visible: it must precede the first access to anything a
+// predecessor produced.  grid_dep_launch() lets the successor's blocks start (they stop at their own wait).
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 template <class Sync>
 __device__ __forceinline__ void commit_classes(const CommitParams& p, int tid, uint32_t* red /* shared, 8 words */,
                                                Sync sync) {

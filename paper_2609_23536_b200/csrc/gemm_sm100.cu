@@ -268,6 +268,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   if (TWO) cluster_sync_all();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above (barriers, tensor memory) touched no global data and may overlap the previous kernel's tail;
+  // operands, scales and the destination may come from it, so wait for it here.
+  grid_dep_wait();
+  grid_dep_launch();
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer

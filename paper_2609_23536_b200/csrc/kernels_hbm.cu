@@ -63,7 +63,9 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_co
   const int rb = lane >> 3, cv = lane & 7;
   const uint32_t row0 = blockIdx.y * 256u + warp * 32u + rb * 8u;
   const uint32_t col0 = blockIdx.x * 64u + cv * 8u;
-  const float scale = __ldg(p.scale);
+  grid_dep_wait();  // the scale (and possibly x) come from earlier kernels
+  grid_dep_launch();
+  const float scale = *p.scale;
   if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && p.sinv_dst) *p.sinv_dst = *p.sinv_src;
 
   uint32_t m = 0;
@@ -129,6 +131,8 @@ Launch make_quantize(const QuantParams& p) {
 // The scale update as a kernel of its own (one block; latency-bound: at most 16 KB read).
 __global__ void __launch_bounds__(256) commit_kernel(const __grid_constant__ CommitParams p) {
   __shared__ uint32_t red[8];
+  grid_dep_wait();
+  grid_dep_launch();
   commit_classes(p, threadIdx.x, red, [] { __syncthreads(); });
 }
 
@@ -144,6 +148,8 @@ Launch make_commit(const CommitParams& p) {
 __global__ void __launch_bounds__(256) amax_pass1_kernel(const __grid_constant__ AmaxParams p) {
   __shared__ uint32_t wmax[8];
   uint32_t m = 0;
+  grid_dep_wait();
+  grid_dep_launch();
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
   uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   // four independent 16-byte loads in flight per thread
@@ -166,6 +172,8 @@ __global__ void __launch_bounds__(256) amax_pass1_kernel(const __grid_constant__
 __global__ void __launch_bounds__(256) amax_pass2_kernel(const __grid_constant__ AmaxParams p) {
   __shared__ uint32_t wmax[8];
   uint32_t m = 0;
+  grid_dep_wait();
+  grid_dep_launch();
   for (uint32_t i = threadIdx.x; i < p.nparts; i += blockDim.x) m = max(m, __float_as_uint(p.partials[i]));
   m = warp_max_u32(m);
   if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
@@ -194,6 +202,8 @@ Launch make_amax_pass2(const AmaxParams& p) {
 
 // ------------------------------------------------------------------------------------------------ copy-add
 __global__ void __launch_bounds__(256) accumulate_kernel(const __grid_constant__ AccumParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
   for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < p.nvec; i += stride) {
     float4 s = __ldcs(p.src + i);

@@ -89,6 +89,7 @@ struct qe_ctx {
   DeviceInfo* dev = nullptr;
   uint32_t exec_mode = QE_EXEC_EAGER;
   cudaStream_t exec_stream = nullptr;
+  bool owns_stream = true;
   cudaEvent_t ev_in = nullptr, ev_out = nullptr;
   qe_registry* registry = nullptr;
   qe_stats stats{};
@@ -103,7 +104,7 @@ static void ctx_release(qe_ctx* c) {
   cudaStreamSynchronize(c->exec_stream);
   cudaEventDestroy(c->ev_in);
   cudaEventDestroy(c->ev_out);
-  cudaStreamDestroy(c->exec_stream);
+  if (c->owns_stream) cudaStreamDestroy(c->exec_stream);
   qe_registry_destroy(c->registry);
   delete c;
 }
@@ -125,9 +126,25 @@ struct qe_layer {
 
 namespace {
 
-int32_t launch_eager(qe_ctx* ctx, const qe::Launch& l) {
+// One launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the stream
+// drains; every kernel of the library waits for its predecessors (griddepcontrol.wait) before touching their data.
+cudaError_t launch_pdl(const qe::Launch& l, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = l.grid;
+  cfg.blockDim = l.block;
+  cfg.dynamicSmemBytes = l.smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   void* args[1] = {const_cast<unsigned char*>(l.params)};
-  QE_CUDA(cudaLaunchKernel(l.func, l.grid, l.block, args, l.smem, ctx->exec_stream));
+  return cudaLaunchKernelExC(&cfg, l.func, args);
+}
+
+int32_t launch_eager(qe_ctx* ctx, const qe::Launch& l) {
+  QE_CUDA(launch_pdl(l, ctx->exec_stream));
   ctx->stats.eager_launches += 1;
   ctx->stats.kernels_launched += 1;
   return QE_OK;
@@ -140,8 +157,7 @@ int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& 
   QE_CUDA(cudaStreamBeginCapture(ctx->exec_stream, cudaStreamCaptureModeThreadLocal));
   cudaError_t err = cudaSuccess;
   for (const qe::Launch& l : ls) {
-    void* args[1] = {const_cast<unsigned char*>(l.params)};
-    err = cudaLaunchKernel(l.func, l.grid, l.block, args, l.smem, ctx->exec_stream);
+    err = launch_pdl(l, ctx->exec_stream);
     if (err != cudaSuccess) break;
   }
   cudaGraph_t graph = nullptr;
@@ -164,12 +180,14 @@ int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& 
   if (nroot != 1) return fail(QE_ERR_CUDA, "captured graph has %zu roots", nroot);
   while (cur) {
     chain.push_back(cur);
+    // the edges carry programmatic-dependency data, which only the _v2 query reports
     size_t nd = 0;
-    QE_CUDA(cudaGraphNodeGetDependentNodes(cur, nullptr, &nd));
+    QE_CUDA(cudaGraphNodeGetDependentNodes_v2(cur, nullptr, nullptr, &nd));
     if (nd == 0) break;
     if (nd != 1) return fail(QE_ERR_CUDA, "captured graph is not a chain");
     cudaGraphNode_t next = nullptr;
-    QE_CUDA(cudaGraphNodeGetDependentNodes(cur, &next, &nd));
+    cudaGraphEdgeData edge{};
+    QE_CUDA(cudaGraphNodeGetDependentNodes_v2(cur, &next, &edge, &nd));
     cur = next;
   }
   if (chain.size() != ls.size()) return fail(QE_ERR_CUDA, "chain of %zu nodes for %zu launches", chain.size(), ls.size());
@@ -335,7 +353,12 @@ int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
   if (!c) return fail(QE_ERR_BAD_ARG, "out of host memory");
   c->dev = d;
   c->exec_mode = cfg->exec_mode;
-  QE_CUDA(cudaStreamCreateWithFlags(&c->exec_stream, cudaStreamNonBlocking));
+  if (cfg->exec_stream) {
+    c->exec_stream = (cudaStream_t)cfg->exec_stream;
+    c->owns_stream = false;
+  } else {
+    QE_CUDA(cudaStreamCreateWithFlags(&c->exec_stream, cudaStreamNonBlocking));
+  }
   QE_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
   QE_CUDA(cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming));
   st = qe_registry_create(&c->registry);
@@ -673,8 +696,7 @@ static int32_t current_device_info(DeviceInfo** d) {
 }
 
 static int32_t launch_on(const qe::Launch& l, cudaStream_t s) {
-  void* args[1] = {const_cast<unsigned char*>(l.params)};
-  QE_CUDA(cudaLaunchKernel(l.func, l.grid, l.block, args, l.smem, s));
+  QE_CUDA(launch_pdl(l, s));
   return QE_OK;
 }
 
