@@ -159,9 +159,11 @@ class OracleLinear:
         return -1
 
     # ------------------------------------------------------------------ F
-    def forward(self, mb: int, gen: int, X_bits: np.ndarray, rows=None):
+    def forward(self, mb: int, gen: int, X_bits: np.ndarray, rows=None, light: bool = False):
         """Returns (tape, Y_bits).  With rows=[...] only those rows of Y are computed
-        (returned as [len(rows), N]) and the Y scaling class is not advanced."""
+        (returned as [len(rows), N]) and the Y scaling class is not advanced.
+        light=True (a test-speed switch, no arithmetic of its own): bookkeeping, amax and scale
+        updates only -- no FP8 bytes are produced, the tape cannot feed a GEMM, Y_bits is None."""
         if self.aborted:
             raise ContractError("ABORTED")
         if not (0 <= mb < 64):
@@ -184,18 +186,22 @@ class OracleLinear:
         # ---- physical action
         aW = None
         if refresh:
+            self._refresh_scale_W = np.float32(self.S["W"].scale)  # the scale this epoch's cache is cast with
             Wf = bf16.decode(self.W_bits)
             aW = amax_bf16(Wf)
-            self.Wq = fp8.quantize(Wf, self.S["W"].scale, fp8.E4M3)
+            self.Wq = None if light else fp8.quantize(Wf, self.S["W"].scale, fp8.E4M3)
             self.cache_sinv_W = np.float32(self.S["W"].scale_inv)
         Xf = bf16.decode(X_bits)
         aX = amax_bf16(Xf)
-        Xq = fp8.quantize(Xf, self.S["X"].scale, fp8.E4M3)
         sinv_X = np.float32(self.S["X"].scale_inv)
-        Y_bits = gemm_fwd(Xq, self.Wq, sinv_X, self.cache_sinv_W, rows)
-        aY = None
-        if rows is None:
-            aY = amax_bf16(bf16.decode(Y_bits))
+        Xq = Y_bits = aY = None
+        if not light:
+            if self.Wq is None:  # the epoch's refresh ran in light mode: produce the cache bytes now, same scale
+                self.Wq = fp8.quantize(bf16.decode(self.W_bits), self._refresh_scale_W, fp8.E4M3)
+            Xq = fp8.quantize(Xf, self.S["X"].scale, fp8.E4M3)
+            Y_bits = gemm_fwd(Xq, self.Wq, sinv_X, self.cache_sinv_W, rows)
+            if rows is None:
+                aY = amax_bf16(bf16.decode(Y_bits))
 
         # ---- commit
         s = self.slots[p]
@@ -213,7 +219,7 @@ class OracleLinear:
         return Tape(key, TapeRef(p, s.gen)), Y_bits
 
     # ------------------------------------------------------------------ dI
-    def backward_dI(self, tape: Tape, dY_bits: np.ndarray, rows=None) -> np.ndarray:
+    def backward_dI(self, tape: Tape, dY_bits: np.ndarray, rows=None, light: bool = False) -> np.ndarray:
         if self.aborted:
             raise ContractError("ABORTED")
         s = self._resolve(tape)
@@ -225,9 +231,11 @@ class OracleLinear:
 
         Gf = bf16.decode(dY_bits)
         aG = amax_bf16(Gf)
-        Gq = fp8.quantize(Gf, self.S["G"].scale, fp8.E5M2)
         sinv_G = np.float32(self.S["G"].scale_inv)
-        dX_bits = gemm_dI(Gq, self.Wq, sinv_G, self.cache_sinv_W, rows)
+        Gq = dX_bits = None
+        if not light:
+            Gq = fp8.quantize(Gf, self.S["G"].scale, fp8.E5M2)
+            dX_bits = gemm_dI(Gq, self.Wq, sinv_G, self.cache_sinv_W, rows)
 
         s.Gq, s.sinv_G = Gq, sinv_G
         s.bits |= DI_BIT
@@ -265,13 +273,14 @@ class OracleLinear:
         if self.write_mask == 0 and mb != 0:
             raise ContractError("ORDER", "microbatch 0 initialises the accumulation")
 
-        D = gemm_dW(s.Gq, s.Xq, s.sinv_G, s.sinv_X, rows)
-        view = buf[off : off + n].reshape(self.N, self.K)
-        sel = slice(None) if rows is None else np.asarray(rows)
-        if self.write_mask == 0:
-            view[sel] = D
-        else:
-            view[sel] = (view[sel] + D).astype(np.float32)  # fp32 + fp32 -> fp32, IEEE RN
+        if s.Xq is not None and s.Gq is not None:  # (a tape made in light mode carries no bytes: bookkeeping only)
+            D = gemm_dW(s.Gq, s.Xq, s.sinv_G, s.sinv_X, rows)
+            view = buf[off : off + n].reshape(self.N, self.K)
+            sel = slice(None) if rows is None else np.asarray(rows)
+            if self.write_mask == 0:
+                view[sel] = D
+            else:
+                view[sel] = (view[sel] + D).astype(np.float32)  # fp32 + fp32 -> fp32, IEEE RN
 
         self.bound_dest = (id(buf), off)
         self.write_mask |= 1 << mb
