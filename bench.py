@@ -97,13 +97,14 @@ class ClockSampler:
 class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
-    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True):
+    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
-                              exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None)
+                              exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
+                              overlap_dw=overlap_dw)
         self.schedule = sched(cfg["M"], *cfg["sched"])
         P = peak_live(self.schedule)
         T, M = cfg["T"], cfg["M"]
@@ -159,12 +160,12 @@ class Stage:
                     L.backward_dI(tapes[(m, i)], self.dY[m][i], self.dX[m][i])
                 else:
                     L.backward_dW(tapes[(m, i)], self.grad, self.offsets[i])
-        if host_io:
-            self.grad_host.copy_(self.grad, non_blocking=True)
-            self.d2h += self.grad.numel() * 4
         self.issue_s += time.perf_counter() - t_issue  # host time to enqueue the step (before the boundary's sync)
         for L in self.layers:
             L.optimizer_boundary(self.cfg["M"])
+        if host_io:  # the step's result: the accumulated gradients, complete after the boundary
+            self.grad_host.copy_(self.grad, non_blocking=True)
+            self.d2h += self.grad.numel() * 4
         self.epoch += 1
 
 
@@ -352,6 +353,7 @@ def main():
     ap.add_argument("--mode", default="graph", choices=["graph", "eager"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, roofline, HBM-kernel and CPU-baseline legs")
+    ap.add_argument("--overlap-dw", action="store_true", help="QE_CTX_OVERLAP_DW: dW actions on a second stream, joined at the optimizer boundary")
     ap.add_argument("--own-stream", action="store_true", help="let the context create its own execution stream (event handoff on every action)")
     args = ap.parse_args()
     cfg_name, cfg = args.config, inputs.CONFIGS[args.config]
@@ -381,7 +383,7 @@ def main():
     peaks = _peaks()
     args.warmup = max(args.warmup, 3)
 
-    stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream)
+    stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream, overlap_dw=args.overlap_dw)
     with ClockSampler(local) as clk:
         ms, launches = time_steps(stage, args.steps, args.warmup, False, dist)
     clocks = clk.summary()
@@ -396,7 +398,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw), "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),
@@ -413,7 +415,7 @@ def main():
     torch.cuda.empty_cache()
 
     if not args.no_extras:
-        stage = Stage(qe, cfg_name, cfg, args.mode, device, host_io=True, same_stream=not args.own_stream)
+        stage = Stage(qe, cfg_name, cfg, args.mode, device, host_io=True, same_stream=not args.own_stream, overlap_dw=args.overlap_dw)
         ms2, _ = time_steps(stage, max(2, args.steps // 2), 3, True, dist)
         n2 = max(2, args.steps // 2)
         line["e2e"] = {"value": round(step_flops(cfg) * n2 * world / (ms2 * 1e-3) / 1e12, 2), "unit": UNIT,

@@ -149,8 +149,17 @@ typedef struct qe_ctx_config {
                          the caller's stream with events).  Non-NULL: a caller-owned cudaStream_t the context executes
                          on; an action called with that same stream as caller_stream needs no event handoff, stream
                          order gives both directions of the completion guarantee.                                     */
-  uint32_t reserved[4];
+  uint32_t flags;     /* QE_CTX_* bits                                                                                 */
+  uint32_t reserved[3];
 } qe_ctx_config;
+/* Run the deferred weight-gradient actions on a second, lower-priority stream of the context so that their
+ * thread blocks fill SMs the forward / input-gradient kernels leave idle (dW never touches scaling state, which is
+ * what makes it deferrable: Eq. 5, Invariant 1).  Ordering kept by events: dW(m) after dI(m); a slot's next forward
+ * after the dW that released it; all dW of a layer in issue order on the one stream (so the accumulation order, and
+ * with it every bit of the gradient buffer, is the same as without the flag).  With this flag qe_backward_dW does
+ * NOT make the caller's stream wait for the dW: the gradient buffer is complete after qe_optimizer_boundary (which
+ * waits for both streams), matching the rule that the optimizer commit requires all arena writes resolved. */
+#define QE_CTX_OVERLAP_DW 1u
 
 typedef struct qe_layer_config {
   uint32_t T, K, N;       /* tokens, in-features, out-features: multiples of 128                             */

@@ -27,6 +27,7 @@ lib = C.CDLL(LIB_PATH)
 QE_MAX_SLOTS = 64
 QE_INVALID_EPOCH = (1 << 64) - 1
 EAGER, GRAPH = 0, 1
+OVERLAP_DW = 1
 CLASS_X, CLASS_W, CLASS_G, CLASS_Y = 0, 1, 2, 3
 CLASS_NAMES = ("X", "W", "G", "Y")
 E4M3, E5M2 = 0, 1
@@ -61,7 +62,7 @@ class qe_contract_view(C.Structure):
 
 
 class qe_ctx_config(C.Structure):
-    _fields_ = [("exec_mode", C.c_uint32), ("device", C.c_int32), ("exec_stream", C.c_void_p), ("reserved", C.c_uint32 * 4)]
+    _fields_ = [("exec_mode", C.c_uint32), ("device", C.c_int32), ("exec_stream", C.c_void_p), ("flags", C.c_uint32), ("reserved", C.c_uint32 * 3)]
 
 
 class qe_layer_config(C.Structure):
@@ -260,9 +261,10 @@ def contract_view_to_dict(v: qe_contract_view) -> dict:
 
 # ---------------------------------------------------------------------------------------- layer API
 class Context:
-    def __init__(self, exec_mode=EAGER, device=0, exec_stream=None):
-        """exec_stream: a cudaStream_t (int) the context should execute on, or None for a context-owned stream."""
-        cfg = qe_ctx_config(exec_mode=exec_mode, device=device, exec_stream=exec_stream)
+    def __init__(self, exec_mode=EAGER, device=0, exec_stream=None, overlap_dw=False):
+        """exec_stream: a cudaStream_t (int) the context should execute on, or None for a context-owned stream.
+        overlap_dw: QE_CTX_OVERLAP_DW (dW actions on a second stream, joined at the optimizer boundary)."""
+        cfg = qe_ctx_config(exec_mode=exec_mode, device=device, exec_stream=exec_stream, flags=OVERLAP_DW if overlap_dw else 0)
         self.h = _P()
         _check(lib.qe_ctx_create(C.byref(cfg), C.byref(self.h)))
         self.exec_mode = exec_mode

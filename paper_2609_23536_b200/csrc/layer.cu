@@ -90,6 +90,8 @@ struct qe_ctx {
   uint32_t exec_mode = QE_EXEC_EAGER;
   cudaStream_t exec_stream = nullptr;
   bool owns_stream = true;
+  cudaStream_t dw_stream = nullptr;  // only with QE_CTX_OVERLAP_DW
+  cudaEvent_t ev_dw_in = nullptr;
   cudaEvent_t ev_in = nullptr, ev_out = nullptr;
   qe_registry* registry = nullptr;
   qe_stats stats{};
@@ -102,6 +104,11 @@ struct qe_ctx {
 static void ctx_release(qe_ctx* c) {
   if (!c->closed || c->layers) return;
   cudaStreamSynchronize(c->exec_stream);
+  if (c->dw_stream) {
+    cudaStreamSynchronize(c->dw_stream);
+    cudaStreamDestroy(c->dw_stream);
+    cudaEventDestroy(c->ev_dw_in);
+  }
   cudaEventDestroy(c->ev_in);
   cudaEventDestroy(c->ev_out);
   if (c->owns_stream) cudaStreamDestroy(c->exec_stream);
@@ -122,6 +129,9 @@ struct qe_layer {
   CUtensorMap tmXq_A[QE_MAX_SLOTS], tmGq_A[QE_MAX_SLOTS], tmGqT_A[QE_MAX_SLOTS], tmXqT_B[QE_MAX_SLOTS];
   CUtensorMap tmWq_B, tmWqT_B;
   ActionGraph gF[QE_MAX_SLOTS], gDI[QE_MAX_SLOTS], gDW[QE_MAX_SLOTS], gDWs[QE_MAX_SLOTS], gRefresh, gCommit;
+  // QE_CTX_OVERLAP_DW: per slot, "dI of the tape in this slot has been enqueued" / "the dW that released it has"
+  cudaEvent_t ev_di[QE_MAX_SLOTS] = {}, ev_dw[QE_MAX_SLOTS] = {};
+  bool dw_pending[QE_MAX_SLOTS] = {};
 };
 
 namespace {
@@ -143,8 +153,8 @@ cudaError_t launch_pdl(const qe::Launch& l, cudaStream_t stream) {
   return cudaLaunchKernelExC(&cfg, l.func, args);
 }
 
-int32_t launch_eager(qe_ctx* ctx, const qe::Launch& l) {
-  QE_CUDA(launch_pdl(l, ctx->exec_stream));
+int32_t launch_eager(qe_ctx* ctx, const qe::Launch& l, cudaStream_t stream) {
+  QE_CUDA(launch_pdl(l, stream));
   ctx->stats.eager_launches += 1;
   ctx->stats.kernels_launched += 1;
   return QE_OK;
@@ -152,16 +162,16 @@ int32_t launch_eager(qe_ctx* ctx, const qe::Launch& l) {
 
 // Capture the launches on the execution stream into a graph, instantiate it, and recover the kernel nodes in
 // launch order by walking the (linear) dependency chain from the root.
-int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls) {
+int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls, cudaStream_t stream) {
   const auto t0 = std::chrono::steady_clock::now();
-  QE_CUDA(cudaStreamBeginCapture(ctx->exec_stream, cudaStreamCaptureModeThreadLocal));
+  QE_CUDA(cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
   cudaError_t err = cudaSuccess;
   for (const qe::Launch& l : ls) {
-    err = launch_pdl(l, ctx->exec_stream);
+    err = launch_pdl(l, stream);
     if (err != cudaSuccess) break;
   }
   cudaGraph_t graph = nullptr;
-  cudaError_t end = cudaStreamEndCapture(ctx->exec_stream, &graph);
+  cudaError_t end = cudaStreamEndCapture(stream, &graph);
   if (err != cudaSuccess) {
     if (graph) cudaGraphDestroy(graph);
     return fail(QE_ERR_CUDA, "launch during capture: %s", cudaGetErrorString(err));
@@ -203,7 +213,7 @@ int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& 
   return QE_OK;
 }
 
-int32_t replay_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls) {
+int32_t replay_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls, cudaStream_t stream) {
   if (ls.size() != g->launches.size()) return fail(QE_ERR_CUDA, "graph shape changed");
   for (size_t i = 0; i < ls.size(); ++i) {
     const qe::Launch& now = ls[i];
@@ -225,7 +235,7 @@ int32_t replay_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>&
     was = now;
     ctx->stats.node_param_updates += 1;
   }
-  QE_CUDA(cudaGraphLaunch(g->exec, ctx->exec_stream));
+  QE_CUDA(cudaGraphLaunch(g->exec, stream));
   ctx->stats.graph_replays += 1;
   ctx->stats.kernels_launched += ls.size();
   return QE_OK;
@@ -248,16 +258,17 @@ int32_t handoff_out(qe_ctx* ctx, cudaStream_t caller) {
   return QE_OK;
 }
 
-int32_t run_action(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls) {
+int32_t run_action(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& ls, cudaStream_t stream = nullptr) {
+  if (!stream) stream = ctx->exec_stream;
   if (ctx->exec_mode == QE_EXEC_GRAPH) {
     if (!g->built) {
-      int32_t st = build_graph(ctx, g, ls);
+      int32_t st = build_graph(ctx, g, ls, stream);
       if (st != QE_OK) return st;
     }
-    return replay_graph(ctx, g, ls);
+    return replay_graph(ctx, g, ls, stream);
   }
   for (const qe::Launch& l : ls) {
-    int32_t st = launch_eager(ctx, l);
+    int32_t st = launch_eager(ctx, l, stream);
     if (st != QE_OK) return st;
   }
   return QE_OK;
@@ -342,6 +353,7 @@ extern "C" {
 int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
   if (!cfg || !out) return fail(QE_ERR_BAD_ARG, "null argument");
   if (cfg->exec_mode > QE_EXEC_GRAPH) return fail(QE_ERR_BAD_ARG, "exec_mode %u", cfg->exec_mode);
+  if (cfg->flags & ~QE_CTX_OVERLAP_DW) return fail(QE_ERR_BAD_ARG, "unknown flags %#x", cfg->flags);
   int ndev = 0;
   cudaError_t e = cudaGetDeviceCount(&ndev);
   if (e != cudaSuccess || ndev == 0) return fail(QE_ERR_UNSUPPORTED, "no CUDA device: %s", cudaGetErrorString(e));
@@ -361,6 +373,12 @@ int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
   }
   QE_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
   QE_CUDA(cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming));
+  if (cfg->flags & QE_CTX_OVERLAP_DW) {
+    int least = 0, greatest = 0;
+    QE_CUDA(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+    QE_CUDA(cudaStreamCreateWithPriority(&c->dw_stream, cudaStreamNonBlocking, least));
+    QE_CUDA(cudaEventCreateWithFlags(&c->ev_dw_in, cudaEventDisableTiming));
+  }
   st = qe_registry_create(&c->registry);
   if (st != QE_OK) return st;
   *out = c;
@@ -431,6 +449,11 @@ int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint6
     delete L;
     return fail(QE_ERR_CUDA, "state initialisation: %s", cudaGetErrorString(e));
   }
+  if (ctx->dw_stream)
+    for (uint32_t p = 0; p < cfg->slots; ++p) {
+      cudaEventCreateWithFlags(&L->ev_di[p], cudaEventDisableTiming);
+      cudaEventCreateWithFlags(&L->ev_dw[p], cudaEventDisableTiming);
+    }
   ctx->stats.workspace_bytes += k.total;
   ctx->layers += 1;
   *out = L;
@@ -440,7 +463,10 @@ int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint6
 int32_t qe_layer_destroy(qe_layer* L) {
   if (!L) return QE_OK;
   cudaStreamSynchronize(L->ctx->exec_stream);
+  if (L->ctx->dw_stream) cudaStreamSynchronize(L->ctx->dw_stream);
   for (uint32_t p = 0; p < L->cfg.slots; ++p) {
+    if (L->ev_di[p]) cudaEventDestroy(L->ev_di[p]);
+    if (L->ev_dw[p]) cudaEventDestroy(L->ev_dw[p]);
     destroy_graph(&L->gF[p]);
     destroy_graph(&L->gDI[p]);
     destroy_graph(&L->gDW[p]);
@@ -469,6 +495,10 @@ int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* 
   cudaStream_t caller = (cudaStream_t)caller_stream;
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (L->dw_pending[p]) {  // the slot's buffers are still being read by the dW that released it (other stream)
+    QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[p], 0));
+    L->dw_pending[p] = false;
+  }
   if (refresh) {  // Invariant 3: first forward of the epoch re-quantises the weight and commits its amax
     std::vector<qe::Launch> ls;
     ls.push_back(quant_launch(L, L->cfg.weight_dev, L->Wq, L->WqT, N, K, QE_CLASS_W, &L->st->cache_sinv_W, QE_E4M3,
@@ -526,6 +556,7 @@ int32_t qe_backward_dI(qe_layer* L, const qe_tape* tape, const void* dy, void* d
   gp.commit = commit_params(L, 1u << QE_CLASS_G, 1, nullptr);  // backward amax/scale updated exactly once, here
   ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
   if ((st = run_action(ctx, &L->gDI[p], ls)) != QE_OK) return st;
+  if (ctx->dw_stream) QE_CUDA(cudaEventRecord(L->ev_di[p], ctx->exec_stream));
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
   return qe_contract_dI_commit(L->contract, tape);
 }
@@ -541,7 +572,17 @@ static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, u
   qe_ctx* ctx = L->ctx;
   cudaStream_t caller = (cudaStream_t)caller_stream;
   const uint32_t p = tape->ref.slot;
-  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  cudaStream_t run_on = ctx->exec_stream;
+  if (ctx->dw_stream) {
+    // overlapped dW: second stream, after the caller's work so far and after this tape's dI
+    run_on = ctx->dw_stream;
+    QE_CUDA(cudaEventRecord(ctx->ev_dw_in, caller));
+    QE_CUDA(cudaStreamWaitEvent(run_on, ctx->ev_dw_in, 0));
+    QE_CUDA(cudaStreamWaitEvent(run_on, L->ev_di[p], 0));
+    ctx->stats.handoffs += 1;
+  } else if ((st = handoff_in(ctx, caller)) != QE_OK) {
+    return st;
+  }
   qe::GemmParams gp{};
   gp.tmA = L->tmGqT_A[p];
   gp.tmB = L->tmXqT_B[p];
@@ -559,7 +600,7 @@ static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, u
     gp.out = grad + off;  // direct placement: the epilogue reads, adds and writes the destination itself
     gp.epi = acc ? 2 : 1;
     ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
-    st = run_action(ctx, &L->gDW[p], ls);
+    st = run_action(ctx, &L->gDW[p], ls, run_on);
   } else {
     gp.out = temp;
     gp.epi = 1;
@@ -570,10 +611,15 @@ static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, u
     ap.nvec = slice / 4;
     ap.accumulate = acc;
     ls.push_back(qe::make_accumulate(ap));
-    st = run_action(ctx, &L->gDWs[p], ls);
+    st = run_action(ctx, &L->gDWs[p], ls, run_on);
   }
   if (st != QE_OK) return st;
-  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  if (ctx->dw_stream) {  // joined at the optimizer boundary and before the slot's next forward
+    QE_CUDA(cudaEventRecord(L->ev_dw[p], run_on));
+    L->dw_pending[p] = true;
+  } else if ((st = handoff_out(ctx, caller)) != QE_OK) {
+    return st;
+  }
   return qe_contract_dW_commit(L->contract, tape, (uint64_t)(uintptr_t)grad, off, slice);
 }
 
@@ -589,6 +635,7 @@ int32_t qe_backward_dW_staged(qe_layer* L, const qe_tape* tape, float* grad, uin
 
 static int32_t read_status(qe_layer* L, uint32_t* status) {
   QE_CUDA(cudaStreamSynchronize(L->ctx->exec_stream));
+  if (L->ctx->dw_stream) QE_CUDA(cudaStreamSynchronize(L->ctx->dw_stream));
   QE_CUDA(cudaMemcpy(status, &L->st->status, sizeof(uint32_t), cudaMemcpyDeviceToHost));
   return QE_OK;
 }
@@ -638,6 +685,7 @@ int32_t qe_next_slot(const qe_layer* L, uint32_t* slot_out) {
 int32_t qe_get_state(qe_layer* L, qe_state_view* out, float* window_out, float* slot_sinv_out) {
   if (!L || !out) return fail(QE_ERR_BAD_ARG, "null argument");
   QE_CUDA(cudaStreamSynchronize(L->ctx->exec_stream));
+  if (L->ctx->dw_stream) QE_CUDA(cudaStreamSynchronize(L->ctx->dw_stream));
   qe::DevState h;
   QE_CUDA(cudaMemcpy(&h, L->st, sizeof(h), cudaMemcpyDeviceToHost));
   std::memset(out, 0, sizeof(*out));

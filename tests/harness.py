@@ -83,8 +83,8 @@ def run_gpu_steps(qe, layer, schedule, steps, M, grad_buf, off, get_inputs, weig
             if on_action:
                 on_action(step, a, m, layer, tapes[m])
         torch.cuda.synchronize()
+        layer.optimizer_boundary(M)  # with overlapped dW the gradient buffer is complete only after the boundary
         outs[(step, "mg")] = grad_buf.clone()
-        layer.optimizer_boundary(M)
     res = {}
     for k, v in outs.items():
         res[k] = v.cpu().numpy() if k[1] == "mg" else inputs.bits(v.cpu())

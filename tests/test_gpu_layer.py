@@ -31,8 +31,8 @@ def _weights(cfg, N, K, steps):
     return [inputs.bits(w) for w in ws]
 
 
-def _mk_layer(qe, mode, T, K, N, H, margin, P):
-    ctx = qe.Context(mode)
+def _mk_layer(qe, mode, T, K, N, H, margin, P, overlap=False):
+    ctx = qe.Context(mode, overlap_dw=overlap)
     w = torch.zeros((N, K), dtype=torch.bfloat16, device=DEV)
     return ctx, qe.Layer(ctx, T, K, N, H, margin, P, w)
 
@@ -112,11 +112,11 @@ def test_config1_every_action_against_oracle(qe, mode):
     assert st["kernels_launched"] == steps * (M * (2 + 2 + 1) + 1)  # quantise+GEMM, quantise+GEMM, GEMM; + weight refresh
 
 
-def _run_variant(qe, mode, schedule, staged=False, T=256, K=384, N=512, M=4, steps=2, H=4):
+def _run_variant(qe, mode, schedule, staged=False, T=256, K=384, N=512, M=4, steps=2, H=4, overlap=False):
     P = max(peak_live(schedule), 2)
     W = _weights("V", N, K, steps)
     get = lambda step, mb: c1_inputs(step, mb, T, K, N, "V")
-    ctx, L = _mk_layer(qe, mode, T, K, N, H, 1, P)
+    ctx, L = _mk_layer(qe, mode, T, K, N, H, 1, P, overlap)
     gbuf = torch.zeros(N * K, device=DEV)
     temp = torch.empty(N * K, device=DEV) if staged else None
     side = torch.cuda.Stream()
@@ -149,6 +149,15 @@ def test_graph_replay_equals_eager_bitwise(qe):
 def test_staged_copy_path_equals_direct_placement_bitwise(qe, mode):
     s = sched(4, 2, 1)
     _same(_run_variant(qe, mode, s), _run_variant(qe, mode, s, staged=True))
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("staged", [False, True])
+def test_overlapped_dW_stream_gives_the_same_bits(qe, mode, staged):
+    # dW on the context's second stream (joined at the optimizer boundary): same outputs, same state
+    s = sched(8, 3, 3)
+    kw = dict(M=8, T=512, K=512, N=768, steps=3)
+    _same(_run_variant(qe, mode, s, staged=staged, **kw), _run_variant(qe, mode, s, staged=staged, overlap=True, **kw))
 
 
 def test_scale_commit_standalone_matches_hand_worked_rollover(qe):
