@@ -56,10 +56,14 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
+            t0 = time.time()
+            while not self.rows and time.time() - t0 < 5.0:  # nvidia-smi takes a moment to deliver its first sample
+                time.sleep(0.01)
+            self.first = len(self.rows)
         except Exception:
             self.proc = None
         return self
@@ -79,7 +83,7 @@ class ClockSampler:
     def summary(self):
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[getattr(self, "first", 0):]:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
@@ -236,6 +240,27 @@ def gemm_roofline(qe, cfg, peaks, device):
         per[name][1] += ms
         del A, B, D
     assert status.item() == 0
+    lib = None
+    try:  # context only: the vendor library's FP8 GEMM (cuBLASLt through torch._scaled_mm) on the forward shapes
+        lf = lm = 0.0
+        for _, K, N in cfg["linears"]:
+            a = torch.randn((T, K), device=device).to(torch.float8_e4m3fn)
+            b = torch.randn((N, K), device=device).to(torch.float8_e4m3fn)
+            f = lambda: torch._scaled_mm(a, b.t(), scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+            for _ in range(3):
+                f()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(20):
+                f()
+            e1.record()
+            torch.cuda.synchronize()
+            lf += 2.0 * T * K * N
+            lm += e0.elapsed_time(e1) / 20
+        lib = round(lf / (lm * 1e-3) / 1e12, 1)
+    except Exception as e:  # noqa: BLE001
+        lib = "unavailable: " + str(e)[:80]
     achieved = tot_flops / (tot_ms * 1e-3) / 1e12
     peak = 2.0 * peaks["bf16_burst"]  # FP8 dense = 2 x the bf16 peak (nominal ratio), kernels timed alone -> burst figure
     return {
@@ -244,6 +269,7 @@ def gemm_roofline(qe, cfg, peaks, device):
         "frac_of_nominal_4500": round(achieved / 4500.0, 4),
         "per_action_tflops": {k: round(v[0] / (v[1] * 1e-3) / 1e12, 1) for k, v in per.items()},
         "gemm_ms_per_microbatch": round(tot_ms, 4),
+        "vendor_library_fp8_forward_tflops_same_shapes": lib,
     }
 
 

@@ -364,29 +364,40 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       uint32_t amax_bits = 0;
       // coalesced view of a 32 x 32 block: this lane owns columns 4*(lane%8)..+3 of rows it*4 + lane/8, it = 0..7
       const uint32_t blk_row0 = m0 + rank * BM + quad * 32u, sub_row = (uint32_t)lane >> 3, sub_col = ((uint32_t)lane & 7u) * 4u;
-#pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        const uint32_t col = col0 + ch * 32u;
-        if (col >= p.N) break;  // ragged last column tile (N a multiple of 128 but not of 256); warp-uniform
-        uint32_t r[32];
-        tmem_ld32(t_row + ch * 32u, r);
-        float4 old[8];
-        if (p.epi == 2) {
-          const float* src = reinterpret_cast<const float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
+      // Software pipeline over the warp's four 32 x 32 blocks: the tensor-memory load and (for the read-modify-
+      // write) the destination loads of block ch+1 are in flight while block ch is scaled, turned and written.
+      const uint32_t nch = col0 >= p.N ? 0u : min(4u, (p.N - col0) / 32u);  // ragged last column tile; warp-uniform
+      uint32_t r[2][32];
+      float4 old[2][8];
+      auto load_old = [&](int ch, float4(&o)[8]) {
+        const float* src = reinterpret_cast<const float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col0 + ch * 32u + sub_col;
 #pragma unroll
-          for (int it = 0; it < 8; ++it)  // in flight together with the tensor-memory load
-            old[it] = *reinterpret_cast<const float4*>(src + (size_t)(it * 4) * p.ldo);
-        }
+        for (int it = 0; it < 8; ++it) o[it] = *reinterpret_cast<const float4*>(src + (size_t)(it * 4) * p.ldo);
+      };
+      if (nch) {
+        tmem_ld32(t_row, r[0]);
+        if (p.epi == 2) load_old(0, old[0]);
+      }
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        if ((uint32_t)ch >= nch) break;
+        const uint32_t col = col0 + ch * 32u;
         tmem_ld_wait();
+        if ((uint32_t)ch + 1 < nch) {
+          tmem_ld32(t_row + (ch + 1) * 32u, r[(ch + 1) & 1]);
+          if (p.epi == 2) load_old(ch + 1, old[(ch + 1) & 1]);
+        }
+        const uint32_t(&rc)[32] = r[ch & 1];
+        const float4(&oc)[8] = old[ch & 1];
         // row-wise (lane = row) into the padded buffer
         float4* wr = reinterpret_cast<float4*>(epi_buf + (uint32_t)lane * EPI_ROW_WORDS);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           float4 v;
-          v.x = __fmul_rn(__uint_as_float(r[4 * j]), alpha);
-          v.y = __fmul_rn(__uint_as_float(r[4 * j + 1]), alpha);
-          v.z = __fmul_rn(__uint_as_float(r[4 * j + 2]), alpha);
-          v.w = __fmul_rn(__uint_as_float(r[4 * j + 3]), alpha);
+          v.x = __fmul_rn(__uint_as_float(rc[4 * j]), alpha);
+          v.y = __fmul_rn(__uint_as_float(rc[4 * j + 1]), alpha);
+          v.z = __fmul_rn(__uint_as_float(rc[4 * j + 2]), alpha);
+          v.w = __fmul_rn(__uint_as_float(rc[4 * j + 3]), alpha);
           wr[j] = v;
         }
         __syncwarp();
@@ -408,10 +419,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           for (int it = 0; it < 8; ++it) {
             float4 v = *reinterpret_cast<const float4*>(rd + it * 4 * EPI_ROW_WORDS);
             if (p.epi == 2) {
-              v.x = __fadd_rn(old[it].x, v.x);
-              v.y = __fadd_rn(old[it].y, v.y);
-              v.z = __fadd_rn(old[it].z, v.z);
-              v.w = __fadd_rn(old[it].w, v.w);
+              v.x = __fadd_rn(oc[it].x, v.x);
+              v.y = __fadd_rn(oc[it].y, v.y);
+              v.z = __fadd_rn(oc[it].z, v.z);
+              v.w = __fadd_rn(oc[it].w, v.w);
             }
             *reinterpret_cast<float4*>(dst + (size_t)(it * 4) * p.ldo) = v;
           }
