@@ -262,10 +262,15 @@ def gemm_roofline(qe, cfg, peaks, device):
     except Exception as e:  # noqa: BLE001
         lib = "unavailable: " + str(e)[:80]
     achieved = tot_flops / (tot_ms * 1e-3) / 1e12
+    # dram__bytes_read + dram__bytes_write per launch, averaged over the twelve GEMMs of a microbatch, from one ncu
+    # capture of `python -m paper_2609_23536_b200.profile_case gemm_microbatch --small` (config-2 shapes only)
+    traffic = 39.8e6 if (T, tuple(cfg["linears"])) == (2048, tuple(inputs.CONFIGS["C2"]["linears"])) else None
     peak = 2.0 * peaks["bf16_burst"]  # FP8 dense = 2 x the bf16 peak (nominal ratio), kernels timed alone -> burst figure
     return {
-        "bound": "tensor", "kernel": "gemm_fp8_kernel", "achieved": round(achieved, 1), "peak": round(peak, 1),
-        "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": None, "peak_source": peaks["source"] + " bf16 burst x2",
+        "bound": "tensor", "kernel": "gemm_fp8_pair_kernel", "achieved": round(achieved, 1), "peak": round(peak, 1),
+        "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": traffic,
+        "algorithmic_bytes_per_launch": round(sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if k == 0 else 8) for _, M_, N_, Kc, _, _, k in shapes) / len(shapes)),
+        "flop_per_launch": round(tot_flops / len(shapes)), "launches_timed": len(shapes), "peak_source": peaks["source"] + " bf16 burst x2",
         "frac_of_nominal_4500": round(achieved / 4500.0, 4),
         "per_action_tflops": {k: round(v[0] / (v[1] * 1e-3) / 1e12, 1) for k, v in per.items()},
         "gemm_ms_per_microbatch": round(tot_ms, 4),
@@ -379,7 +384,8 @@ def main():
     ap.add_argument("--mode", default="graph", choices=["graph", "eager"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, roofline, HBM-kernel and CPU-baseline legs")
-    ap.add_argument("--overlap-dw", action="store_true", help="QE_CTX_OVERLAP_DW: dW actions on a second stream, joined at the optimizer boundary")
+    ap.add_argument("--no-overlap-dw", dest="overlap_dw", action="store_false",
+                    help="run dW on the execution stream too (default: QE_CTX_OVERLAP_DW, dW on a second stream joined at the optimizer boundary)")
     ap.add_argument("--own-stream", action="store_true", help="let the context create its own execution stream (event handoff on every action)")
     args = ap.parse_args()
     cfg_name, cfg = args.config, inputs.CONFIGS[args.config]

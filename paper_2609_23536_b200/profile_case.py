@@ -1,6 +1,6 @@
 """Small single-kernel cases for profiling (ncu) and quick timing.
 
-    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|quantize|quantize_t|amax|accumulate [--reps N]
+    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|gemm_microbatch|quantize|quantize_t|amax|accumulate [--reps N]
 
 Each case holds well under 2 GB on the device, uses operands larger than the 126 MB L2 where DRAM traffic is
 the question, does 2 warm-up launches and then `reps` launches, and prints the CUDA-event time per launch.
@@ -29,7 +29,24 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     T, H, F = (2048, 2048, 11264) if a.small else (4096, 4096, 28672)
     work = None
-    if a.case.startswith("gemm"):
+    if a.case == "gemm_microbatch":
+        # the twelve GEMMs (F, dI, dW of four linears) one microbatch of the Llama-style block launches, in order
+        shapes = []
+        for K, N in ((H, 6144), (H, H), (H, F), (F // 2, H)):
+            shapes += [(T, N, K, 0, 0), (T, K, N, 1, 0), (N, K, T, 1, 2)]
+        ops = []
+        for M, N, Kc, af, kind in shapes:
+            ops.append((torch.randint(0, 120, (M, Kc), dtype=torch.uint8, device=dev),
+                        torch.randint(0, 120, (N, Kc), dtype=torch.uint8, device=dev),
+                        torch.zeros((M, N), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=dev), af, kind))
+
+        def fn():
+            for A, B, D, af, kind in ops:
+                qe.qe_gemm_fp8(A, af, B, 0, one, one, D, kind, None, status)
+
+        work = {"flop": sum(2.0 * M * N * Kc for M, N, Kc, _, _ in shapes),
+                "bytes": sum(M * Kc + N * Kc + M * N * (2 if k == 0 else 8) for M, N, Kc, _, k in shapes)}
+    elif a.case.startswith("gemm"):
         # gate/up projection: F: [T,H]x[F,H]^T ; dI: [T,F]x[H,F]^T ; dW: [F,T]x[H,T]^T (FP32 read-modify-write)
         M, N, Kc, af, kind = {"gemm_f": (T, F, H, 0, 0), "gemm_di": (T, H, F, 1, 0), "gemm_dw": (F, H, T, 1, 2)}[a.case]
         A = torch.randint(0, 120, (M, Kc), dtype=torch.uint8, device=dev)
