@@ -173,6 +173,22 @@ class Stage:
         self.epoch += 1
 
 
+def max_over_ranks(ms: float, dist, device="cuda") -> float:
+    """Slowest rank's time (every rank returns it); dist is torch.distributed or None for a single process."""
+    if dist is None:
+        return ms
+    import torch
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flop_per_step: float, steps: int, world: int, ms_max: float) -> float:
+    """Aggregate TFLOP/s of all replicas: every rank did `steps` steps within the slowest rank's time."""
+    return flop_per_step * steps * world / (ms_max * 1e-3) / 1e12
+
+
 def time_steps(stage, steps, warmup, host_io, dist):
     import torch
 
@@ -192,11 +208,9 @@ def time_steps(stage, steps, warmup, host_io, dist):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
+    ms = max_over_ranks(ms, dist)
     if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-        ms = float(t.item())
     return ms, stage.ctx.stats()["kernels_launched"] - k0
 
 
@@ -419,8 +433,7 @@ def main():
     with ClockSampler(local) as clk:
         ms, launches = time_steps(stage, args.steps, args.warmup, False, dist)
     clocks = clk.summary()
-    flops = step_flops(cfg) * args.steps * world
-    value = flops / (ms * 1e-3) / 1e12
+    value = whole_job_value(step_flops(cfg), args.steps, world, ms)
     stats = stage.ctx.stats()
     status = max(L.state()["device_status"] for L in stage.layers[:1])
     line = {
