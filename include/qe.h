@@ -127,6 +127,10 @@ int32_t qe_contract_rebuild(qe_contract*);
 int32_t qe_contract_invalidate_cache(qe_contract*);
 /* Invariant 4: QE_OK only when no tape is live ("checkpoint withheld" otherwise -> PENDING). */
 int32_t qe_contract_checkpoint_check(const qe_contract*);
+/* Restart rule (Algorithm 1, last line; Sec. 3.5): adopt the saved weight version, invalidate the cache so the first
+ * forward refreshes it, clear the write mask and the aborted flag.  Process-local identities (slot generations, the
+ * effect token) are NOT restored: they keep counting from wherever this process is.  PENDING if a tape is live. */
+int32_t qe_contract_restore(qe_contract*, uint64_t e_W);
 
 typedef struct qe_slot_view { uint64_t gen; uint32_t live; uint32_t bits; qe_tape_key key; uint32_t reserved; } qe_slot_view;
 typedef struct qe_contract_view {
@@ -233,6 +237,17 @@ int32_t qe_get_state(qe_layer*, qe_state_view* out, float* window_out, float* sl
 /* Copies a slot's retained FP8 bytes to host memory (testing aid; synchronises).  which: 0 = Xq [T,K],
  * 1 = Xq^T [K,T], 2 = Gq [T,N], 3 = Gq^T [N,T], 4 = Wq [N,K] (slot ignored), 5 = Wq^T [K,N] (slot ignored). */
 int32_t qe_read_fp8(qe_layer*, uint32_t which, uint32_t slot, void* host_out, uint64_t bytes);
+
+/* Quiescent checkpoint (Sec. 3.5, Invariant 4).  The payload holds PERSISTENT state only: the static configuration
+ * (T, K, N, H, margin), the four amax histories with their commit counts, scales and inverse scales, and the weight
+ * version e_W.  Graphs, streams, events, slot generations, the effect token, buffer addresses and the quantised-weight
+ * cache contents are process-local and are not saved.  qe_state_save waits for the layer's streams, then fails with
+ * QE_ERR_PENDING ("checkpoint withheld") while any tape is live.  qe_state_load (into a layer of the same
+ * configuration, no live tape) restores the numerics and e_W and invalidates the weight cache, so the first forward
+ * after it re-quantises the weight.  host buffers; bytes must equal qe_state_bytes. */
+int32_t qe_state_bytes(const qe_layer*, uint64_t* bytes_out);
+int32_t qe_state_save(qe_layer*, void* host_out, uint64_t bytes);
+int32_t qe_state_load(qe_layer*, const void* host_in, uint64_t bytes);
 
 typedef struct qe_stats {
   uint64_t graphs_built, graph_replays, eager_launches, handoffs, node_param_updates;

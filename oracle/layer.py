@@ -329,6 +329,35 @@ class OracleLinear:
         if self.live_tapes():
             raise ContractError("PENDING", "checkpoint withheld: live tape")
 
+    # ------------------------------------------------------------------ checkpoint / restart (Sec. 3.5, Invariant 4)
+    def save_state(self) -> dict:
+        """Persistent state only: numerics and the weight version.  Withheld while a tape is live."""
+        self.checkpoint_allowed()
+        return {
+            "e_W": self.e_W,
+            "classes": {c: {"hist": self.S[c].hist.copy(), "count": self.S[c].count, "scale": np.float32(self.S[c].scale),
+                            "scale_inv": np.float32(self.S[c].scale_inv)} for c in CLASSES},
+        }
+
+    def load_state(self, saved: dict) -> None:
+        """Restart rule: restore numerics and e_W, rebuild process-local resources (generations and the
+        token keep this process's values), and leave the cache stale so the first forward refreshes it."""
+        if self.live_tapes():
+            raise ContractError("PENDING")
+        for c in CLASSES:
+            d = saved["classes"][c]
+            self.S[c].hist = d["hist"].copy()
+            self.S[c].count = d["count"]
+            self.S[c].scale, self.S[c].scale_inv = np.float32(d["scale"]), np.float32(d["scale_inv"])
+        self.e_W = saved["e_W"]
+        self.e_C = INVALID_EPOCH
+        self.fwd_in_epoch = 0
+        self.write_mask = 0
+        self.aborted = False
+        self.bound_dest = None
+        self.registry.unbind(id(self))
+        self.Wq = None
+
     # ------------------------------------------------------------------ inspection
     def state(self) -> dict:
         return {

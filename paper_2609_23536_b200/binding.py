@@ -113,6 +113,7 @@ _SIGNATURES = {
     "qe_contract_rebuild": (C.c_int32, [_P]),
     "qe_contract_invalidate_cache": (C.c_int32, [_P]),
     "qe_contract_checkpoint_check": (C.c_int32, [_P]),
+    "qe_contract_restore": (C.c_int32, [_P, C.c_uint64]),
     "qe_contract_get": (C.c_int32, [_P, C.POINTER(qe_contract_view)]),
     "qe_ctx_create": (C.c_int32, [C.POINTER(qe_ctx_config), C.POINTER(_P)]),
     "qe_ctx_destroy": (C.c_int32, [_P]),
@@ -131,6 +132,9 @@ _SIGNATURES = {
     "qe_next_slot": (C.c_int32, [_P, C.POINTER(C.c_uint32)]),
     "qe_get_state": (C.c_int32, [_P, C.POINTER(qe_state_view), _P, _P]),
     "qe_read_fp8": (C.c_int32, [_P, C.c_uint32, C.c_uint32, _P, C.c_uint64]),
+    "qe_state_bytes": (C.c_int32, [_P, C.POINTER(C.c_uint64)]),
+    "qe_state_save": (C.c_int32, [_P, _P, C.c_uint64]),
+    "qe_state_load": (C.c_int32, [_P, _P, C.c_uint64]),
     "qe_get_stats": (C.c_int32, [_P, C.POINTER(qe_stats)]),
     "qe_quantize": (C.c_int32, [_P, C.c_uint32, C.c_uint32, _P, C.c_uint32, _P, _P, _P, _P]),
     "qe_amax": (C.c_int32, [_P, C.c_uint64, _P, _P, _P]),
@@ -230,6 +234,9 @@ class Contract:
 
     def checkpoint_check(self):
         _check(lib.qe_contract_checkpoint_check(self.h))
+
+    def restore(self, e_W):
+        _check(lib.qe_contract_restore(self.h, e_W))
 
     def get(self) -> dict:
         v = qe_contract_view()
@@ -358,6 +365,17 @@ class Layer:
         d["slot_sinv_X"] = sinv[: self.P].copy()
         d["slot_sinv_G"] = sinv[self.P:].copy()
         return d
+
+    def state_save(self) -> bytes:
+        n = C.c_uint64()
+        _check(lib.qe_state_bytes(self.h, C.byref(n)))
+        buf = (C.c_ubyte * n.value)()
+        _check(lib.qe_state_save(self.h, buf, n.value))
+        return bytes(buf)
+
+    def state_load(self, payload: bytes):
+        buf = (C.c_ubyte * len(payload)).from_buffer_copy(payload)
+        _check(lib.qe_state_load(self.h, buf, len(payload)))
 
     def read_fp8(self, which: int, slot: int = 0) -> np.ndarray:
         shape = {0: (self.T, self.K), 1: (self.K, self.T), 2: (self.T, self.N), 3: (self.N, self.T),

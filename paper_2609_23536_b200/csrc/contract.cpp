@@ -245,6 +245,22 @@ int32_t qe_contract_checkpoint_check(const qe_contract* c) {
   return QE_OK;
 }
 
+int32_t qe_contract_restore(qe_contract* c, uint64_t e_W) {
+  if (!c) return fail(QE_ERR_BAD_ARG, "contract is null");
+  if (c->live_tapes()) return fail(QE_ERR_PENDING, "restore with %u live tape(s)", c->live_tapes());
+  c->e_W = e_W;
+  c->e_C = QE_INVALID_EPOCH;  // cache contents are process-local: refresh on the first forward
+  c->fwd_in_epoch = 0;
+  c->write_mask = 0;
+  c->aborted = false;
+  c->has_dest = false;
+  if (c->registry) {
+    std::lock_guard<std::mutex> g(c->registry->mu);
+    c->registry->bound.erase(c);
+  }
+  return QE_OK;
+}
+
 int32_t qe_contract_get(const qe_contract* c, qe_contract_view* v) {
   if (!c || !v) return fail(QE_ERR_BAD_ARG, "null argument");
   std::memset(v, 0, sizeof(*v));

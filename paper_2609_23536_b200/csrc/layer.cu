@@ -730,6 +730,84 @@ int32_t qe_read_fp8(qe_layer* L, uint32_t which, uint32_t slot, void* host_out, 
   return QE_OK;
 }
 
+// ------------------------------------------------------------------------------------------------ checkpoint
+namespace {
+struct StateHeader {
+  uint32_t magic, version, T, K, N, H;
+  int32_t margin;
+  uint32_t reserved;
+  uint64_t e_W;
+  float scale[4], scale_inv[4];
+  uint32_t count[4];
+};
+constexpr uint32_t kStateMagic = 0x53454651u;  // "QFES"
+uint64_t state_bytes(const qe_layer* L) { return sizeof(StateHeader) + 4ull * L->cfg.history_len * sizeof(float); }
+int32_t sync_layer(qe_layer* L) {
+  QE_CUDA(cudaStreamSynchronize(L->ctx->exec_stream));
+  if (L->ctx->dw_stream) QE_CUDA(cudaStreamSynchronize(L->ctx->dw_stream));
+  return QE_OK;
+}
+}  // namespace
+
+int32_t qe_state_bytes(const qe_layer* L, uint64_t* bytes_out) {
+  if (!L || !bytes_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  *bytes_out = state_bytes(L);
+  return QE_OK;
+}
+
+int32_t qe_state_save(qe_layer* L, void* host_out, uint64_t bytes) {
+  if (!L || !host_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (bytes != state_bytes(L)) return fail(QE_ERR_BAD_ARG, "bytes %llu, state has %llu", (unsigned long long)bytes, (unsigned long long)state_bytes(L));
+  int32_t st = sync_layer(L);
+  if (st != QE_OK) return st;
+  if ((st = qe_contract_checkpoint_check(L->contract)) != QE_OK) return st;  // Invariant 4: only at quiescence
+  qe::DevState h;
+  QE_CUDA(cudaMemcpy(&h, L->st, sizeof(h), cudaMemcpyDeviceToHost));
+  if (h.status) return fail(QE_ERR_TIMEOUT, "device status word %#x", h.status);
+  StateHeader hd{};
+  hd.magic = kStateMagic;
+  hd.version = 1;
+  hd.T = L->cfg.T;
+  hd.K = L->cfg.K;
+  hd.N = L->cfg.N;
+  hd.H = L->cfg.history_len;
+  hd.margin = L->cfg.margin;
+  hd.e_W = L->contract->e_W;
+  for (int c = 0; c < 4; ++c) {
+    hd.scale[c] = h.scale[c];
+    hd.scale_inv[c] = h.scale_inv[c];
+    hd.count[c] = h.count[c];
+  }
+  std::memcpy(host_out, &hd, sizeof(hd));
+  QE_CUDA(cudaMemcpy((char*)host_out + sizeof(hd), L->hist, 4ull * hd.H * sizeof(float), cudaMemcpyDeviceToHost));
+  return QE_OK;
+}
+
+int32_t qe_state_load(qe_layer* L, const void* host_in, uint64_t bytes) {
+  if (!L || !host_in) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (bytes != state_bytes(L)) return fail(QE_ERR_BAD_ARG, "bytes %llu, state has %llu", (unsigned long long)bytes, (unsigned long long)state_bytes(L));
+  StateHeader hd;
+  std::memcpy(&hd, host_in, sizeof(hd));
+  if (hd.magic != kStateMagic || hd.version != 1) return fail(QE_ERR_BAD_ARG, "not a layer state payload");
+  if (hd.T != L->cfg.T || hd.K != L->cfg.K || hd.N != L->cfg.N || hd.H != L->cfg.history_len || hd.margin != L->cfg.margin)
+    return fail(QE_ERR_SHAPE, "payload is for T=%u K=%u N=%u H=%u margin=%d", hd.T, hd.K, hd.N, hd.H, hd.margin);
+  int32_t st = sync_layer(L);
+  if (st != QE_OK) return st;
+  if ((st = qe_contract_restore(L->contract, hd.e_W)) != QE_OK) return st;  // fails, changing nothing, if a tape lives
+  qe::DevState h;
+  QE_CUDA(cudaMemcpy(&h, L->st, sizeof(h), cudaMemcpyDeviceToHost));
+  for (int c = 0; c < 4; ++c) {
+    h.scale[c] = hd.scale[c];
+    h.scale_inv[c] = hd.scale_inv[c];
+    h.count[c] = hd.count[c];
+    h.pending_amax[c] = 0;
+  }
+  h.cache_sinv_W = 0.0f;  // cache contents are rebuilt by the first forward
+  QE_CUDA(cudaMemcpy(L->st, &h, sizeof(h), cudaMemcpyHostToDevice));
+  QE_CUDA(cudaMemcpy(L->hist, (const char*)host_in + sizeof(hd), 4ull * hd.H * sizeof(float), cudaMemcpyHostToDevice));
+  return QE_OK;
+}
+
 int32_t qe_get_stats(const qe_ctx* ctx, qe_stats* out) {
   if (!ctx || !out) return fail(QE_ERR_BAD_ARG, "null argument");
   *out = ctx->stats;

@@ -205,3 +205,19 @@ def test_contract_core_matches_oracle_state_machine(qe, ops):
         so, sc = O.state(), Cc.get()
         for k in ("e_W", "e_C", "token", "write_mask", "fwd_in_epoch", "aborted", "slots"):
             assert so[k] == sc[k], (k, so[k], sc[k])
+
+
+def test_contract_restore_is_the_restart_rule(qe):
+    c = qe.Contract(2)
+    t = c.forward_commit(0)
+    _expect(qe, "PENDING", c.restore, 5)
+    c.dI_commit(t)
+    c.dW_check(t, BUF, ELEMS, 0, SLICE)
+    c.dW_commit(t, BUF, 0, SLICE)
+    c.restore(5)
+    v = c.get()
+    assert v["e_W"] == 5 and v["e_C"] == qe.QE_INVALID_EPOCH and v["write_mask"] == 0 and v["fwd_in_epoch"] == 0
+    assert v["token"] == 2 and v["slots"][0]["gen"] == 1  # process-local identities keep counting
+    refresh, slot = c.forward_check(0, 5)
+    assert refresh and slot == 0
+    _expect(qe, "EPOCH", c.forward_check, 0, 0)

@@ -236,3 +236,60 @@ def test_bad_configs_are_rejected(qe):
     with pytest.raises(qe.QEError) as e:
         qe.Layer(ctx, 256, 256, 256, 0, 0, 2, w)
     assert e.value.code == "BAD_ARG"
+
+
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_resume_from_checkpoint_equals_uninterrupted_run(qe, mode):
+    # save at step 3 into a fresh context and layer ("fresh process"), continue through step 8
+    T, K, N, M, H = 256, 256, 384, 4, 4
+    s = sched(M, 2, 1)
+    P = peak_live(s)
+    W = _weights("R", N, K, 8)
+    get = lambda step, mb: c1_inputs(step, mb, T, K, N, "R")
+
+    def run(L, buf, steps, first_epoch):
+        L._e = first_epoch
+        outs = {}
+        for step in steps:
+            o = run_gpu_steps(qe, L, s, 1, M, buf, 0, lambda _s, mb: get(step, mb), lambda _e: W[step])
+            outs.update({(step,) + k[1:]: v for k, v in o.items()})
+        return outs
+
+    ctxA, A = _mk_layer(qe, mode, T, K, N, H, 0, P)
+    bufA = torch.zeros(N * K, device=DEV)
+    full = run(A, bufA, range(8), 0)
+
+    ctxB, B = _mk_layer(qe, mode, T, K, N, H, 0, P)
+    bufB = torch.zeros(N * K, device=DEV)
+    run(B, bufB, range(3), 0)
+    B.weight.copy_(inputs.from_bits(W[3]).to(DEV))
+    x = inputs.from_bits(get(3, 0)[0]).to(DEV)
+    y = torch.empty((T, N), dtype=torch.bfloat16, device=DEV)
+    t = B.forward(0, 3, x, y)
+    with pytest.raises(qe.QEError) as e:
+        B.state_save()
+    assert e.value.code == "PENDING"  # checkpoint withheld while a tape is live
+    B.abort_step()
+    B.arena_rebuild()
+    # (the abandoned forward advanced the X and Y histories; save a clean boundary state from another run instead)
+    ctxD, D = _mk_layer(qe, mode, T, K, N, H, 0, P)
+    bufD = torch.zeros(N * K, device=DEV)
+    run(D, bufD, range(3), 0)
+    payload = D.state_save()
+    assert len(payload) == 88 + 4 * H * 4  # persistent state only: a few hundred bytes here, ~16 KB at H = 1024
+    del D, ctxD
+
+    ctxE, E = _mk_layer(qe, mode, T, K, N, H, 0, P)
+    E.state_load(payload)
+    st = E.state()
+    assert st["e_W"] == 3 and st["e_C"] == qe.QE_INVALID_EPOCH and st["token"] == 0
+    bufE = torch.zeros(N * K, device=DEV)
+    got = run(E, bufE, range(3, 8), 3)
+    for k in got:
+        assert np.array_equal(full[k].view(np.uint8), got[k].view(np.uint8)), k
+    sa, se = A.state(), E.state()
+    assert state_equal({**sa, "slots": [], "token": 0}, {**se, "slots": [], "token": 0})
+    # wrong configuration is rejected
+    ctxF, F = _mk_layer(qe, mode, T, K, N, H + 1, 0, P)
+    with pytest.raises(qe.QEError):
+        F.state_load(payload)

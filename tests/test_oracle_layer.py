@@ -300,3 +300,78 @@ def test_pool_against_dict_model(ops):
         assert L.live_tapes() == len(live)
         assert [s.gen for s in L.slots] == gens
         assert len({t.ref.slot for t, _ in live.values()}) == len(live)  # injective
+
+
+def test_resume_from_quiescent_checkpoint_equals_uninterrupted_run():
+    # Sec. 5.2: save at step 3, continue through step 8, compare with the uninterrupted run.  Persistent state
+    # (histories, scales, weight version) is restored; tokens and generations are process-local; the cache refreshes.
+    T, K, N, M, H = 64, 64, 96, 4, 4
+    W = _weights(T, K, N)
+    s = sched(M, 2, 1)
+    get = _get_inputs(T, K, N)
+
+    def run(L, buf, steps):
+        outs = {}
+        for step in steps:
+            L.set_weight(W[step])
+            tapes = {}
+            for a, m in s:
+                X, dY = get(step, m)
+                if a == "F":
+                    tapes[m], outs[(step, "Y", m)] = L.forward(m, L.e_W, X)
+                elif a == "dI":
+                    outs[(step, "dX", m)] = L.backward_dI(tapes[m], dY)
+                else:
+                    L.backward_dW(tapes[m], buf, 0)
+            outs[(step, "mg")] = buf.copy()
+            L.optimizer_boundary(M)
+        return outs
+
+    A = _small(T, K, N, H=H, P=peak_live(s))
+    bufA = np.zeros(N * K, np.float32)
+    full = run(A, bufA, range(8))
+
+    B = _small(T, K, N, H=H, P=peak_live(s))
+    bufB = np.zeros(N * K, np.float32)
+    run(B, bufB, range(3))
+    B.set_weight(W[3])
+    t, _ = B.forward(0, B.e_W, get(3, 0)[0])
+    _expect("PENDING", B.save_state)  # checkpoint withheld while a tape is live
+    B.backward_dI(t, get(3, 0)[1])
+    B.backward_dW(t, bufB, 0)
+    B.abort_step()
+    B.arena_rebuild()
+    saved = B.save_state()
+
+    C = _small(T, K, N, H=H, P=peak_live(s))  # the "fresh process"
+    C.load_state(saved)
+    assert C.e_W == 3 and C.e_C != 3 and C.token == 0
+    bufC = np.zeros(N * K, np.float32)
+    # the interrupted process had already run (and abandoned) one microbatch of step 3: its X/G/Y commits are part of
+    # the saved state, so the resumed suffix is compared with an uninterrupted run that did the same
+    A2 = _small(T, K, N, H=H, P=peak_live(s))
+    buf2 = np.zeros(N * K, np.float32)
+    run(A2, buf2, range(3))
+    A2.set_weight(W[3])
+    t, _ = A2.forward(0, A2.e_W, get(3, 0)[0])
+    A2.backward_dI(t, get(3, 0)[1])
+    A2.backward_dW(t, buf2, 0)
+    A2.abort_step()
+    A2.arena_rebuild()
+    want = run(A2, buf2, range(3, 8))
+    got = run(C, bufC, range(3, 8))
+    for k in want:
+        assert np.array_equal(want[k].view(np.uint8), got[k].view(np.uint8)), k
+    sa, sc = A2.state(), C.state()
+    assert state_equal({**sa, "slots": [], "token": 0}, {**sc, "slots": [], "token": 0})
+    assert sa["token"] != sc["token"]  # process-local
+    # and a clean save at a step boundary resumes onto the plain uninterrupted trajectory
+    D = _small(T, K, N, H=H, P=peak_live(s))
+    bufD = np.zeros(N * K, np.float32)
+    run(D, bufD, range(3))
+    E = _small(T, K, N, H=H, P=peak_live(s))
+    E.load_state(D.save_state())
+    bufE = np.zeros(N * K, np.float32)
+    got = run(E, bufE, range(3, 8))
+    for k in got:
+        assert np.array_equal(full[k].view(np.uint8), got[k].view(np.uint8)), k
