@@ -358,37 +358,35 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) asm volatile("prefetch.global.L2 [%0];" ::"l"(d + 128 * j));
       }
-      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, ERR_EPILOGUE))) break;
-      tc_fence_after();
-      const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN + half * 128u;
-      uint32_t amax_bits = 0;
       // coalesced view of a 32 x 32 block: this lane owns columns 4*(lane%8)..+3 of rows it*4 + lane/8, it = 0..7
       const uint32_t blk_row0 = m0 + rank * BM + quad * 32u, sub_row = (uint32_t)lane >> 3, sub_col = ((uint32_t)lane & 7u) * 4u;
-      // Software pipeline over the warp's four 32 x 32 blocks: the tensor-memory load and (for the read-modify-
-      // write) the destination loads of block ch+1 are in flight while block ch is scaled, turned and written.
       const uint32_t nch = col0 >= p.N ? 0u : min(4u, (p.N - col0) / 32u);  // ragged last column tile; warp-uniform
       uint32_t r[2][32];
-      float4 old[2][8];
+      float4 old[2][8];  // destination values are fetched two blocks ahead (they do not depend on the accumulator)
       auto load_old = [&](int ch, float4(&o)[8]) {
         const float* src = reinterpret_cast<const float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col0 + ch * 32u + sub_col;
 #pragma unroll
         for (int it = 0; it < 8; ++it) o[it] = *reinterpret_cast<const float4*>(src + (size_t)(it * 4) * p.ldo);
       };
-      if (nch) {
-        tmem_ld32(t_row, r[0]);
-        if (p.epi == 2) load_old(0, old[0]);
+      if (p.epi == 2) {  // the first two blocks' destination values travel while the tile's MMAs still run
+        if (nch > 0) load_old(0, old[0]);
+        if (nch > 1) load_old(1, old[1]);
       }
+      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, ERR_EPILOGUE))) break;
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN + half * 128u;
+      uint32_t amax_bits = 0;
+      // Software pipeline over the warp's four 32 x 32 blocks: the tensor-memory load and (for the read-modify-
+      // write) the destination loads of block ch+1 are in flight while block ch is scaled, turned and written.
+      if (nch) tmem_ld32(t_row, r[0]);
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         if ((uint32_t)ch >= nch) break;
         const uint32_t col = col0 + ch * 32u;
         tmem_ld_wait();
-        if ((uint32_t)ch + 1 < nch) {
-          tmem_ld32(t_row + (ch + 1) * 32u, r[(ch + 1) & 1]);
-          if (p.epi == 2) load_old(ch + 1, old[(ch + 1) & 1]);
-        }
+        if ((uint32_t)ch + 1 < nch) tmem_ld32(t_row + (ch + 1) * 32u, r[(ch + 1) & 1]);
         const uint32_t(&rc)[32] = r[ch & 1];
-        const float4(&oc)[8] = old[ch & 1];
+        float4(&oc)[8] = old[ch & 1];
         // row-wise (lane = row) into the padded buffer
         float4* wr = reinterpret_cast<float4*>(epi_buf + (uint32_t)lane * EPI_ROW_WORDS);
 #pragma unroll
@@ -426,6 +424,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
             }
             *reinterpret_cast<float4*>(dst + (size_t)(it * 4) * p.ldo) = v;
           }
+          if (p.epi == 2 && (uint32_t)ch + 2 < nch) load_old(ch + 2, oc);  // this block's values are consumed: refill
         }
         __syncwarp();  // the buffer is rewritten by the next block
       }
