@@ -164,6 +164,12 @@ typedef struct qe_ctx_config {
  * NOT make the caller's stream wait for the dW: the gradient buffer is complete after qe_optimizer_boundary (which
  * waits for both streams), matching the rule that the optimizer commit requires all arena writes resolved. */
 #define QE_CTX_OVERLAP_DW 1u
+/* DIAGNOSTIC ONLY -- reproduces the defective one-way handoff of Sec. 2.3 so that it can be measured against the
+ * two-way protocol: the execution stream still waits for the caller, but the caller's stream is NOT made to wait for
+ * the action's tail.  A consumer on the caller's stream then reads outputs and state before the action has finished
+ * (stale data; no fault).  Never set this outside that experiment.  Ignored when the context executes on the
+ * caller's own stream. */
+#define QE_CTX_UNSAFE_ONE_WAY_HANDOFF 2u
 
 typedef struct qe_layer_config {
   uint32_t T, K, N;       /* tokens, in-features, out-features: multiples of 128                             */

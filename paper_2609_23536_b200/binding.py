@@ -28,6 +28,7 @@ QE_MAX_SLOTS = 64
 QE_INVALID_EPOCH = (1 << 64) - 1
 EAGER, GRAPH = 0, 1
 OVERLAP_DW = 1
+UNSAFE_ONE_WAY_HANDOFF = 2  # diagnostic: the one-way handoff of the paper's stale-read experiment
 CLASS_X, CLASS_W, CLASS_G, CLASS_Y = 0, 1, 2, 3
 CLASS_NAMES = ("X", "W", "G", "Y")
 E4M3, E5M2 = 0, 1
@@ -268,10 +269,10 @@ def contract_view_to_dict(v: qe_contract_view) -> dict:
 
 # ---------------------------------------------------------------------------------------- layer API
 class Context:
-    def __init__(self, exec_mode=EAGER, device=0, exec_stream=None, overlap_dw=False):
+    def __init__(self, exec_mode=EAGER, device=0, exec_stream=None, overlap_dw=False, unsafe_one_way=False):
         """exec_stream: a cudaStream_t (int) the context should execute on, or None for a context-owned stream.
         overlap_dw: QE_CTX_OVERLAP_DW (dW actions on a second stream, joined at the optimizer boundary)."""
-        cfg = qe_ctx_config(exec_mode=exec_mode, device=device, exec_stream=exec_stream, flags=OVERLAP_DW if overlap_dw else 0)
+        cfg = qe_ctx_config(exec_mode=exec_mode, device=device, exec_stream=exec_stream, flags=(OVERLAP_DW if overlap_dw else 0) | (UNSAFE_ONE_WAY_HANDOFF if unsafe_one_way else 0))
         self.h = _P()
         _check(lib.qe_ctx_create(C.byref(cfg), C.byref(self.h)))
         self.exec_mode = exec_mode

@@ -90,6 +90,7 @@ struct qe_ctx {
   uint32_t exec_mode = QE_EXEC_EAGER;
   cudaStream_t exec_stream = nullptr;
   bool owns_stream = true;
+  bool one_way = false;              // QE_CTX_UNSAFE_ONE_WAY_HANDOFF
   cudaStream_t dw_stream = nullptr;  // only with QE_CTX_OVERLAP_DW
   cudaEvent_t ev_dw_in = nullptr;
   cudaEvent_t ev_in = nullptr, ev_out = nullptr;
@@ -252,6 +253,7 @@ int32_t handoff_in(qe_ctx* ctx, cudaStream_t caller) {
 // ...and the caller's stream waits on the action's tail before it may consume anything.
 int32_t handoff_out(qe_ctx* ctx, cudaStream_t caller) {
   if (caller == ctx->exec_stream) return QE_OK;
+  if (ctx->one_way) return QE_OK;  // the defective protocol, kept for the stale-read experiment only
   QE_CUDA(cudaEventRecord(ctx->ev_out, ctx->exec_stream));
   QE_CUDA(cudaStreamWaitEvent(caller, ctx->ev_out, 0));
   ctx->stats.handoffs += 1;
@@ -353,7 +355,7 @@ extern "C" {
 int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
   if (!cfg || !out) return fail(QE_ERR_BAD_ARG, "null argument");
   if (cfg->exec_mode > QE_EXEC_GRAPH) return fail(QE_ERR_BAD_ARG, "exec_mode %u", cfg->exec_mode);
-  if (cfg->flags & ~QE_CTX_OVERLAP_DW) return fail(QE_ERR_BAD_ARG, "unknown flags %#x", cfg->flags);
+  if (cfg->flags & ~(QE_CTX_OVERLAP_DW | QE_CTX_UNSAFE_ONE_WAY_HANDOFF)) return fail(QE_ERR_BAD_ARG, "unknown flags %#x", cfg->flags);
   int ndev = 0;
   cudaError_t e = cudaGetDeviceCount(&ndev);
   if (e != cudaSuccess || ndev == 0) return fail(QE_ERR_UNSUPPORTED, "no CUDA device: %s", cudaGetErrorString(e));
@@ -373,6 +375,7 @@ int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
   }
   QE_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
   QE_CUDA(cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming));
+  c->one_way = (cfg->flags & QE_CTX_UNSAFE_ONE_WAY_HANDOFF) != 0;
   if (cfg->flags & QE_CTX_OVERLAP_DW) {
     int least = 0, greatest = 0;
     QE_CUDA(cudaDeviceGetStreamPriorityRange(&least, &greatest));

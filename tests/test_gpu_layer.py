@@ -293,3 +293,40 @@ def test_resume_from_checkpoint_equals_uninterrupted_run(qe, mode):
     ctxF, F = _mk_layer(qe, mode, T, K, N, H + 1, 0, P)
     with pytest.raises(qe.QEError):
         F.state_load(payload)
+
+
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_one_way_handoff_reads_stale_outputs_two_way_never_does(qe, mode):
+    # Sec. 2.3: fixed producer/consumer pairs, 200 checks per protocol.  The producer is a forward on the context's
+    # own stream; the consumer, on the caller's stream, copies Y right after the call returns.  With the one-way
+    # handoff the copy runs before the forward has finished and sees the sentinel the buffer held; with the two-way
+    # handshake it never does.  (A stale read is wrong data, not a fault.)
+    T, K, N = 2048, 4096, 4096
+    stale = {}
+    for one_way in (True, False):
+        ctx = qe.Context(mode, unsafe_one_way=one_way)
+        w = inputs.weights("H", 0, 0, N, K).to(DEV)
+        L = qe.Layer(ctx, T, K, N, 4, 0, 1, w)
+        x = inputs.activations("H", 0, 0, 0, 0, T, K).to(DEV)
+        dy = inputs.upstream_grads("H", 0, 0, 0, 0, T, N).to(DEV)
+        y = torch.empty((T, N), dtype=torch.bfloat16, device=DEV)
+        seen = torch.empty_like(y)
+        dx = torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+        buf = torch.zeros(N * K, device=DEV)
+        caller = torch.cuda.Stream()
+        n_stale = 0
+        with torch.cuda.stream(caller):
+            for i in range(200):
+                y.fill_(-7.0)  # sentinel, on the caller's stream (the forward waits for it: caller -> exec edge)
+                t = L.forward(0, i, x, y)
+                seen.copy_(y)  # the consumer
+                torch.cuda.synchronize()
+                n_stale += int((seen == -7.0).any().item())
+                assert not (y == -7.0).any().item()  # the producer itself always completes
+                L.backward_dI(t, dy, dx)
+                L.backward_dW(t, buf, 0)
+                torch.cuda.synchronize()
+                L.optimizer_boundary(1)
+        stale[one_way] = n_stale
+    assert stale[False] == 0
+    assert stale[True] >= 190, stale
