@@ -188,7 +188,10 @@ int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& 
   size_t nroot = 1;
   cudaGraphNode_t cur = nullptr;
   QE_CUDA(cudaGraphGetRootNodes(graph, &cur, &nroot));
-  if (nroot != 1) return fail(QE_ERR_CUDA, "captured graph has %zu roots", nroot);
+  if (nroot != 1) {
+    cudaGraphDestroy(graph);
+    return fail(QE_ERR_CUDA, "captured graph has %zu roots", nroot);
+  }
   while (cur) {
     chain.push_back(cur);
     // the edges carry programmatic-dependency data, which only the _v2 query reports
@@ -201,9 +204,16 @@ int32_t build_graph(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& 
     QE_CUDA(cudaGraphNodeGetDependentNodes_v2(cur, &next, &edge, &nd));
     cur = next;
   }
-  if (chain.size() != ls.size()) return fail(QE_ERR_CUDA, "chain of %zu nodes for %zu launches", chain.size(), ls.size());
+  if (chain.size() != ls.size()) {
+    cudaGraphDestroy(graph);
+    return fail(QE_ERR_CUDA, "chain of %zu nodes for %zu launches", chain.size(), ls.size());
+  }
   cudaGraphExec_t exec = nullptr;
-  QE_CUDA(cudaGraphInstantiate(&exec, graph, 0));
+  cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+  if (ie != cudaSuccess) {
+    cudaGraphDestroy(graph);
+    return fail(QE_ERR_CUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(ie));
+  }
   g->graph = graph;
   g->exec = exec;
   g->nodes = chain;
@@ -367,23 +377,32 @@ int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
   if (!c) return fail(QE_ERR_BAD_ARG, "out of host memory");
   c->dev = d;
   c->exec_mode = cfg->exec_mode;
+  c->one_way = (cfg->flags & QE_CTX_UNSAFE_ONE_WAY_HANDOFF) != 0;
+  e = cudaSuccess;
   if (cfg->exec_stream) {
     c->exec_stream = (cudaStream_t)cfg->exec_stream;
     c->owns_stream = false;
   } else {
-    QE_CUDA(cudaStreamCreateWithFlags(&c->exec_stream, cudaStreamNonBlocking));
+    e = cudaStreamCreateWithFlags(&c->exec_stream, cudaStreamNonBlocking);
   }
-  QE_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
-  QE_CUDA(cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming));
-  c->one_way = (cfg->flags & QE_CTX_UNSAFE_ONE_WAY_HANDOFF) != 0;
-  if (cfg->flags & QE_CTX_OVERLAP_DW) {
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming);
+  if (e == cudaSuccess && (cfg->flags & QE_CTX_OVERLAP_DW)) {
     int least = 0, greatest = 0;
-    QE_CUDA(cudaDeviceGetStreamPriorityRange(&least, &greatest));
-    QE_CUDA(cudaStreamCreateWithPriority(&c->dw_stream, cudaStreamNonBlocking, least));
-    QE_CUDA(cudaEventCreateWithFlags(&c->ev_dw_in, cudaEventDisableTiming));
+    e = cudaDeviceGetStreamPriorityRange(&least, &greatest);
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&c->dw_stream, cudaStreamNonBlocking, least);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_dw_in, cudaEventDisableTiming);
   }
-  st = qe_registry_create(&c->registry);
-  if (st != QE_OK) return st;
+  st = e == cudaSuccess ? qe_registry_create(&c->registry) : fail(QE_ERR_CUDA, "context resources: %s", cudaGetErrorString(e));
+  if (st != QE_OK) {  // release whatever was created
+    if (c->ev_in) cudaEventDestroy(c->ev_in);
+    if (c->ev_out) cudaEventDestroy(c->ev_out);
+    if (c->ev_dw_in) cudaEventDestroy(c->ev_dw_in);
+    if (c->dw_stream) cudaStreamDestroy(c->dw_stream);
+    if (c->owns_stream && c->exec_stream) cudaStreamDestroy(c->exec_stream);
+    delete c;
+    return st;
+  }
   *out = c;
   return QE_OK;
 }

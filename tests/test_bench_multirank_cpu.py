@@ -50,7 +50,7 @@ def test_reference_arm_runs_on_rank_zero_only():
     assert out.returncode == 0 and out.stdout.strip() == ""
 
 
-def test_step_flops_match_the_survey_figures():
+def test_step_flops_and_gradient_offsets_of_the_configurations():
     sys.path.insert(0, ROOT)
     import bench
     from paper_2609_23536_b200 import inputs
