@@ -160,6 +160,28 @@ def test_overlapped_dW_stream_gives_the_same_bits(qe, mode, staged):
     _same(_run_variant(qe, mode, s, staged=staged, **kw), _run_variant(qe, mode, s, staged=staged, overlap=True, **kw))
 
 
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_shapes_that_take_the_single_cta_gemm_against_oracle(qe, mode):
+    # T and N multiples of 128 but not of 256: F, dI and dW all run the 128 x 256-tile variant, with ragged last tiles
+    T, K, N, M, H = 384, 640, 896, 3, 4
+    s = sched(M, 2, 1)
+    P = peak_live(s)
+    W = _weights("S", N, K, 2)
+    get = lambda step, mb: c1_inputs(step, mb, T, K, N, "S")
+    O = OracleLinear(T, K, N, H, 0, P)
+    obuf = np.zeros(N * K, np.float32)
+    want = run_oracle_steps(O, s, 2, M, obuf, 0, get, lambda e: W[e])
+    ctx, L = _mk_layer(qe, mode, T, K, N, H, 0, P)
+    gbuf = torch.full((N * K,), -1.0, device=DEV)
+    got = run_gpu_steps(qe, L, s, 2, M, gbuf, 0, get, lambda e: W[e])
+    for k in want:
+        if k[1] == "mg":
+            assert assert_grad_close(got[k], want[k], k) < 1e-5
+        else:
+            assert_gemm_close(got[k], want[k], k)
+    assert state_equal_except_Y(L.state(), O.state())
+
+
 def test_scale_commit_standalone_matches_hand_worked_rollover(qe):
     ctx, L = _mk_layer(qe, 0, 256, 256, 256, 4, 0, 1)
     seq = [1, 8, 2, 2, 2, 2, 0.5, 0, 0, 0, 0, 3]
