@@ -119,26 +119,29 @@ class Stage:
         for l in range(cfg["layers"]):
             for j, (_, K, N) in enumerate(lin):
                 w = inputs.weights(cfg_name, l, j, N, K).to(device)
-                self.layers.append(qe.Layer(self.ctx, T, K, N, cfg["H"], cfg["margin"], P, w, stage=0, unit=l * len(lin) + j))
+                self.layers.append(qe.Layer(self.ctx, T, K, N, cfg["H"], cfg["margin"], P, w, stage=0, unit=l * len(lin) + j, host_io=host_io))
                 self.offsets.append(l * per_layer + offs[j])
         # distinct synthetic tensors per (microbatch, linear); drawn on the host once, outside any timed region
         g = torch.Generator(device="cpu")
         g.manual_seed(inputs.seed_for(cfg_name, "bench"))
-        self.X, self.dY, self.Y, self.dX, self.Xh, self.dYh = [], [], [], [], [], []
+        self.X, self.dY, self.Y, self.dX, self.Xh, self.dYh, self.Yh, self.dXh = [], [], [], [], [], [], [], []
         for m in range(M):
-            xs, gs, ys, dxs, xh, gh = [], [], [], [], [], []
+            xs, gs, ys, dxs, xh, gh, yh, dxh = [], [], [], [], [], [], [], []
             for L in self.layers:
                 x = torch.randn((T, L.K), generator=g, dtype=torch.float32).to(torch.bfloat16)
                 dy = (torch.randn((T, L.N), generator=g, dtype=torch.float32) * 1e-3).to(torch.bfloat16)
-                if host_io:
+                if host_io:  # the end-to-end leg keeps inputs and outputs in pinned host memory only
                     xh.append(x.pin_memory())
                     gh.append(dy.pin_memory())
-                xs.append(x.to(device))
-                gs.append(dy.to(device))
-                ys.append(torch.empty((T, L.N), dtype=torch.bfloat16, device=device))
-                dxs.append(torch.empty((T, L.K), dtype=torch.bfloat16, device=device))
+                    yh.append(torch.empty((T, L.N), dtype=torch.bfloat16).pin_memory())
+                    dxh.append(torch.empty((T, L.K), dtype=torch.bfloat16).pin_memory())
+                else:
+                    xs.append(x.to(device))
+                    gs.append(dy.to(device))
+                    ys.append(torch.empty((T, L.N), dtype=torch.bfloat16, device=device))
+                    dxs.append(torch.empty((T, L.K), dtype=torch.bfloat16, device=device))
             self.X.append(xs); self.dY.append(gs); self.Y.append(ys); self.dX.append(dxs)
-            self.Xh.append(xh); self.dYh.append(gh)
+            self.Xh.append(xh); self.dYh.append(gh); self.Yh.append(yh); self.dXh.append(dxh)
         self.grad_host = torch.empty(self.grad.shape, dtype=torch.float32).pin_memory() if host_io else None
         self.epoch = 0
         self.h2d = self.d2h = 0
@@ -153,15 +156,19 @@ class Stage:
             for i in order:
                 L = self.layers[i]
                 if a == "F":
-                    if host_io:
-                        self.X[m][i].copy_(self.Xh[m][i], non_blocking=True)
+                    if host_io:  # host pointers straight into the C-ABI: it stages, runs and reads back
+                        tapes[(m, i)] = L.forward_host(m, self.epoch, self.Xh[m][i], self.Yh[m][i])
                         self.h2d += self.Xh[m][i].numel() * 2
-                    tapes[(m, i)] = L.forward(m, self.epoch, self.X[m][i], self.Y[m][i])
+                        self.d2h += self.Yh[m][i].numel() * 2
+                    else:
+                        tapes[(m, i)] = L.forward(m, self.epoch, self.X[m][i], self.Y[m][i])
                 elif a == "dI":
                     if host_io:
-                        self.dY[m][i].copy_(self.dYh[m][i], non_blocking=True)
+                        L.backward_dI_host(tapes[(m, i)], self.dYh[m][i], self.dXh[m][i])
                         self.h2d += self.dYh[m][i].numel() * 2
-                    L.backward_dI(tapes[(m, i)], self.dY[m][i], self.dX[m][i])
+                        self.d2h += self.dXh[m][i].numel() * 2
+                    else:
+                        L.backward_dI(tapes[(m, i)], self.dY[m][i], self.dX[m][i])
                 else:
                     L.backward_dW(tapes[(m, i)], self.grad, self.offsets[i])
         self.issue_s += time.perf_counter() - t_issue  # host time to enqueue the step (before the boundary's sync)
@@ -466,7 +473,7 @@ def main():
         line["e2e"] = {"value": round(step_flops(cfg) * n2 * world / (ms2 * 1e-3) / 1e12, 2), "unit": UNIT,
                        "h2d_bytes_per_step": stage.h2d // n2, "d2h_bytes_per_step": stage.d2h // n2,
                        "ms_per_step": round(ms2 / n2, 3),
-                       "what": "X and dY of every microbatch copied from pinned host memory, gradient buffer read back, each step"}
+                       "what": "qe_forward_host / qe_backward_dI_host with pinned host X, dY, Y, dX for every microbatch; gradient buffer read back after each step"}
         del stage
         torch.cuda.empty_cache()
         if rank == 0:

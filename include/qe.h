@@ -177,7 +177,7 @@ typedef struct qe_layer_config {
   int32_t margin;         /* scale = fp8_max / max(history) / 2^margin; margin in [-32, 32]                  */
   uint32_t slots;         /* tape slots P in [1, QE_MAX_SLOTS]                                               */
   uint32_t stage, unit, inv; /* s, u, i of Eq. 1                                                             */
-  uint32_t reserved0;
+  uint32_t host_io;       /* 1: reserve staging buffers in the workspace for qe_forward_host / qe_backward_dI_host    */
   const void* weight_dev; /* bf16 W[N,K]; caller-owned; read on the first forward of every epoch             */
   uint64_t reserved1[4];
 } qe_layer_config;
@@ -202,6 +202,16 @@ int32_t qe_forward(qe_layer*, uint32_t mb, uint64_t gen, const void* x_dev, void
 /* dI (Eq. 4).  dy_dev bf16 [T,N] in, dx_dev bf16 [T,K] out.  Quantises dY to E5M2 (and its transpose, retained for
  * dW), dX = bf16((Gq Wq) * sinv_G * sinv_W), commits the gradient amax/scale once. */
 int32_t qe_backward_dI(qe_layer*, const qe_tape*, const void* dy_dev, void* dx_dev, void* caller_stream);
+/* F and dI with HOST buffers (layer created with host_io = 1).  The input is copied host-to-device into the layer's
+ * fixed staging buffer on the execution stream after the caller->execution edge (the dynamic-input copy of Sec. 4.4),
+ * the action runs on the staging buffers -- in graph mode the graph's addresses therefore never change -- and the output
+ * is copied device-to-host before the execution->caller edge, so it is complete for work the caller queues after the
+ * call (or after synchronising caller_stream on the host).  Pinned host memory makes the copies asynchronous; y_host /
+ * dx_host may be NULL to skip the read-back.  Same checks, state transitions and results as qe_forward /
+ * qe_backward_dI. */
+int32_t qe_forward_host(qe_layer*, uint32_t mb, uint64_t gen, const void* x_host, void* y_host, void* caller_stream,
+                        qe_tape* tape_out);
+int32_t qe_backward_dI_host(qe_layer*, const qe_tape*, const void* dy_host, void* dx_host, void* caller_stream);
 /* dW (Eq. 5) with direct gradient placement (Sec. 3.4).  D = (Gq^T Xq) * sinv_G * sinv_X using the inverse scales
  * snapshotted in the tape; grad_buf_dev[offset + n*K + k] = D (first write of the epoch) or += D (FP32, in place,
  * one owner thread per element: deterministic).  No staging copy, no scale-state change. */

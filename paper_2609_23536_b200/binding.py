@@ -69,7 +69,7 @@ class qe_ctx_config(C.Structure):
 class qe_layer_config(C.Structure):
     _fields_ = [
         ("T", C.c_uint32), ("K", C.c_uint32), ("N", C.c_uint32), ("history_len", C.c_uint32), ("margin", C.c_int32),
-        ("slots", C.c_uint32), ("stage", C.c_uint32), ("unit", C.c_uint32), ("inv", C.c_uint32), ("reserved0", C.c_uint32),
+        ("slots", C.c_uint32), ("stage", C.c_uint32), ("unit", C.c_uint32), ("inv", C.c_uint32), ("host_io", C.c_uint32),
         ("weight_dev", C.c_void_p), ("reserved1", C.c_uint64 * 4),
     ]
 
@@ -123,6 +123,8 @@ _SIGNATURES = {
     "qe_layer_destroy": (C.c_int32, [_P]),
     "qe_forward": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
     "qe_backward_dI": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
+    "qe_forward_host": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
+    "qe_backward_dI_host": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
     "qe_optimizer_boundary": (C.c_int32, [_P, C.c_uint32]),
@@ -294,14 +296,14 @@ class Context:
 class Layer:
     """One FP8 delayed-scaling linear.  Holds the torch-allocated workspace and the weight tensor alive."""
 
-    def __init__(self, ctx: Context, T, K, N, H, margin, slots, weight, stage=0, unit=0, inv=0):
+    def __init__(self, ctx: Context, T, K, N, H, margin, slots, weight, stage=0, unit=0, inv=0, host_io=False):
         import torch
 
         assert weight.dtype == torch.bfloat16 and weight.is_cuda and weight.is_contiguous() and tuple(weight.shape) == (N, K)
         self.ctx, self.T, self.K, self.N, self.H, self.P = ctx, T, K, N, H, slots
         self.weight = weight
         self.cfg = qe_layer_config(T=T, K=K, N=N, history_len=H, margin=margin, slots=slots, stage=stage, unit=unit,
-                                   inv=inv, weight_dev=weight.data_ptr())
+                                   inv=inv, host_io=int(host_io), weight_dev=weight.data_ptr())
         nbytes = C.c_uint64()
         _check(lib.qe_layer_workspace_bytes(C.byref(self.cfg), C.byref(nbytes)))
         self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=weight.device)
@@ -314,6 +316,15 @@ class Layer:
         t = qe_tape()
         _check(lib.qe_forward(self.h, mb, gen, _ptr(x), _ptr(y), _stream(stream), C.byref(t)))
         return t
+
+    def forward_host(self, mb, gen, x_host, y_host, stream=None) -> qe_tape:
+        """x_host / y_host: CPU tensors (pinned for asynchronous copies); y_host may be None."""
+        t = qe_tape()
+        _check(lib.qe_forward_host(self.h, mb, gen, _ptr(x_host), _ptr(y_host), _stream(stream), C.byref(t)))
+        return t
+
+    def backward_dI_host(self, tape, dy_host, dx_host, stream=None):
+        _check(lib.qe_backward_dI_host(self.h, C.byref(tape), _ptr(dy_host), _ptr(dx_host), _stream(stream)))
 
     def backward_dI(self, tape, dy, dx, stream=None):
         _check(lib.qe_backward_dI(self.h, C.byref(tape), _ptr(dy), _ptr(dx), _stream(stream)))

@@ -125,6 +125,7 @@ struct qe_layer {
   qe::DevState* st = nullptr;
   float* hist = nullptr;
   uint8_t *Wq = nullptr, *WqT = nullptr;
+  uint8_t *x_stage = nullptr, *dx_stage = nullptr, *y_stage = nullptr, *dy_stage = nullptr;  // host_io only
   uint8_t *Xq[QE_MAX_SLOTS], *XqT[QE_MAX_SLOTS], *Gq[QE_MAX_SLOTS], *GqT[QE_MAX_SLOTS];
   // tensor maps: A-role boxes are 128 rows, B-role boxes 256 rows
   CUtensorMap tmXq_A[QE_MAX_SLOTS], tmGq_A[QE_MAX_SLOTS], tmGqT_A[QE_MAX_SLOTS], tmXqT_B[QE_MAX_SLOTS];
@@ -295,7 +296,7 @@ void destroy_graph(ActionGraph* g) {
 }
 
 struct Carve {
-  uint64_t hist, Wq, WqT, slot0, per_slot, xq, xqT, gq, gqT, total;
+  uint64_t hist, Wq, WqT, slot0, per_slot, xq, xqT, gq, gqT, total, stage_tk = 0, stage_tn = 0;
 };
 Carve carve(const qe_layer_config& c) {
   Carve k{};
@@ -313,7 +314,14 @@ Carve carve(const qe_layer_config& c) {
   k.gq = k.xqT + align_up(tk, 1024);
   k.gqT = k.gq + align_up(tn, 1024);
   k.per_slot = k.gqT + align_up(tn, 1024);
-  k.total = o + k.per_slot * c.slots;
+  o += k.per_slot * c.slots;
+  if (c.host_io) {  // x / dx [T,K] and y / dy [T,N] bf16 staging for the host-buffer entry points
+    k.stage_tk = o;
+    o += 2 * align_up(2 * tk, 1024);
+    k.stage_tn = o;
+    o += 2 * align_up(2 * tn, 1024);
+  }
+  k.total = o;
   return k;
 }
 
@@ -324,6 +332,7 @@ int32_t check_config(const qe_layer_config* c) {
   if (c->history_len < 1 || c->history_len > QE_MAX_HISTORY) return fail(QE_ERR_BAD_ARG, "history_len %u", c->history_len);
   if (c->margin < -32 || c->margin > 32) return fail(QE_ERR_BAD_ARG, "margin %d", c->margin);
   if (c->slots < 1 || c->slots > QE_MAX_SLOTS) return fail(QE_ERR_BAD_ARG, "slots %u", c->slots);
+  if (c->host_io > 1) return fail(QE_ERR_BAD_ARG, "host_io %u", c->host_io);
   return QE_OK;
 }
 
@@ -444,6 +453,12 @@ int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint6
   L->hist = (float*)(base + k.hist);
   L->Wq = base + k.Wq;
   L->WqT = base + k.WqT;
+  if (cfg->host_io) {
+    L->x_stage = base + k.stage_tk;
+    L->dx_stage = L->x_stage + align_up(2ull * cfg->T * cfg->K, 1024);
+    L->y_stage = base + k.stage_tn;
+    L->dy_stage = L->y_stage + align_up(2ull * cfg->T * cfg->N, 1024);
+  }
   const DeviceInfo* d = ctx->dev;
   const uint32_t T = cfg->T, K = cfg->K, N = cfg->N;
   for (uint32_t p = 0; p < cfg->slots; ++p) {
@@ -505,10 +520,9 @@ int32_t qe_layer_destroy(qe_layer* L) {
   return QE_OK;
 }
 
-int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* y, void* caller_stream,
-                   qe_tape* tape_out) {
-  if (!L || !x || !y || !tape_out) return fail(QE_ERR_BAD_ARG, "null argument");
-  if (((uintptr_t)x | (uintptr_t)y) & 15u) return fail(QE_ERR_BAD_ARG, "x and y must be 16-byte aligned");
+// x_host / y_host: non-null for the host-buffer entry point (x and y are then the layer's staging buffers)
+static int32_t forward_impl(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* y, void* caller_stream,
+                            qe_tape* tape_out, const void* x_host, void* y_host) {
   int32_t refresh = 0;
   uint32_t p = 0;
   int32_t st = qe_contract_forward_check(L->contract, mb, gen, &refresh, &p);  // check ...
@@ -517,6 +531,8 @@ int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* 
   cudaStream_t caller = (cudaStream_t)caller_stream;
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (x_host)  // dynamic-input copy, after the caller -> execution edge
+    QE_CUDA(cudaMemcpyAsync(const_cast<void*>(x), x_host, 2ull * T * K, cudaMemcpyHostToDevice, ctx->exec_stream));
   if (L->dw_pending[p]) {  // the slot's buffers are still being read by the dW that released it (other stream)
     QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[p], 0));
     L->dw_pending[p] = false;
@@ -546,19 +562,35 @@ int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* 
   gp.commit = commit_params(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr);  // done by the GEMM's last CTA
   ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
   if ((st = run_action(ctx, &L->gF[p], ls)) != QE_OK) return st;  // ... run ...
+  if (y_host) QE_CUDA(cudaMemcpyAsync(y_host, y, 2ull * T * N, cudaMemcpyDeviceToHost, ctx->exec_stream));
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
   return qe_contract_forward_commit(L->contract, mb, tape_out);  // ... commit
 }
 
-int32_t qe_backward_dI(qe_layer* L, const qe_tape* tape, const void* dy, void* dx, void* caller_stream) {
-  if (!L || !tape || !dy || !dx) return fail(QE_ERR_BAD_ARG, "null argument");
-  if (((uintptr_t)dy | (uintptr_t)dx) & 15u) return fail(QE_ERR_BAD_ARG, "dy and dx must be 16-byte aligned");
+int32_t qe_forward(qe_layer* L, uint32_t mb, uint64_t gen, const void* x, void* y, void* caller_stream,
+                   qe_tape* tape_out) {
+  if (!L || !x || !y || !tape_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (((uintptr_t)x | (uintptr_t)y) & 15u) return fail(QE_ERR_BAD_ARG, "x and y must be 16-byte aligned");
+  return forward_impl(L, mb, gen, x, y, caller_stream, tape_out, nullptr, nullptr);
+}
+
+int32_t qe_forward_host(qe_layer* L, uint32_t mb, uint64_t gen, const void* x_host, void* y_host, void* caller_stream,
+                        qe_tape* tape_out) {
+  if (!L || !x_host || !tape_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (!L->x_stage) return fail(QE_ERR_BAD_ARG, "layer was created without host_io");
+  return forward_impl(L, mb, gen, L->x_stage, L->y_stage, caller_stream, tape_out, x_host, y_host);
+}
+
+static int32_t backward_dI_impl(qe_layer* L, const qe_tape* tape, const void* dy, void* dx, void* caller_stream,
+                                const void* dy_host, void* dx_host) {
   int32_t st = qe_contract_dI_check(L->contract, tape);
   if (st != QE_OK) return st;
   qe_ctx* ctx = L->ctx;
   cudaStream_t caller = (cudaStream_t)caller_stream;
   const uint32_t p = tape->ref.slot, T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (dy_host)
+    QE_CUDA(cudaMemcpyAsync(const_cast<void*>(dy), dy_host, 2ull * T * N, cudaMemcpyHostToDevice, ctx->exec_stream));
   std::vector<qe::Launch> ls;
   ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
   qe::GemmParams gp{};
@@ -579,8 +611,21 @@ int32_t qe_backward_dI(qe_layer* L, const qe_tape* tape, const void* dy, void* d
   ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
   if ((st = run_action(ctx, &L->gDI[p], ls)) != QE_OK) return st;
   if (ctx->dw_stream) QE_CUDA(cudaEventRecord(L->ev_di[p], ctx->exec_stream));
+  if (dx_host) QE_CUDA(cudaMemcpyAsync(dx_host, dx, 2ull * T * K, cudaMemcpyDeviceToHost, ctx->exec_stream));
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
   return qe_contract_dI_commit(L->contract, tape);
+}
+
+int32_t qe_backward_dI(qe_layer* L, const qe_tape* tape, const void* dy, void* dx, void* caller_stream) {
+  if (!L || !tape || !dy || !dx) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (((uintptr_t)dy | (uintptr_t)dx) & 15u) return fail(QE_ERR_BAD_ARG, "dy and dx must be 16-byte aligned");
+  return backward_dI_impl(L, tape, dy, dx, caller_stream, nullptr, nullptr);
+}
+
+int32_t qe_backward_dI_host(qe_layer* L, const qe_tape* tape, const void* dy_host, void* dx_host, void* caller_stream) {
+  if (!L || !tape || !dy_host) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (!L->dy_stage) return fail(QE_ERR_BAD_ARG, "layer was created without host_io");
+  return backward_dI_impl(L, tape, L->dy_stage, L->dx_stage, caller_stream, dy_host, dx_host);
 }
 
 static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, uint64_t elems, uint64_t off,

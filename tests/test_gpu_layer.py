@@ -352,3 +352,53 @@ def test_one_way_handoff_reads_stale_outputs_two_way_never_does(qe, mode):
         stale[one_way] = n_stale
     assert stale[False] == 0
     assert stale[True] >= 190, stale
+
+
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_host_buffer_entry_points_equal_the_device_ones_bitwise(qe, mode):
+    T, K, N, M = 256, 384, 512, 3
+    s = sched(M, 2, 1)
+    P = peak_live(s)
+    w = inputs.weights("HB", 0, 0, N, K).to(DEV)
+    res = []
+    for host in (False, True):
+        ctx = qe.Context(mode)
+        L = qe.Layer(ctx, T, K, N, 4, 0, P, w.clone(), host_io=host)
+        buf = torch.zeros(N * K, device=DEV)
+        outs, tapes = {}, {}
+        for a, m in s:
+            X, dY = c1_inputs(0, m, T, K, N, "HB")
+            if a == "F":
+                x = inputs.from_bits(X)
+                if host:
+                    y = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
+                    tapes[m] = L.forward_host(m, 0, x.pin_memory(), y)
+                else:
+                    y = torch.empty((T, N), dtype=torch.bfloat16, device=DEV)
+                    tapes[m] = L.forward(m, 0, x.to(DEV), y)
+                outs[("Y", m)] = y
+            elif a == "dI":
+                g = inputs.from_bits(dY)
+                if host:
+                    dx = torch.empty((T, K), dtype=torch.bfloat16).pin_memory()
+                    L.backward_dI_host(tapes[m], g.pin_memory(), dx)
+                else:
+                    dx = torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+                    L.backward_dI(tapes[m], g.to(DEV), dx)
+                outs[("dX", m)] = dx
+            else:
+                L.backward_dW(tapes[m], buf, 0)
+        torch.cuda.synchronize()
+        L.optimizer_boundary(M)
+        res.append(({k: inputs.bits(v.cpu()) for k, v in outs.items()}, buf.cpu().numpy(), L.state()))
+    (oa, ga, sa), (ob, gb, sb) = res
+    for k in oa:
+        assert np.array_equal(oa[k], ob[k]), k
+    assert np.array_equal(ga.view(np.uint32), gb.view(np.uint32))
+    assert state_equal(sa, sb)
+    # a layer created without staging refuses the host entry points
+    ctx = qe.Context(mode)
+    L = qe.Layer(ctx, T, K, N, 4, 0, P, w.clone())
+    with pytest.raises(qe.QEError) as e:
+        L.forward_host(0, 0, torch.zeros((T, K), dtype=torch.bfloat16), None)
+    assert e.value.code == "BAD_ARG"
