@@ -101,7 +101,7 @@ class ClockSampler:
 class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
-    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False):
+    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
@@ -116,6 +116,7 @@ class Stage:
         lin = cfg["linears"]
         offs, per_layer = inputs.grad_offsets(lin)
         self.grad = torch.zeros(per_layer * cfg["layers"], dtype=torch.float32, device=device)
+        self.temp = torch.empty(max(K * N for _, K, N in lin), dtype=torch.float32, device=device) if staged else None
         for l in range(cfg["layers"]):
             for j, (_, K, N) in enumerate(lin):
                 w = inputs.weights(cfg_name, l, j, N, K).to(device)
@@ -147,7 +148,22 @@ class Stage:
         self.h2d = self.d2h = 0
         self.issue_s = 0.0
 
+    def make_plan(self):
+        """The whole step as one qe_step_run call (native host loop; one graph for the step in graph mode)."""
+        n = len(self.layers)
+        acts = [(a, i, m) for a, m in self.schedule for i in (range(n) if a == "F" else range(n - 1, -1, -1))]
+        self.plan = self.qe.StepPlan(self.ctx, self.layers, acts, self.cfg["M"], self.X, self.Y, self.dY, self.dX,
+                                     self.grad, self.offsets, self.temp)
+
     def step(self, host_io=False):
+        if getattr(self, "plan", None) is not None and not host_io:
+            t_issue = time.perf_counter()
+            self.plan.run()
+            self.issue_s += time.perf_counter() - t_issue
+            for L in self.layers:
+                L.optimizer_boundary(self.cfg["M"])
+            self.epoch += 1
+            return
         tapes = {}
         n = len(self.layers)
         t_issue = time.perf_counter()
@@ -169,6 +185,8 @@ class Stage:
                         self.d2h += self.dXh[m][i].numel() * 2
                     else:
                         L.backward_dI(tapes[(m, i)], self.dY[m][i], self.dX[m][i])
+                elif self.temp is not None:
+                    L.backward_dW_staged(tapes[(m, i)], self.grad, self.offsets[i], self.temp)
                 else:
                     L.backward_dW(tapes[(m, i)], self.grad, self.offsets[i])
         self.issue_s += time.perf_counter() - t_issue  # host time to enqueue the step (before the boundary's sync)
@@ -407,6 +425,10 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, roofline, HBM-kernel and CPU-baseline legs")
     ap.add_argument("--no-overlap-dw", dest="overlap_dw", action="store_false",
                     help="run dW on the execution stream too (default: QE_CTX_OVERLAP_DW, dW on a second stream joined at the optimizer boundary)")
+    ap.add_argument("--step-api", action="store_true",
+                    help="qe_step_run: the whole step in one C call (native host loop; ONE graph per step in graph mode; dW not overlapped). "
+                         "Default: one C-ABI call per action with dW overlapped on the context's second stream")
+    ap.add_argument("--staged", action="store_true", help="copied-gradient comparison path: dW into a temporary, then a copy-add kernel")
     ap.add_argument("--own-stream", action="store_true", help="let the context create its own execution stream (event handoff on every action)")
     args = ap.parse_args()
     cfg_name, cfg = args.config, inputs.CONFIGS[args.config]
@@ -436,7 +458,11 @@ def main():
     peaks = _peaks()
     args.warmup = max(args.warmup, 3)
 
-    stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream, overlap_dw=args.overlap_dw)
+    use_step = args.step_api
+    stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
+                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged)
+    if use_step:
+        stage.make_plan()
     with ClockSampler(local) as clk:
         ms, launches = time_steps(stage, args.steps, args.warmup, False, dist)
     clocks = clk.summary()
@@ -450,7 +476,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw), "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "gradient_path": "staged copy-add" if args.staged else "direct placement", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),

@@ -234,6 +234,25 @@ int32_t qe_invalidate_cache(qe_layer*);
 /* Slot the next successful qe_forward will occupy (lowest free index), or QE_ERR_POOL_FULL. */
 int32_t qe_next_slot(const qe_layer*, uint32_t* slot_out);
 
+/* ---- A whole list of actions in one call (host loop in native code; in graph mode ONE graph for the whole list) ---
+ * Equivalent to calling qe_forward / qe_backward_dI / qe_backward_dW (or _staged when temp_dev is non-NULL) for
+ * actions[0..n) in order, each with gen = its layer's current weight version; the tapes are kept inside the call.
+ * All layers must belong to ctx.  io[layer * microbatches + mb] holds the device pointers of that unit (x, y for F;
+ * dy, dx for dI).  Layer l's gradient slice is grad_buf_dev + offsets[l].  Every action is checked and committed on
+ * the host exactly like the single calls; the kernels of the whole list are then issued behind ONE caller->execution
+ * wait and ONE execution->caller event: in eager mode as plain launches, in graph mode as one captured graph that is
+ * cached per (layers, actions) and replayed, with kernel-node parameters patched where pointers or the accumulate flag
+ * differ from the previous replay.  dW runs on the execution stream here (QE_CTX_OVERLAP_DW does not apply).
+ * If a check fails at action k, the kernels of actions 0..k-1 are still issued (device and host state stay in step),
+ * then every layer of the list is aborted as at a failure boundary (Sec. 4.5) and the failing check's status is
+ * returned; qe_arena_rebuild restarts the epoch. */
+typedef struct qe_step_action { uint32_t kind; uint32_t layer; uint32_t mb; uint32_t reserved; } qe_step_action;
+enum { QE_ACT_F = 0, QE_ACT_DI = 1, QE_ACT_DW = 2 };
+typedef struct qe_step_io { const void* x_dev; void* y_dev; const void* dy_dev; void* dx_dev; } qe_step_io;
+int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, const qe_step_action* actions,
+                    uint32_t n_actions, uint32_t microbatches, const qe_step_io* io, float* grad_buf_dev,
+                    uint64_t grad_buf_elems, const uint64_t* offsets, float* temp_dev, void* caller_stream);
+
 typedef struct qe_class_state {
   float scale, scale_inv;
   uint32_t count;      /* commits so far */

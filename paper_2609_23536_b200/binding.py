@@ -74,6 +74,14 @@ class qe_layer_config(C.Structure):
     ]
 
 
+class qe_step_action(C.Structure):
+    _fields_ = [("kind", C.c_uint32), ("layer", C.c_uint32), ("mb", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class qe_step_io(C.Structure):
+    _fields_ = [("x_dev", C.c_void_p), ("y_dev", C.c_void_p), ("dy_dev", C.c_void_p), ("dx_dev", C.c_void_p)]
+
+
 class qe_class_state(C.Structure):
     _fields_ = [("scale", C.c_float), ("scale_inv", C.c_float), ("count", C.c_uint32), ("reserved", C.c_uint32)]
 
@@ -127,6 +135,8 @@ _SIGNATURES = {
     "qe_backward_dI_host": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
+    "qe_step_run": (C.c_int32, [_P, C.POINTER(_P), C.c_uint32, C.POINTER(qe_step_action), C.c_uint32, C.c_uint32,
+                                C.POINTER(qe_step_io), _P, C.c_uint64, C.POINTER(C.c_uint64), _P, _P]),
     "qe_optimizer_boundary": (C.c_int32, [_P, C.c_uint32]),
     "qe_scale_commit": (C.c_int32, [_P, C.c_uint32, _P, _P]),
     "qe_abort_step": (C.c_int32, [_P]),
@@ -443,3 +453,29 @@ def qe_gemm_fp8_staged_noalloc(a, a_fmt, b, b_fmt, alpha_a_dev, alpha_b_dev, dst
 
 def qe_noalloc_staging_elems() -> int:
     return lib.qe_noalloc_staging_elems()
+
+
+ACT = {"F": 0, "dI": 1, "dW": 2}
+
+
+class StepPlan:
+    """Arguments of qe_step_run marshalled once: a list of (kind, layer index, microbatch) over `layers`, the device
+    tensors of every (layer, microbatch) unit, the flat gradient buffer with per-layer element offsets, and the
+    optional temporary of the copied-gradient path.  run() is one C call."""
+
+    def __init__(self, ctx: Context, layers, actions, microbatches, X, Y, dY, dX, grad_buf, offsets, temp=None):
+        self.ctx, self.layers, self.M = ctx, list(layers), microbatches
+        self.keep = (X, Y, dY, dX, grad_buf, temp)  # the tensors must outlive the plan
+        n = len(self.layers)
+        self.c_layers = (_P * n)(*[L.h for L in self.layers])
+        self.c_actions = (qe_step_action * len(actions))(*[qe_step_action(ACT[k], l, m, 0) for k, l, m in actions])
+        self.c_io = (qe_step_io * (n * microbatches))()
+        for l in range(n):
+            for m in range(microbatches):
+                self.c_io[l * microbatches + m] = qe_step_io(_ptr(X[m][l]), _ptr(Y[m][l]), _ptr(dY[m][l]), _ptr(dX[m][l]))
+        self.c_offsets = (C.c_uint64 * n)(*offsets)
+        self.grad, self.temp = grad_buf, temp
+
+    def run(self, stream=None):
+        _check(lib.qe_step_run(self.ctx.h, self.c_layers, len(self.layers), self.c_actions, len(self.c_actions), self.M,
+                               self.c_io, _ptr(self.grad), self.grad.numel(), self.c_offsets, _ptr(self.temp), _stream(stream)))

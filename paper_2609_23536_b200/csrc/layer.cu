@@ -2,6 +2,7 @@
 // (eager launches or one CUDA graph per (action, slot), both bracketed by the two-way stream handshake).
 #include <chrono>
 #include <cmath>
+#include <cstdio>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -100,11 +101,20 @@ struct qe_ctx {
   // so the two destroy calls may come in either order.
   uint32_t layers = 0;
   bool closed = false;
+  // whole-step graphs, one per distinct (layers, actions) list
+  struct StepGraph { uint64_t key; ActionGraph g; };
+  std::vector<StepGraph*> step_graphs;
 };
+
+static void destroy_graph(ActionGraph* g);
 
 static void ctx_release(qe_ctx* c) {
   if (!c->closed || c->layers) return;
   cudaStreamSynchronize(c->exec_stream);
+  for (auto* sg : c->step_graphs) {
+    destroy_graph(&sg->g);
+    delete sg;
+  }
   if (c->dw_stream) {
     cudaStreamSynchronize(c->dw_stream);
     cudaStreamDestroy(c->dw_stream);
@@ -287,13 +297,15 @@ int32_t run_action(qe_ctx* ctx, ActionGraph* g, const std::vector<qe::Launch>& l
   return QE_OK;
 }
 
-void destroy_graph(ActionGraph* g) {
+}  // namespace
+static void destroy_graph(ActionGraph* g) {
   if (g->exec) cudaGraphExecDestroy(g->exec);
   if (g->graph) cudaGraphDestroy(g->graph);
   g->exec = nullptr;
   g->graph = nullptr;
   g->built = false;
 }
+namespace {
 
 struct Carve {
   uint64_t hist, Wq, WqT, slot0, per_slot, xq, xqT, gq, gqT, total, stage_tk = 0, stage_tn = 0;
@@ -364,6 +376,88 @@ qe::Launch quant_launch(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uin
   qp.fmt = fmt;
   if (commit_mask) qp.commit = commit_params(L, commit_mask, 0, nullptr);
   return qe::make_quantize(qp);
+}
+
+
+// ---- the launches of each action (shared by the per-action calls and the whole-step call)
+void add_refresh(qe_layer* L, std::vector<qe::Launch>& ls) {
+  // Invariant 3: first forward of the epoch re-quantises the weight; the kernel's last block commits its amax
+  ls.push_back(quant_launch(L, L->cfg.weight_dev, L->Wq, L->WqT, L->cfg.N, L->cfg.K, QE_CLASS_W, &L->st->cache_sinv_W,
+                            QE_E4M3, 1u << QE_CLASS_W));
+}
+
+void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe::Launch>& ls) {
+  const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
+  ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
+  qe::GemmParams gp{};
+  gp.tmA = L->tmXq_A[p];
+  gp.tmB = L->tmWq_B;
+  gp.M = T;
+  gp.N = N;
+  gp.Kc = K;
+  gp.idesc = qe::gemm_idesc(QE_E4M3, QE_E4M3, T);
+  gp.alpha_a = &L->st->slot_sinv_X[p];
+  gp.alpha_b = &L->st->cache_sinv_W;
+  gp.out = y;
+  gp.ldo = N;
+  gp.epi = 0;
+  gp.amax_bits = &L->st->pending_amax[QE_CLASS_Y];
+  gp.status = &L->st->status;
+  gp.commit = commit_params(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr);  // done by the GEMM's last CTA
+  ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
+}
+
+void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::Launch>& ls) {
+  const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
+  ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
+  qe::GemmParams gp{};
+  gp.tmA = L->tmGq_A[p];
+  gp.tmB = L->tmWqT_B;
+  gp.M = T;
+  gp.N = K;
+  gp.Kc = N;
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, T);
+  gp.alpha_a = &L->st->slot_sinv_G[p];
+  gp.alpha_b = &L->st->cache_sinv_W;
+  gp.out = dx;
+  gp.ldo = K;
+  gp.epi = 0;
+  gp.amax_bits = nullptr;
+  gp.status = &L->st->status;
+  gp.commit = commit_params(L, 1u << QE_CLASS_G, 1, nullptr);  // backward amax/scale updated exactly once, here
+  ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
+}
+
+// dst = first element of the layer's gradient slice; temp != null selects the copied-gradient comparison path
+void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp, std::vector<qe::Launch>& ls) {
+  const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
+  qe::GemmParams gp{};
+  gp.tmA = L->tmGqT_A[p];
+  gp.tmB = L->tmXqT_B[p];
+  gp.M = N;
+  gp.N = K;
+  gp.Kc = T;
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, N);
+  gp.alpha_a = &L->st->slot_sinv_G[p];  // snapshots taken when dY_m and X_m were quantised, never the current state
+  gp.alpha_b = &L->st->slot_sinv_X[p];
+  gp.ldo = K;
+  gp.amax_bits = nullptr;
+  gp.status = &L->st->status;
+  if (!temp) {
+    gp.out = dst;  // direct placement: the epilogue reads, adds and writes the destination itself
+    gp.epi = accumulate ? 2 : 1;
+    ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
+  } else {
+    gp.out = temp;
+    gp.epi = 1;
+    ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
+    qe::AccumParams ap{};
+    ap.dst = (float4*)dst;
+    ap.src = (const float4*)temp;
+    ap.nvec = (uint64_t)N * K / 4;
+    ap.accumulate = accumulate;
+    ls.push_back(qe::make_accumulate(ap));
+  }
 }
 
 }  // namespace
@@ -537,30 +631,13 @@ static int32_t forward_impl(qe_layer* L, uint32_t mb, uint64_t gen, const void* 
     QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[p], 0));
     L->dw_pending[p] = false;
   }
-  if (refresh) {  // Invariant 3: first forward of the epoch re-quantises the weight and commits its amax
-    std::vector<qe::Launch> ls;
-    ls.push_back(quant_launch(L, L->cfg.weight_dev, L->Wq, L->WqT, N, K, QE_CLASS_W, &L->st->cache_sinv_W, QE_E4M3,
-                              1u << QE_CLASS_W));
-    if ((st = run_action(ctx, &L->gRefresh, ls)) != QE_OK) return st;
+  if (refresh) {
+    std::vector<qe::Launch> rs;
+    add_refresh(L, rs);
+    if ((st = run_action(ctx, &L->gRefresh, rs)) != QE_OK) return st;
   }
   std::vector<qe::Launch> ls;
-  ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
-  qe::GemmParams gp{};
-  gp.tmA = L->tmXq_A[p];
-  gp.tmB = L->tmWq_B;
-  gp.M = T;
-  gp.N = N;
-  gp.Kc = K;
-  gp.idesc = qe::gemm_idesc(QE_E4M3, QE_E4M3, T);
-  gp.alpha_a = &L->st->slot_sinv_X[p];
-  gp.alpha_b = &L->st->cache_sinv_W;
-  gp.out = y;
-  gp.ldo = N;
-  gp.epi = 0;
-  gp.amax_bits = &L->st->pending_amax[QE_CLASS_Y];
-  gp.status = &L->st->status;
-  gp.commit = commit_params(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr);  // done by the GEMM's last CTA
-  ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
+  add_forward(L, p, x, y, ls);
   if ((st = run_action(ctx, &L->gF[p], ls)) != QE_OK) return st;  // ... run ...
   if (y_host) QE_CUDA(cudaMemcpyAsync(y_host, y, 2ull * T * N, cudaMemcpyDeviceToHost, ctx->exec_stream));
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
@@ -592,23 +669,7 @@ static int32_t backward_dI_impl(qe_layer* L, const qe_tape* tape, const void* dy
   if (dy_host)
     QE_CUDA(cudaMemcpyAsync(const_cast<void*>(dy), dy_host, 2ull * T * N, cudaMemcpyHostToDevice, ctx->exec_stream));
   std::vector<qe::Launch> ls;
-  ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
-  qe::GemmParams gp{};
-  gp.tmA = L->tmGq_A[p];
-  gp.tmB = L->tmWqT_B;
-  gp.M = T;
-  gp.N = K;
-  gp.Kc = N;
-  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, T);
-  gp.alpha_a = &L->st->slot_sinv_G[p];
-  gp.alpha_b = &L->st->cache_sinv_W;
-  gp.out = dx;
-  gp.ldo = K;
-  gp.epi = 0;
-  gp.amax_bits = nullptr;
-  gp.status = &L->st->status;
-  gp.commit = commit_params(L, 1u << QE_CLASS_G, 1, nullptr);  // backward amax/scale updated exactly once, here
-  ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
+  add_dI(L, p, dy, dx, ls);
   if ((st = run_action(ctx, &L->gDI[p], ls)) != QE_OK) return st;
   if (ctx->dw_stream) QE_CUDA(cudaEventRecord(L->ev_di[p], ctx->exec_stream));
   if (dx_host) QE_CUDA(cudaMemcpyAsync(dx_host, dx, 2ull * T * K, cudaMemcpyDeviceToHost, ctx->exec_stream));
@@ -631,7 +692,7 @@ int32_t qe_backward_dI_host(qe_layer* L, const qe_tape* tape, const void* dy_hos
 static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, uint64_t elems, uint64_t off,
                                 float* temp, void* caller_stream) {
   if (!L || !tape) return fail(QE_ERR_BAD_ARG, "null argument");
-  const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
+  const uint32_t K = L->cfg.K, N = L->cfg.N;
   const uint64_t slice = (uint64_t)N * K;
   int32_t acc = 0;
   int32_t st = qe_contract_dW_check(L->contract, tape, (uint64_t)(uintptr_t)grad, elems, off, slice, &acc);
@@ -650,36 +711,9 @@ static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, u
   } else if ((st = handoff_in(ctx, caller)) != QE_OK) {
     return st;
   }
-  qe::GemmParams gp{};
-  gp.tmA = L->tmGqT_A[p];
-  gp.tmB = L->tmXqT_B[p];
-  gp.M = N;
-  gp.N = K;
-  gp.Kc = T;
-  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, N);
-  gp.alpha_a = &L->st->slot_sinv_G[p];  // snapshots taken when dY_m and X_m were quantised, never the current state
-  gp.alpha_b = &L->st->slot_sinv_X[p];
-  gp.ldo = K;
-  gp.amax_bits = nullptr;
-  gp.status = &L->st->status;
   std::vector<qe::Launch> ls;
-  if (!temp) {
-    gp.out = grad + off;  // direct placement: the epilogue reads, adds and writes the destination itself
-    gp.epi = acc ? 2 : 1;
-    ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
-    st = run_action(ctx, &L->gDW[p], ls, run_on);
-  } else {
-    gp.out = temp;
-    gp.epi = 1;
-    ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
-    qe::AccumParams ap{};
-    ap.dst = (float4*)(grad + off);
-    ap.src = (const float4*)temp;
-    ap.nvec = slice / 4;
-    ap.accumulate = acc;
-    ls.push_back(qe::make_accumulate(ap));
-    st = run_action(ctx, &L->gDWs[p], ls, run_on);
-  }
+  add_dW(L, p, grad + off, acc, temp, ls);
+  st = run_action(ctx, temp ? &L->gDWs[p] : &L->gDW[p], ls, run_on);
   if (st != QE_OK) return st;
   if (ctx->dw_stream) {  // joined at the optimizer boundary and before the slot's next forward
     QE_CUDA(cudaEventRecord(L->ev_dw[p], run_on));
@@ -698,6 +732,109 @@ int32_t qe_backward_dW_staged(qe_layer* L, const qe_tape* tape, float* grad, uin
                               float* temp, void* stream) {
   if (!temp || ((uintptr_t)temp & 15u)) return fail(QE_ERR_BAD_ARG, "temp_dev must be non-null and 16-byte aligned");
   return backward_dW_impl(L, tape, grad, elems, off, temp, stream);
+}
+
+// ------------------------------------------------------------------------------------------------ whole-step call
+int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, const qe_step_action* actions,
+                    uint32_t n_actions, uint32_t M, const qe_step_io* io, float* grad, uint64_t grad_elems,
+                    const uint64_t* offsets, float* temp, void* caller_stream) {
+  if (!ctx || !layers || !actions || !io || !offsets) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (n_layers == 0 || n_actions == 0 || M == 0 || M > QE_MAX_MICROBATCHES) return fail(QE_ERR_BAD_ARG, "empty list or bad microbatch count");
+  if (temp && ((uintptr_t)temp & 15u)) return fail(QE_ERR_BAD_ARG, "temp_dev must be 16-byte aligned");
+  for (uint32_t l = 0; l < n_layers; ++l)
+    if (!layers[l] || layers[l]->ctx != ctx) return fail(QE_ERR_BAD_ARG, "layer %u is null or belongs to another context", l);
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+
+  // ---- host pass: check -> collect launches -> commit, action by action (Algorithm 1)
+  std::vector<qe_tape> tapes((size_t)n_layers * M);
+  std::vector<uint8_t> have((size_t)n_layers * M, 0);
+  std::vector<qe::Launch> ls;
+  ls.reserve(2 * (size_t)n_actions + n_layers);
+  int32_t st = QE_OK;
+  uint32_t k = 0;
+  for (; k < n_actions && st == QE_OK; ++k) {
+    const qe_step_action& a = actions[k];
+    if (a.layer >= n_layers || a.mb >= M || a.kind > QE_ACT_DW) {
+      st = fail(QE_ERR_BAD_ARG, "action %u: kind %u layer %u mb %u", k, a.kind, a.layer, a.mb);
+      break;
+    }
+    qe_layer* L = layers[a.layer];
+    const size_t u = (size_t)a.layer * M + a.mb;
+    const qe_step_io& b = io[u];
+    if (a.kind == QE_ACT_F) {
+      int32_t refresh = 0;
+      uint32_t p = 0;
+      if (!b.x_dev || !b.y_dev || (((uintptr_t)b.x_dev | (uintptr_t)b.y_dev) & 15u)) { st = fail(QE_ERR_BAD_ARG, "action %u: x/y null or misaligned", k); break; }
+      if ((st = qe_contract_forward_check(L->contract, a.mb, L->contract->e_W, &refresh, &p)) != QE_OK) break;
+      if (L->dw_pending[p]) {  // a dW issued earlier through the overlapped per-action path still reads this slot
+        cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[p], 0);
+        L->dw_pending[p] = false;
+      }
+      if (refresh) add_refresh(L, ls);
+      add_forward(L, p, b.x_dev, b.y_dev, ls);
+      st = qe_contract_forward_commit(L->contract, a.mb, &tapes[u]);
+      have[u] = 1;
+    } else if (a.kind == QE_ACT_DI) {
+      if (!have[u]) { st = fail(QE_ERR_ORDER, "action %u: dI before F in this list", k); break; }
+      if (!b.dy_dev || !b.dx_dev || (((uintptr_t)b.dy_dev | (uintptr_t)b.dx_dev) & 15u)) { st = fail(QE_ERR_BAD_ARG, "action %u: dy/dx null or misaligned", k); break; }
+      if ((st = qe_contract_dI_check(L->contract, &tapes[u])) != QE_OK) break;
+      add_dI(L, tapes[u].ref.slot, b.dy_dev, b.dx_dev, ls);
+      st = qe_contract_dI_commit(L->contract, &tapes[u]);
+    } else {
+      if (!have[u]) { st = fail(QE_ERR_ORDER, "action %u: dW before F in this list", k); break; }
+      const uint64_t slice = (uint64_t)L->cfg.N * L->cfg.K;
+      int32_t acc = 0;
+      if ((st = qe_contract_dW_check(L->contract, &tapes[u], (uint64_t)(uintptr_t)grad, grad_elems, offsets[a.layer], slice, &acc)) != QE_OK) break;
+      add_dW(L, tapes[u].ref.slot, grad + offsets[a.layer], acc, temp, ls);
+      st = qe_contract_dW_commit(L->contract, &tapes[u], (uint64_t)(uintptr_t)grad, offsets[a.layer], slice);
+    }
+  }
+  const int32_t check_status = st;
+  char saved_msg[512];
+  std::snprintf(saved_msg, sizeof(saved_msg), "%s", qe_last_error());
+
+  // ---- device pass: the launches of every action that passed, behind one handshake
+  int32_t run_status = QE_OK;
+  if (!ls.empty()) {
+    run_status = handoff_in(ctx, caller);
+    if (run_status == QE_OK) {
+      if (ctx->exec_mode == QE_EXEC_GRAPH && check_status == QE_OK) {
+        uint64_t key = 1469598103934665603ull;  // FNV-1a over the list's identity
+        auto mix = [&key](const void* ptr, size_t n) {
+          const unsigned char* c = (const unsigned char*)ptr;
+          for (size_t i = 0; i < n; ++i) key = (key ^ c[i]) * 1099511628211ull;
+        };
+        mix(layers, sizeof(qe_layer*) * n_layers);
+        mix(actions, sizeof(qe_step_action) * n_actions);
+        mix(&M, sizeof(M));
+        qe_ctx::StepGraph* sg = nullptr;
+        for (auto* c : ctx->step_graphs)
+          if (c->key == key) sg = c;
+        if (sg && sg->g.launches.size() != ls.size()) {  // same list, different kernels (e.g. no weight refresh this time)
+          destroy_graph(&sg->g);
+          sg->g = ActionGraph();
+        }
+        if (!sg) {
+          sg = new (std::nothrow) qe_ctx::StepGraph();
+          if (!sg) return fail(QE_ERR_BAD_ARG, "out of host memory");
+          sg->key = key;
+          ctx->step_graphs.push_back(sg);
+        }
+        run_status = run_action(ctx, &sg->g, ls);
+      } else {
+        for (const qe::Launch& l : ls)
+          if ((run_status = launch_eager(ctx, l, ctx->exec_stream)) != QE_OK) break;
+      }
+    }
+    if (run_status == QE_OK) run_status = handoff_out(ctx, caller);
+  }
+  if (check_status != QE_OK || run_status != QE_OK) {
+    // failure boundary: outstanding tapes aborted, arenas unusable for the epoch
+    for (uint32_t l = 0; l < n_layers; ++l) qe_contract_abort(layers[l]->contract);
+    if (check_status != QE_OK) return fail(check_status, "step aborted at action %u: %s", k, saved_msg);
+    return run_status;
+  }
+  return QE_OK;
 }
 
 static int32_t read_status(qe_layer* L, uint32_t* status) {
