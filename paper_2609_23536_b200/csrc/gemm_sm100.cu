@@ -237,6 +237,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   const uint32_t num_kb = p.Kc / BK;
   const bool m_fastest = p.M <= p.N;
 
+  if (threadIdx.x == 32) {  // descriptor fetch overlaps the rest of the prologue (and the predecessor's tail)
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full_bar(s), 1);
