@@ -402,3 +402,43 @@ def test_host_buffer_entry_points_equal_the_device_ones_bitwise(qe, mode):
     with pytest.raises(qe.QEError) as e:
         L.forward_host(0, 0, torch.zeros((T, K), dtype=torch.bfloat16), None)
     assert e.value.code == "BAD_ARG"
+
+
+def test_limits_longest_history_most_slots_and_microbatches(qe):
+    # H = 4096 (longest history), 64 slots and 64 microbatches (the write mask's width): all forwards first, then all
+    # input-grads, then all weight-grads, against the oracle's state; a 65th microbatch index is rejected.
+    T = K = N = 256
+    M = 64
+    ctx, L = _mk_layer(qe, 1, T, K, N, 4096, 2, 64)
+    O = OracleLinear(T, K, N, 4096, 2, 64)
+    w = inputs.weights("LIM", 0, 0, N, K)
+    L.weight.copy_(w.to(DEV))
+    O.set_weight(inputs.bits(w))
+    buf = torch.zeros(N * K, device=DEV)
+    obuf = np.zeros(N * K, np.float32)
+    y = torch.empty((T, N), dtype=torch.bfloat16, device=DEV)
+    dx = torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+    gt, ot = {}, {}
+    for m in range(M):
+        X, _ = c1_inputs(0, m % 4, T, K, N, "LIM")
+        gt[m] = L.forward(m, 0, inputs.from_bits(X).to(DEV), y)
+        ot[m], _ = O.forward(m, 0, X, rows=[0])
+        assert gt[m].astuple() == (tuple(ot[m].key), tuple(ot[m].ref))
+    with pytest.raises(qe.QEError) as e:
+        L.forward(64, 0, inputs.from_bits(X).to(DEV), y)
+    assert e.value.code == "BAD_ARG"
+    with pytest.raises(qe.QEError) as e:
+        L.forward(0, 0, inputs.from_bits(X).to(DEV), y)
+    assert e.value.code == "KEY_LIVE"
+    for m in range(M):
+        _, dY = c1_inputs(0, m % 4, T, K, N, "LIM")
+        L.backward_dI(gt[m], inputs.from_bits(dY).to(DEV), dx)
+        O.backward_dI(ot[m], dY, rows=[0])
+    for m in range(M):
+        L.backward_dW(gt[m], buf, 0)
+        O.backward_dW(ot[m], obuf, 0)
+    assert state_equal_except_Y(L.state(), O.state())
+    assert assert_grad_close(buf.cpu().numpy(), obuf, "64 microbatches") < 1e-5
+    L.optimizer_boundary(64)
+    O.optimizer_boundary(64)
+    assert L.state()["e_W"] == 1 and L.state()["write_mask"] == 0
