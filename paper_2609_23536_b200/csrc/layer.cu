@@ -797,6 +797,13 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
   int32_t run_status = QE_OK;
   if (!ls.empty()) {
     run_status = handoff_in(ctx, caller);
+    if (run_status == QE_OK && ctx->dw_stream) {
+      // weight-gradient work issued earlier through the overlapped per-action path must finish first: this list's
+      // dW kernels run on the execution stream and accumulate into the same buffer
+      cudaError_t e = cudaEventRecord(ctx->ev_dw_in, ctx->dw_stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_dw_in, 0);
+      if (e != cudaSuccess) run_status = fail(QE_ERR_CUDA, "joining the dW stream: %s", cudaGetErrorString(e));
+    }
     if (run_status == QE_OK) {
       if (ctx->exec_mode == QE_EXEC_GRAPH && check_status == QE_OK) {
         uint64_t key = 1469598103934665603ull;  // FNV-1a over the list's identity
