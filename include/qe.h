@@ -23,7 +23,7 @@
  *     no device memory.
  *   - Tensors are dense row-major.  bf16 = IEEE bfloat16 bit patterns (2 bytes).  Tokens T, in-features K,
  *     out-features N:  X[T,K], W[N,K], Y[T,N], dY[T,N], dX[T,K]; a gradient slice is [N,K] FP32 at
- *     grad_buf + offset (offset in ELEMENTS).  T, K, N must be multiples of 128.
+ *     grad_buf + offset (offset in ELEMENTS).  T, K, N must be multiples of 128 in [256, 2^20].
  *   - Streams are cudaStream_t passed as void* (NULL = the legacy default stream).  Work is issued on the
  *     context's own execution stream; each action first makes that stream wait on the caller's stream and
  *     finally makes the caller's stream wait on the action's tail, so the caller may use its outputs on
@@ -44,7 +44,7 @@ extern "C" {
 typedef enum qe_status {
   QE_OK = 0,
   QE_ERR_BAD_ARG = -1,      /* null pointer, index out of range, unknown enum value                           */
-  QE_ERR_SHAPE = -2,        /* T, K or N not a multiple of 128, zero, or beyond the supported range           */
+  QE_ERR_SHAPE = -2,        /* T, K or N not a multiple of 128 or outside [256, 2^20]                         */
   QE_ERR_KEY_LIVE = -3,     /* forward: the same TapeKey already has a live tape (mapping must stay injective)*/
   QE_ERR_POOL_FULL = -4,    /* forward: no free slot; an occupied slot is never pre-empted                    */
   QE_ERR_STALE_CACHE = -5,  /* forward: e_C != e_W on a non-first forward ("cache refresh required")          */
@@ -172,7 +172,7 @@ typedef struct qe_ctx_config {
 #define QE_CTX_UNSAFE_ONE_WAY_HANDOFF 2u
 
 typedef struct qe_layer_config {
-  uint32_t T, K, N;       /* tokens, in-features, out-features: multiples of 128                             */
+  uint32_t T, K, N;       /* tokens, in-features, out-features: multiples of 128 in [256, 2^20]          */
   uint32_t history_len;   /* H in [1, QE_MAX_HISTORY]                                                        */
   int32_t margin;         /* scale = fp8_max / max(history) / 2^margin; margin in [-32, 32]                  */
   uint32_t slots;         /* tape slots P in [1, QE_MAX_SLOTS]                                               */
@@ -308,7 +308,8 @@ uint32_t qe_amax_partials(void);
 int32_t qe_accumulate(float* dst_dev, const float* src_dev, uint64_t n, int32_t accumulate, void* stream);
 /* One FP8 GEMM on the tensor cores: D[m,n] = (sum_k A[m,k] B[n,k]) * *alpha_a_dev * *alpha_b_dev with A [M,Kc] and
  * B [Nn,Kc] both contraction-major bytes.  out_kind 0: bf16 D (amax_dev optional, as in qe_quantize); 1: FP32
- * D overwrite; 2: FP32 D accumulate.  M, Nn, Kc multiples of 128.  status_dev: one uint32 the kernel ORs error
+ * D overwrite; 2: FP32 D accumulate.  M, Kc multiples of 128 (>= 128), Nn a multiple of 128 (>= 256).  A 256-row paired-CTA variant runs when
+ * M is a multiple of 256, a single-CTA 128-row variant otherwise.  status_dev: one uint32 the kernel ORs error
  * bits into (caller zeroes it). */
 int32_t qe_gemm_fp8(const void* a_dev, uint32_t a_format, const void* b_dev, uint32_t b_format, uint32_t M,
                     uint32_t Nn, uint32_t Kc, const float* alpha_a_dev, const float* alpha_b_dev, void* d_dev,
