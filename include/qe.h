@@ -315,6 +315,15 @@ int32_t qe_gemm_fp8(const void* a_dev, uint32_t a_format, const void* b_dev, uin
                     uint32_t Nn, uint32_t Kc, const float* alpha_a_dev, const float* alpha_b_dev, void* d_dev,
                     uint32_t out_kind, float* amax_dev, uint32_t* status_dev, void* stream);
 
+/* As qe_gemm_fp8, with either operand optionally given MN-major: a_mn = 1 means a_dev holds A as [Kc, M] bytes (M
+ * contiguous) instead of [M, Kc]; b_mn = 1 means b_dev holds B as [Kc, Nn].  The tensor cores read such tiles
+ * directly, so no transposed copy of a row-major tensor is needed to contract over its rows.  MN-major operands
+ * require M to be a multiple of 256 (QE_ERR_UNSUPPORTED otherwise). */
+int32_t qe_gemm_fp8_ex(const void* a_dev, uint32_t a_format, uint32_t a_mn, const void* b_dev, uint32_t b_format,
+                       uint32_t b_mn, uint32_t M, uint32_t Nn, uint32_t Kc, const float* alpha_a_dev,
+                       const float* alpha_b_dev, void* d_dev, uint32_t out_kind, float* amax_dev, uint32_t* status_dev,
+                       void* stream);
+
 /* (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
  * The copied-gradient step without any allocation: D = (A . B^T) * *alpha_a_dev * *alpha_b_dev is written to a
  * staging area that is built into the library (a fixed device array of qe_noalloc_staging_elems() = 2^20 FP32

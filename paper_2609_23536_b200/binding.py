@@ -154,6 +154,7 @@ _SIGNATURES = {
     "qe_amax_partials": (C.c_uint32, []),
     "qe_accumulate": (C.c_int32, [_P, _P, C.c_uint64, C.c_int32, _P]),
     "qe_gemm_fp8": (C.c_int32, [_P, C.c_uint32, _P, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, _P, _P, _P, C.c_uint32, _P, _P, _P]),
+    "qe_gemm_fp8_ex": (C.c_int32, [_P, C.c_uint32, C.c_uint32, _P, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, _P, _P, _P, C.c_uint32, _P, _P, _P]),
     "qe_gemm_fp8_staged_noalloc": (C.c_int32, [_P, C.c_uint32, _P, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, _P, _P, _P, C.c_int32, _P, _P]),
     "qe_noalloc_staging_elems": (C.c_uint64, []),
     "qe_last_error": (C.c_char_p, []),
@@ -439,6 +440,14 @@ def qe_gemm_fp8(a, a_fmt, b, b_fmt, alpha_a_dev, alpha_b_dev, d, out_kind, amax_
     assert Kc == Kc2
     _check(lib.qe_gemm_fp8(_ptr(a), a_fmt, _ptr(b), b_fmt, M, Nn, Kc, _ptr(alpha_a_dev), _ptr(alpha_b_dev), _ptr(d),
                            out_kind, _ptr(amax_dev), _ptr(status_dev), _stream(stream)))
+
+
+def qe_gemm_fp8_ex(a, a_fmt, a_mn, b, b_fmt, b_mn, alpha_a_dev, alpha_b_dev, d, out_kind, amax_dev=None, status_dev=None, stream=None):
+    """a is [M, Kc] (a_mn False) or [Kc, M] (a_mn True); likewise b with Nn."""
+    M, Kc = (a.shape[1], a.shape[0]) if a_mn else a.shape
+    Nn = b.shape[1] if b_mn else b.shape[0]
+    _check(lib.qe_gemm_fp8_ex(_ptr(a), a_fmt, int(a_mn), _ptr(b), b_fmt, int(b_mn), M, Nn, Kc, _ptr(alpha_a_dev), _ptr(alpha_b_dev),
+                              _ptr(d), out_kind, _ptr(amax_dev), _ptr(status_dev), _stream(stream)))
 
 
 def qe_gemm_fp8_staged_noalloc(a, a_fmt, b, b_fmt, alpha_a_dev, alpha_b_dev, dst, accumulate: bool, status_dev, stream=None):

@@ -293,8 +293,13 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
             // both CTAs credit the even CTA's barrier, which expects the bytes of the whole pair
             if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
             const uint32_t bar = map_to_cta(full_bar(s), 0);
-            tma_load_2d_pair(a_dst, &p.tmA, bar, (int)(kb * BK), (int)(m0 + rank * BM));
-            tma_load_2d_pair(b_dst, &p.tmB, bar, (int)(kb * BK), (int)(n0 + rank * C::B_ROWS));
+            // contraction-major operand: box = 128 K-bytes x 128 rows at (k, row); MN-major operand (stored as
+            // [Kc, rows]): box = 128 row-bytes x 128 K-rows at (row, k).  Either way 16 KB land in shared memory.
+            const int ka = (int)(kb * BK), ra = (int)(m0 + rank * BM), rb = (int)(n0 + rank * C::B_ROWS);
+            if (p.a_mn) tma_load_2d_pair(a_dst, &p.tmA, bar, ra, ka);
+            else tma_load_2d_pair(a_dst, &p.tmA, bar, ka, ra);
+            if (p.b_mn) tma_load_2d_pair(b_dst, &p.tmB, bar, rb, ka);
+            else tma_load_2d_pair(b_dst, &p.tmB, bar, ka, rb);
           } else {
             mbar_expect_tx(full_bar(s), STAGE_BYTES);
             tma_load_2d(a_dst, &p.tmA, full_bar(s), (int)(kb * BK), (int)m0);
@@ -326,8 +331,9 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           const uint64_t adesc = make_desc(a_src), bdesc = make_desc(b_src);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
-            // advancing 32 bytes along the contraction inside the 128-byte swizzle row: +2 in the address field
-            if (TWO) tc_mma_f8_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | (uint32_t)k) != 0u);
+            // advancing 32 along the contraction: 32 bytes inside the 128-byte swizzle row for a contraction-major
+            // tile (+2 in the address field), 32 rows of 128 bytes for an MN-major one (+256)
+            if (TWO) tc_mma_f8_pair(d_tmem, adesc + (p.a_mn ? 256u : 2u) * k, bdesc + (p.b_mn ? 256u : 2u) * k, p.idesc, (kb | (uint32_t)k) != 0u);
             else tc_mma_f8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | (uint32_t)k) != 0u);
           }
           if (TWO) tc_commit_pair(empty_bar(s));  // stage reusable (in both CTAs) once these MMAs have read it
@@ -477,12 +483,12 @@ bool gemm_uses_pair(uint32_t M) { return M % 256 == 0; }
 
 uint32_t gemm_b_box_rows(uint32_t M) { return gemm_uses_pair(M) ? 128u : 256u; }
 
-uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M) {
+uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M, bool a_mn, bool b_mn) {
   // bits 4-5: accumulator format (1 = FP32); 7-9 / 10-12: A / B format (0 = E4M3, 1 = E5M2); 15 / 16: A / B major
   // (0 = contraction-major); 17-22: N >> 3; 24-28: M >> 4 (128 per CTA, 256 for a CTA pair).
   const uint32_t mma_m = gemm_uses_pair(M) ? 256u : 128u;
-  return (1u << 4) | ((uint32_t)a_fmt << 7) | ((uint32_t)b_fmt << 10) | ((uint32_t)(BN >> 3) << 17) |
-         ((mma_m >> 4) << 24);
+  return (1u << 4) | ((uint32_t)a_fmt << 7) | ((uint32_t)b_fmt << 10) | ((a_mn ? 1u : 0u) << 15) |
+         ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((mma_m >> 4) << 24);
 }
 
 cudaError_t gemm_prepare() {

@@ -71,7 +71,8 @@ struct GemmParams {
   CUtensorMap tmA;             // A [M, Kc] bytes, box 128 x 128, 128-byte swizzle
   CUtensorMap tmB;             // B [N, Kc] bytes, box 128 x gemm_b_box_rows(M)
   uint32_t M, N, Kc;
-  uint32_t idesc;              // tcgen05 instruction descriptor (formats, 128 x 256 shape)
+  uint32_t idesc;              // tcgen05 instruction descriptor (formats, majors, shape)
+  uint32_t a_mn, b_mn;         // operand given MN-major (as [Kc, M] / [Kc, N] bytes): paired variant only
   const float* alpha_a;
   const float* alpha_b;
   void* out;                   // bf16 or FP32 [M, N], row pitch ldo elements
@@ -104,7 +105,8 @@ Launch make_amax_pass2(const AmaxParams& p);
 Launch make_accumulate(const AccumParams& p);
 Launch make_gemm(const GemmParams& p, int num_sms);
 cudaError_t gemm_prepare();  // opt in to the dynamic shared memory the GEMM needs (once per device)
-uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M);
+uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M, bool a_mn = false, bool b_mn = false);
+bool gemm_uses_pair(uint32_t M);
 uint32_t gemm_b_box_rows(uint32_t M);  // rows of the B operand's TMA box for a GEMM with M rows (128 paired, 256 single)
 constexpr uint32_t kAmaxPartials = 2048;
 

@@ -1083,24 +1083,31 @@ int32_t qe_accumulate(float* dst, const float* src, uint64_t n, int32_t accumula
   return launch_on(qe::make_accumulate(ap), (cudaStream_t)stream);
 }
 
-int32_t qe_gemm_fp8(const void* a, uint32_t a_fmt, const void* b, uint32_t b_fmt, uint32_t M, uint32_t Nn, uint32_t Kc,
-                    const float* alpha_a, const float* alpha_b, void* d, uint32_t out_kind, float* amax_dev,
-                    uint32_t* status_dev, void* stream) {
+int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void* b, uint32_t b_fmt, uint32_t b_mn,
+                       uint32_t M, uint32_t Nn, uint32_t Kc, const float* alpha_a, const float* alpha_b, void* d,
+                       uint32_t out_kind, float* amax_dev, uint32_t* status_dev, void* stream) {
   if (!a || !b || !alpha_a || !alpha_b || !d || !status_dev) return fail(QE_ERR_BAD_ARG, "null argument");
-  if (a_fmt > QE_E5M2 || b_fmt > QE_E5M2 || out_kind > 2) return fail(QE_ERR_BAD_ARG, "bad enum");
+  if (a_fmt > QE_E5M2 || b_fmt > QE_E5M2 || out_kind > 2 || a_mn > 1 || b_mn > 1) return fail(QE_ERR_BAD_ARG, "bad enum");
   if (!shape_ok(M) && M != 128) return fail(QE_ERR_SHAPE, "M=%u", M);
-  if (!shape_ok(Nn) || !shape_ok(Kc) && Kc != 128) return fail(QE_ERR_SHAPE, "N=%u Kc=%u", Nn, Kc);
+  if (!shape_ok(Nn) || (!shape_ok(Kc) && Kc != 128)) return fail(QE_ERR_SHAPE, "N=%u Kc=%u", Nn, Kc);
+  if ((a_mn || b_mn) && !qe::gemm_uses_pair(M))
+    return fail(QE_ERR_UNSUPPORTED, "MN-major operands need M to be a multiple of 256 (paired-CTA variant), M=%u", M);
   if ((((uintptr_t)a | (uintptr_t)b | (uintptr_t)d) & 15u)) return fail(QE_ERR_BAD_ARG, "misaligned pointer");
   DeviceInfo* dev = nullptr;
   int32_t st = current_device_info(&dev);
   if (st != QE_OK) return st;
   qe::GemmParams gp{};
-  if ((st = make_map(dev, &gp.tmA, a, M, Kc, 128)) != QE_OK) return st;
-  if ((st = make_map(dev, &gp.tmB, b, Nn, Kc, qe::gemm_b_box_rows(M))) != QE_OK) return st;
+  // contraction-major operand: [rows, Kc]; MN-major operand: [Kc, rows] with a 128 x 128 box
+  st = a_mn ? make_map(dev, &gp.tmA, a, Kc, M, 128) : make_map(dev, &gp.tmA, a, M, Kc, 128);
+  if (st != QE_OK) return st;
+  st = b_mn ? make_map(dev, &gp.tmB, b, Kc, Nn, 128) : make_map(dev, &gp.tmB, b, Nn, Kc, qe::gemm_b_box_rows(M));
+  if (st != QE_OK) return st;
   gp.M = M;
   gp.N = Nn;
   gp.Kc = Kc;
-  gp.idesc = qe::gemm_idesc((int)a_fmt, (int)b_fmt, M);
+  gp.idesc = qe::gemm_idesc((int)a_fmt, (int)b_fmt, M, a_mn != 0, b_mn != 0);
+  gp.a_mn = a_mn;
+  gp.b_mn = b_mn;
   gp.alpha_a = alpha_a;
   gp.alpha_b = alpha_b;
   gp.out = d;
@@ -1109,6 +1116,12 @@ int32_t qe_gemm_fp8(const void* a, uint32_t a_fmt, const void* b, uint32_t b_fmt
   gp.amax_bits = (uint32_t*)amax_dev;
   gp.status = status_dev;
   return launch_on(qe::make_gemm(gp, dev->num_sms), (cudaStream_t)stream);
+}
+
+int32_t qe_gemm_fp8(const void* a, uint32_t a_fmt, const void* b, uint32_t b_fmt, uint32_t M, uint32_t Nn, uint32_t Kc,
+                    const float* alpha_a, const float* alpha_b, void* d, uint32_t out_kind, float* amax_dev,
+                    uint32_t* status_dev, void* stream) {
+  return qe_gemm_fp8_ex(a, a_fmt, 0, b, b_fmt, 0, M, Nn, Kc, alpha_a, alpha_b, d, out_kind, amax_dev, status_dev, stream);
 }
 
 }  // extern "C"

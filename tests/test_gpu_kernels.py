@@ -174,3 +174,33 @@ def test_gemm_random_bytes_within_tolerance(qe, afmt, bfmt, M, Nn, Kc):
     floor = 2.0**-6 * np.sqrt(np.mean(acc**2))
     assert np.all(np.abs(got - want) <= 4 * bf16.ulp(np.maximum(np.abs(want), floor)))
     assert amax == float(np.abs(got).max())  # self-consistent with what was stored
+
+
+@pytest.mark.parametrize("a_mn,b_mn", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("M,Nn,Kc", [(256, 256, 128), (512, 768, 1024), (2048, 1280, 384)])
+def test_gemm_mn_major_operands_integer_exact(qe, a_mn, b_mn, M, Nn, Kc):
+    # the same product with operands handed over transposed ([Kc, M] / [Kc, Nn]): bit-exact on integer inputs
+    rng = np.random.default_rng(M + Nn + Kc + 2 * a_mn + b_mn)
+    A, Av = _int_codes(rng, (M, Kc), 8, fp8.E5M2)
+    B, Bv = _int_codes(rng, (Nn, Kc), 4, fp8.E4M3)
+    want = (Av.astype(np.float64) @ Bv.astype(np.float64).T).astype(np.float32)
+    Ad = torch.from_numpy(np.ascontiguousarray(A.T) if a_mn else A).to(DEV)
+    Bd = torch.from_numpy(np.ascontiguousarray(B.T) if b_mn else B).to(DEV)
+    one = torch.ones(1, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    D = torch.full((M, Nn), float("nan"), device=DEV)
+    qe.qe_gemm_fp8_ex(Ad, 1, a_mn, Bd, 0, b_mn, one, one, D, 1, None, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(D.cpu().numpy(), want)
+
+
+def test_gemm_mn_major_needs_the_paired_variant(qe):
+    one = torch.ones(1, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    A = torch.zeros((128, 384), dtype=torch.uint8, device=DEV)  # [Kc, M] with M = 384
+    B = torch.zeros((256, 128), dtype=torch.uint8, device=DEV)
+    D = torch.zeros((384, 256), device=DEV)
+    with pytest.raises(qe.QEError) as e:
+        qe.qe_gemm_fp8_ex(A, 0, True, B, 0, False, one, one, D, 1, None, status)
+    assert e.value.code == "UNSUPPORTED"
