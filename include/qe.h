@@ -193,13 +193,13 @@ int32_t qe_layer_create(qe_ctx*, const qe_layer_config*, void* workspace_dev, ui
 int32_t qe_layer_destroy(qe_layer*);
 
 /* F (Eq. 3).  x_dev bf16 [T,K] in, y_dev bf16 [T,N] out.  `gen` is the caller's view of the weight version and must
- * equal e_W.  On the first forward of an epoch the weight is re-quantised (E4M3, plus its transpose) and its amax
+ * equal e_W.  On the first forward of an epoch the weight is re-quantised (E4M3; plus its transpose where dI needs one) and its amax
  * committed.  Then: X quantised to E4M3 with the current scale (amax taken in the same pass; the inverse scale is
  * snapshotted into the tape slot), Y = bf16((Xq Wq^T) * sinv_X * sinv_W) on the tensor cores with max|Y| reduced in
  * the epilogue, and the X and Y histories/scales updated.  *tape_out names the retained work. */
 int32_t qe_forward(qe_layer*, uint32_t mb, uint64_t gen, const void* x_dev, void* y_dev, void* caller_stream,
                    qe_tape* tape_out);
-/* dI (Eq. 4).  dy_dev bf16 [T,N] in, dx_dev bf16 [T,K] out.  Quantises dY to E5M2 (and its transpose, retained for
+/* dI (Eq. 4).  dy_dev bf16 [T,N] in, dx_dev bf16 [T,K] out.  Quantises dY to E5M2 (and, where dW needs it, its transpose, retained for
  * dW), dX = bf16((Gq Wq) * sinv_G * sinv_W), commits the gradient amax/scale once. */
 int32_t qe_backward_dI(qe_layer*, const qe_tape*, const void* dy_dev, void* dx_dev, void* caller_stream);
 /* F and dI with HOST buffers (layer created with host_io = 1).  The input is copied host-to-device into the layer's
@@ -270,7 +270,9 @@ typedef struct qe_state_view {
  * sinv_X of slot p at [p], sinv_G at [P+p]. */
 int32_t qe_get_state(qe_layer*, qe_state_view* out, float* window_out, float* slot_sinv_out);
 /* Copies a slot's retained FP8 bytes to host memory (testing aid; synchronises).  which: 0 = Xq [T,K],
- * 1 = Xq^T [K,T], 2 = Gq [T,N], 3 = Gq^T [N,T], 4 = Wq [N,K] (slot ignored), 5 = Wq^T [K,N] (slot ignored). */
+ * 1 = Xq^T [K,T], 2 = Gq [T,N], 3 = Gq^T [N,T], 4 = Wq [N,K] (slot ignored), 5 = Wq^T [K,N] (slot ignored).
+ * Transposed copies exist only where a GEMM needs them: Wq^T when T is not a multiple of 256, Xq^T and Gq^T when N
+ * is not (otherwise the tensor cores read the row-major tensor as an MN-major operand) -- QE_ERR_UNSUPPORTED if absent. */
 int32_t qe_read_fp8(qe_layer*, uint32_t which, uint32_t slot, void* host_out, uint64_t bytes);
 
 /* Quiescent checkpoint (Sec. 3.5, Invariant 4).  The payload holds PERSISTENT state only: the static configuration

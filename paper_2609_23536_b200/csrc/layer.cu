@@ -139,7 +139,7 @@ struct qe_layer {
   uint8_t *Xq[QE_MAX_SLOTS], *XqT[QE_MAX_SLOTS], *Gq[QE_MAX_SLOTS], *GqT[QE_MAX_SLOTS];
   // tensor maps: A-role boxes are 128 rows, B-role boxes 256 rows
   CUtensorMap tmXq_A[QE_MAX_SLOTS], tmGq_A[QE_MAX_SLOTS], tmGqT_A[QE_MAX_SLOTS], tmXqT_B[QE_MAX_SLOTS];
-  CUtensorMap tmWq_B, tmWqT_B;
+  CUtensorMap tmWq_B, tmWqT_B, tmWq_B_mn;
   ActionGraph gF[QE_MAX_SLOTS], gDI[QE_MAX_SLOTS], gDW[QE_MAX_SLOTS], gDWs[QE_MAX_SLOTS], gRefresh, gCommit;
   // QE_CTX_OVERLAP_DW: per slot, "dI of the tape in this slot has been enqueued" / "the dW that released it has"
   cudaEvent_t ev_di[QE_MAX_SLOTS] = {}, ev_dw[QE_MAX_SLOTS] = {};
@@ -316,16 +316,19 @@ Carve carve(const qe_layer_config& c) {
   k.hist = o;
   o = align_up(o + 4ull * c.history_len * sizeof(float), 1024);
   const uint64_t nk = (uint64_t)c.N * c.K, tk = (uint64_t)c.T * c.K, tn = (uint64_t)c.T * c.N;
+  // Transposed FP8 copies exist only where a GEMM cannot take the row-major tensor as an MN-major operand: the dI
+  // GEMM (M = T) needs Wq^T, the dW GEMM (M = N) needs Xq^T and Gq^T, when that M is not a multiple of 256.
+  const bool wT = !qe::gemm_uses_pair(c.T), xgT = !qe::gemm_uses_pair(c.N);
   k.Wq = o;
   o += align_up(nk, 1024);
   k.WqT = o;
-  o += align_up(nk, 1024);
+  if (wT) o += align_up(nk, 1024);
   k.slot0 = o;
   k.xq = 0;
   k.xqT = align_up(tk, 1024);
-  k.gq = k.xqT + align_up(tk, 1024);
+  k.gq = k.xqT + (xgT ? align_up(tk, 1024) : 0);
   k.gqT = k.gq + align_up(tn, 1024);
-  k.per_slot = k.gqT + align_up(tn, 1024);
+  k.per_slot = k.gqT + (xgT ? align_up(tn, 1024) : 0);
   o += k.per_slot * c.slots;
   if (c.host_io) {  // x / dx [T,K] and y / dy [T,N] bf16 staging for the host-buffer entry points
     k.stage_tk = o;
@@ -411,12 +414,14 @@ void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::L
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
   qe::GemmParams gp{};
+  const bool b_mn = L->WqT == nullptr;  // no transposed weight copy: Wq [N,K] is B in MN-major form
   gp.tmA = L->tmGq_A[p];
-  gp.tmB = L->tmWqT_B;
+  gp.tmB = b_mn ? L->tmWq_B_mn : L->tmWqT_B;
   gp.M = T;
   gp.N = K;
   gp.Kc = N;
-  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, T);
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, T, false, b_mn);
+  gp.b_mn = b_mn;
   gp.alpha_a = &L->st->slot_sinv_G[p];
   gp.alpha_b = &L->st->cache_sinv_W;
   gp.out = dx;
@@ -432,12 +437,14 @@ void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::L
 void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp, std::vector<qe::Launch>& ls) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   qe::GemmParams gp{};
+  const bool mn = L->GqT[p] == nullptr;  // Gq [T,N] and Xq [T,K] themselves, read as MN-major operands
   gp.tmA = L->tmGqT_A[p];
   gp.tmB = L->tmXqT_B[p];
   gp.M = N;
   gp.N = K;
   gp.Kc = T;
-  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, N);
+  gp.idesc = qe::gemm_idesc(QE_E5M2, QE_E4M3, N, mn, mn);
+  gp.a_mn = gp.b_mn = mn;
   gp.alpha_a = &L->st->slot_sinv_G[p];  // snapshots taken when dY_m and X_m were quantised, never the current state
   gp.alpha_b = &L->st->slot_sinv_X[p];
   gp.ldo = K;
@@ -545,8 +552,9 @@ int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint6
   uint8_t* base = (uint8_t*)ws;
   L->st = (qe::DevState*)base;
   L->hist = (float*)(base + k.hist);
+  const bool wT = !qe::gemm_uses_pair(cfg->T), xgT = !qe::gemm_uses_pair(cfg->N);
   L->Wq = base + k.Wq;
-  L->WqT = base + k.WqT;
+  L->WqT = wT ? base + k.WqT : nullptr;
   if (cfg->host_io) {
     L->x_stage = base + k.stage_tk;
     L->dx_stage = L->x_stage + align_up(2ull * cfg->T * cfg->K, 1024);
@@ -558,16 +566,22 @@ int32_t qe_layer_create(qe_ctx* ctx, const qe_layer_config* cfg, void* ws, uint6
   for (uint32_t p = 0; p < cfg->slots; ++p) {
     uint8_t* s = base + k.slot0 + k.per_slot * p;
     L->Xq[p] = s + k.xq;
-    L->XqT[p] = s + k.xqT;
+    L->XqT[p] = xgT ? s + k.xqT : nullptr;
     L->Gq[p] = s + k.gq;
-    L->GqT[p] = s + k.gqT;
+    L->GqT[p] = xgT ? s + k.gqT : nullptr;
     if ((st = make_map(d, &L->tmXq_A[p], L->Xq[p], T, K, 128)) != QE_OK) break;   // F:  A = Xq  [T,K]
     if ((st = make_map(d, &L->tmGq_A[p], L->Gq[p], T, N, 128)) != QE_OK) break;   // dI: A = Gq  [T,N]
-    if ((st = make_map(d, &L->tmGqT_A[p], L->GqT[p], N, T, 128)) != QE_OK) break; // dW: A = Gq^T [N,T]
-    if ((st = make_map(d, &L->tmXqT_B[p], L->XqT[p], K, T, qe::gemm_b_box_rows(N))) != QE_OK) break; // dW: B = Xq^T [K,T]
+    if (xgT) {
+      if ((st = make_map(d, &L->tmGqT_A[p], L->GqT[p], N, T, 128)) != QE_OK) break; // dW: A = Gq^T [N,T]
+      if ((st = make_map(d, &L->tmXqT_B[p], L->XqT[p], K, T, qe::gemm_b_box_rows(N))) != QE_OK) break; // dW: B = Xq^T [K,T]
+    } else {  // dW reads Gq [T,N] and Xq [T,K] as MN-major operands: 128 x 128 boxes over the row-major tensors
+      if ((st = make_map(d, &L->tmGqT_A[p], L->Gq[p], T, N, 128)) != QE_OK) break;
+      if ((st = make_map(d, &L->tmXqT_B[p], L->Xq[p], T, K, 128)) != QE_OK) break;
+    }
   }
   if (st == QE_OK) st = make_map(d, &L->tmWq_B, L->Wq, N, K, qe::gemm_b_box_rows(T));    // F:  B = Wq   [N,K]
-  if (st == QE_OK) st = make_map(d, &L->tmWqT_B, L->WqT, K, N, qe::gemm_b_box_rows(T));  // dI: B = Wq^T [K,N]
+  if (st == QE_OK)  // dI: B = Wq^T [K,N], or Wq [N,K] itself as an MN-major operand
+    st = wT ? make_map(d, &L->tmWqT_B, L->WqT, K, N, qe::gemm_b_box_rows(T)) : make_map(d, &L->tmWq_B_mn, L->Wq, N, K, 128);
   if (st != QE_OK) { qe_contract_destroy(L->contract); delete L; return st; }
   // state: histories 0, scales 1, everything else 0
   qe::DevState init{};
@@ -934,6 +948,7 @@ int32_t qe_read_fp8(qe_layer* L, uint32_t which, uint32_t slot, void* host_out, 
   if (which > 5 || (which < 4 && slot >= L->cfg.slots)) return fail(QE_ERR_BAD_ARG, "which %u slot %u", which, slot);
   const uint8_t* src = which == 0 ? L->Xq[slot] : which == 1 ? L->XqT[slot] : which == 2 ? L->Gq[slot]
                      : which == 3 ? L->GqT[slot] : which == 4 ? L->Wq : L->WqT;
+  if (!src) return fail(QE_ERR_UNSUPPORTED, "this layer keeps no transposed copy %u (its GEMM reads the row-major tensor directly)", which);
   const uint64_t need = which < 2 ? tk : which < 4 ? tn : nk;
   if (bytes != need) return fail(QE_ERR_BAD_ARG, "bytes %llu, tensor has %llu", (unsigned long long)bytes, (unsigned long long)need);
   QE_CUDA(cudaStreamSynchronize(L->ctx->exec_stream));

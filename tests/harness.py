@@ -128,3 +128,15 @@ def state_equal_except_Y(gpu: dict, orc: dict) -> bool:
             return False
     keys = ("token", "e_W", "e_C", "write_mask", "fwd_in_epoch", "aborted", "slots")
     return all(gpu[k] == orc[k] for k in keys)
+
+
+def transposed_or_none(layer, which, slot=0):
+    """A layer's transposed FP8 copy (which = 1, 3, 5), or None when the layer keeps none because its GEMMs read the
+    row-major tensor as an MN-major operand."""
+    from paper_2609_23536_b200 import binding as qe
+
+    try:
+        return layer.read_fp8(which, slot)
+    except qe.QEError as e:
+        assert e.code == "UNSUPPORTED"
+        return None

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from harness import (assert_gemm_close, assert_grad_close, c1_inputs, run_gpu_steps, run_oracle_steps, state_equal,
-                     state_equal_except_Y)
+                     state_equal_except_Y, transposed_or_none)
 from oracle import bf16, fp8
 from oracle.layer import ContractError, OracleLinear
 from paper_2609_23536_b200 import inputs
@@ -72,12 +72,13 @@ def test_config1_every_action_against_oracle(qe, mode):
         assert g["device_status"] == 0 and g["device_token"] == g["token"]
         assert state_equal_except_Y(g, ostate), (step, a, m)
         assert np.float32(g["cache_sinv_W"]).view(np.uint32) == np.float32(osinvW).view(np.uint32)
-        assert np.array_equal(layer.read_fp8(4), oWq) and np.array_equal(layer.read_fp8(5), oWq.T)
+        assert np.array_equal(layer.read_fp8(4), oWq)
+        assert transposed_or_none(layer, 5) is None  # 256-multiples: the dI GEMM reads Wq itself, MN-major
         for p, (Xq, Gq, sX, sG) in oslots.items():
-            assert np.array_equal(layer.read_fp8(0, p), Xq) and np.array_equal(layer.read_fp8(1, p), Xq.T)
+            assert np.array_equal(layer.read_fp8(0, p), Xq) and transposed_or_none(layer, 1, p) is None
             assert g["slot_sinv_X"][p].view(np.uint32) == np.float32(sX).view(np.uint32)
             if Gq is not None:
-                assert np.array_equal(layer.read_fp8(2, p), Gq) and np.array_equal(layer.read_fp8(3, p), Gq.T)
+                assert np.array_equal(layer.read_fp8(2, p), Gq) and transposed_or_none(layer, 3, p) is None
                 assert g["slot_sinv_G"][p].view(np.uint32) == np.float32(sG).view(np.uint32)
         # class Y: newest entry is max|Y_gpu| exactly; its scale is the closed form of the GPU's own window
         gy = g["classes"]["Y"]
@@ -180,6 +181,9 @@ def test_shapes_that_take_the_single_cta_gemm_against_oracle(qe, mode):
         else:
             assert_gemm_close(got[k], want[k], k)
     assert state_equal_except_Y(L.state(), O.state())
+    # these shapes keep transposed copies (their dI / dW GEMMs take contraction-major operands only)
+    assert np.array_equal(L.read_fp8(5), O.Wq.T) and np.array_equal(L.read_fp8(4), O.Wq)
+    assert L.read_fp8(1, 0).shape == (K, T) and L.read_fp8(3, 0).shape == (N, T)
 
 
 def test_scale_commit_standalone_matches_hand_worked_rollover(qe):
