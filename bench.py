@@ -248,26 +248,27 @@ def gemm_roofline(qe, cfg, peaks, device):
     T = cfg["T"]
     shapes = []
     for _, K, N in cfg["linears"]:
-        shapes += [("F", T, N, K, 0, 0, 0), ("dI", T, K, N, 1, 0, 0), ("dW", N, K, T, 1, 0, 2)]
+        # (name, M, N, Kc, A format, A MN-major, B MN-major, epilogue): operand majors as the layer uses them
+        shapes += [("F", T, N, K, 0, 0, 0, 0), ("dI", T, K, N, 1, 0, 1, 0), ("dW", N, K, T, 1, 1, 1, 2)]
     one = torch.ones(1, dtype=torch.float32, device=device)
     status = torch.zeros(1, dtype=torch.int32, device=device)
     tot_flops = tot_ms = 0.0
     per = {}
-    for name, M_, N_, Kc, af, bf, kind in shapes:
+    for name, M_, N_, Kc, af, amn, bmn, kind in shapes:
         nset = max(2, int(160e6 // (M_ * Kc + N_ * Kc + M_ * N_ * (2 if kind == 0 else 8))) + 1)
         nset = min(nset, 24)
-        A = [torch.randint(0, 120, (M_, Kc), dtype=torch.uint8, device=device) for _ in range(nset)]
-        B = [torch.randint(0, 120, (N_, Kc), dtype=torch.uint8, device=device) for _ in range(nset)]
+        A = [torch.randint(0, 120, (Kc, M_) if amn else (M_, Kc), dtype=torch.uint8, device=device) for _ in range(nset)]
+        B = [torch.randint(0, 120, (Kc, N_) if bmn else (N_, Kc), dtype=torch.uint8, device=device) for _ in range(nset)]
         D = [torch.zeros((M_, N_), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=device) for _ in range(nset)]
         reps = 3 * nset
         for i in range(nset):
-            qe.qe_gemm_fp8(A[i], af, B[i], bf, one, one, D[i], kind, None, status)
+            qe.qe_gemm_fp8_ex(A[i], af, bool(amn), B[i], 0, bool(bmn), one, one, D[i], kind, None, status)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for r in range(reps):
             i = r % nset
-            qe.qe_gemm_fp8(A[i], af, B[i], bf, one, one, D[i], kind, None, status)
+            qe.qe_gemm_fp8_ex(A[i], af, bool(amn), B[i], 0, bool(bmn), one, one, D[i], kind, None, status)
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
@@ -308,7 +309,7 @@ def gemm_roofline(qe, cfg, peaks, device):
     return {
         "bound": "tensor", "kernel": "gemm_fp8_pair_kernel", "achieved": round(achieved, 1), "peak": round(peak, 1),
         "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": traffic,
-        "algorithmic_bytes_per_launch": round(sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if k == 0 else 8) for _, M_, N_, Kc, _, _, k in shapes) / len(shapes)),
+        "algorithmic_bytes_per_launch": round(sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if k == 0 else 8) for _, M_, N_, Kc, _, _, _, k in shapes) / len(shapes)),
         "flop_per_launch": round(tot_flops / len(shapes)), "launches_timed": len(shapes), "peak_source": peaks["source"] + " bf16 burst x2",
         "frac_of_nominal_4500": round(achieved / 4500.0, 4),
         "per_action_tflops": {k: round(v[0] / (v[1] * 1e-3) / 1e12, 1) for k, v in per.items()},

@@ -32,27 +32,30 @@ def main():
     if a.case == "gemm_microbatch":
         # the twelve GEMMs (F, dI, dW of four linears) one microbatch of the Llama-style block launches, in order
         shapes = []
+        # operand majors as the layer uses them: F both contraction-major; dI takes Wq [N,K] as an MN-major B;
+        # dW takes Gq [T,N] and Xq [T,K] as MN-major A and B
         for K, N in ((H, 6144), (H, H), (H, F), (F // 2, H)):
-            shapes += [(T, N, K, 0, 0), (T, K, N, 1, 0), (N, K, T, 1, 2)]
+            shapes += [(T, N, K, 0, 0, 0, 0), (T, K, N, 1, 0, 0, 1), (N, K, T, 1, 2, 1, 1)]
         ops = []
-        for M, N, Kc, af, kind in shapes:
-            ops.append((torch.randint(0, 120, (M, Kc), dtype=torch.uint8, device=dev),
-                        torch.randint(0, 120, (N, Kc), dtype=torch.uint8, device=dev),
-                        torch.zeros((M, N), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=dev), af, kind))
+        for M, N, Kc, af, kind, amn, bmn in shapes:
+            ops.append((torch.randint(0, 120, (Kc, M) if amn else (M, Kc), dtype=torch.uint8, device=dev),
+                        torch.randint(0, 120, (Kc, N) if bmn else (N, Kc), dtype=torch.uint8, device=dev),
+                        torch.zeros((M, N), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=dev), af, kind, amn, bmn))
 
         def fn():
-            for A, B, D, af, kind in ops:
-                qe.qe_gemm_fp8(A, af, B, 0, one, one, D, kind, None, status)
+            for A, B, D, af, kind, amn, bmn in ops:
+                qe.qe_gemm_fp8_ex(A, af, bool(amn), B, 0, bool(bmn), one, one, D, kind, None, status)
 
-        work = {"flop": sum(2.0 * M * N * Kc for M, N, Kc, _, _ in shapes),
-                "bytes": sum(M * Kc + N * Kc + M * N * (2 if k == 0 else 8) for M, N, Kc, _, k in shapes)}
+        work = {"flop": sum(2.0 * M * N * Kc for M, N, Kc, *_ in shapes),
+                "bytes": sum(M * Kc + N * Kc + M * N * (2 if k == 0 else 8) for M, N, Kc, _, k, _, _ in shapes)}
     elif a.case.startswith("gemm"):
         # gate/up projection: F: [T,H]x[F,H]^T ; dI: [T,F]x[H,F]^T ; dW: [F,T]x[H,T]^T (FP32 read-modify-write)
-        M, N, Kc, af, kind = {"gemm_f": (T, F, H, 0, 0), "gemm_di": (T, H, F, 1, 0), "gemm_dw": (F, H, T, 1, 2)}[a.case]
-        A = torch.randint(0, 120, (M, Kc), dtype=torch.uint8, device=dev)
-        B = torch.randint(0, 120, (N, Kc), dtype=torch.uint8, device=dev)
+        M, N, Kc, af, kind, amn, bmn = {"gemm_f": (T, F, H, 0, 0, 0, 0), "gemm_di": (T, H, F, 1, 0, 0, 1),
+                                        "gemm_dw": (F, H, T, 1, 2, 1, 1)}[a.case]
+        A = torch.randint(0, 120, (Kc, M) if amn else (M, Kc), dtype=torch.uint8, device=dev)
+        B = torch.randint(0, 120, (Kc, N) if bmn else (N, Kc), dtype=torch.uint8, device=dev)
         D = torch.zeros((M, N), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=dev)
-        fn = lambda: qe.qe_gemm_fp8(A, af, B, 0, one, one, D, kind, None, status)
+        fn = lambda: qe.qe_gemm_fp8_ex(A, af, bool(amn), B, 0, bool(bmn), one, one, D, kind, None, status)
         work = {"flop": 2.0 * M * N * Kc, "bytes": M * Kc + N * Kc + M * N * (2 if kind == 0 else 8)}
     else:
         rows, cols = 8192, 16384
