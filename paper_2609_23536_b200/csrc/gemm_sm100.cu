@@ -1,8 +1,10 @@
-// FP8 GEMM for sm_100a: D[M,N] = (A[M,Kc] . B[N,Kc]^T) * alpha, A and B contraction-major bytes (E4M3 or E5M2,
-// mixed freely), FP32 accumulation in tensor memory.
+// FP8 GEMM for sm_100a: D[M,N] = (A[M,Kc] . B[N,Kc]^T) * alpha, A and B bytes (E4M3 or E5M2, mixed freely), each
+// stored contraction-major ([rows, Kc]) or, in the paired variant, MN-major ([Kc, rows]: the transposed view of a
+// row-major tensor, read by the tensor cores directly), FP32 accumulation in tensor memory.
 //
 // Structure (one persistent CTA per SM, 320 threads):
-//   warp 0      TMA producer: cp.async.bulk.tensor 2D tiles (128-byte swizzle) into a 4-stage shared-memory ring
+//   warp 0      TMA producer: cp.async.bulk.tensor 2D tiles (128-byte swizzle) into a shared-memory ring (5 stages
+//               of 32 KB in the paired variant, 3 of 48 KB in the single-CTA one)
 //   warp 1      allocates tensor memory, then one lane issues tcgen05.mma (128 x 256 x 32 per instruction) and
 //               tcgen05.commit to release ring stages / publish a finished accumulator
 //   warps 2-9   epilogue: tcgen05.ld the 128 x 256 FP32 accumulator (two warps per 32-lane quadrant, 128 columns
@@ -18,7 +20,7 @@
 // Two variants share the code below.  The single-CTA one computes 128 x 256 tiles.  The paired one (used whenever M
 // is a multiple of 256) runs as clusters of two CTAs on neighbouring SMs that compute one 256 x 256 tile together
 // with tcgen05.mma.cta_group::2: each CTA loads its own 128 rows of A and its own 128 rows of B (32 KB per stage
-// instead of 48 KB, six stages), the even CTA issues the MMAs for the pair, tcgen05.commit multicasts stage-free and
+// instead of 48 KB), the even CTA issues the MMAs for the pair, tcgen05.commit multicasts stage-free and
 // accumulator-ready arrivals to both CTAs, and each CTA drains its own 128 accumulator rows.  That halves the
 // B-operand shared-memory traffic per SM, which is what bounds the single-CTA variant.  No TMA multicast is used.
 // Each output element is produced by exactly one thread with a fixed contraction order, so results do not depend
