@@ -43,7 +43,10 @@ constexpr uint32_t A_BYTES = BM * BK;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int MAX_STAGES = 6;
 constexpr uint32_t EPI_ROW_WORDS = 36;                       // 32 columns + 4 words of padding: conflict-free both ways
-constexpr uint32_t EPI_BUF_BYTES = 32 * EPI_ROW_WORDS * 4;    // per epilogue warp
+constexpr uint32_t EPI_BUF_BYTES = 5120;                     // per epilogue warp: the padded 32 x 36-word buffer of the
+                                                             // read-modify-write path (4608 B), or two 2 KB / one 4 KB
+                                                             // swizzled tiles that bulk stores read (1 KB-aligned)
+static_assert(32 * EPI_ROW_WORDS * 4 <= EPI_BUF_BYTES, "epilogue buffer");
 template <bool TWO>
 struct Cfg {
   static constexpr int STAGES = TWO ? 5 : 3;
@@ -150,6 +153,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Bulk tensor store of a shared-memory tile (issued by one lane), with group tracking.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {  // at most N groups may still be reading shared memory
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -219,14 +236,15 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;  // 1 KB-aligned
+  const uint32_t bar_base = epi_base + 8 * EPI_BUF_BYTES;
   // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], then tmem address + abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8 * (2 * MAX_STAGES + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8 * EPI_BUF_BYTES + 8 * (2 * MAX_STAGES + 4));
   volatile uint32_t* abort_flag = tmem_slot + 1;
   uint32_t* last_flag = tmem_slot + 2;
   uint32_t* red = tmem_slot + 4;  // 8 words for the commit's reduction
@@ -242,6 +260,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   if (threadIdx.x == 32) {  // descriptor fetch overlaps the rest of the prologue (and the predecessor's tail)
     asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
+    if (p.epi != 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmD) : "memory");
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -353,7 +372,9 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
     const uint32_t quad = (uint32_t)warp & 3u;          // tensor-memory lane quadrant this warp may read
     const uint32_t half = ((uint32_t)warp - 2u) >> 2;   // which 128 of the tile's 256 columns
     const int etid = (int)threadIdx.x - 64;
-    float* epi_buf = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + 256 + (uint32_t)(warp - 2) * EPI_BUF_BYTES);
+    float* epi_buf = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + (uint32_t)(warp - 2) * EPI_BUF_BYTES);
+    const uint32_t epi_smem = epi_base + (uint32_t)(warp - 2) * EPI_BUF_BYTES;  // same buffer, shared-space address
+    uint32_t n_groups = 0;  // bulk-store groups this warp has committed (buffer parity for the bf16 path)
     const float alpha = __fmul_rn(*p.alpha_a, *p.alpha_b);
     uint32_t acc = 0, acc_ph = 0;
     bool ok = true;
@@ -399,7 +420,50 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         if ((uint32_t)ch + 1 < nch) tmem_ld32(t_row + (ch + 1) * 32u, r[(ch + 1) & 1]);
         const uint32_t(&rc)[32] = r[ch & 1];
         float4(&oc)[8] = old[ch & 1];
-        // row-wise (lane = row) into the padded buffer
+        if (p.epi != 2) {
+          // ---- bf16 / FP32 overwrite: each lane (= row) writes its 32 columns into a swizzled shared-memory tile
+          // (conflict-free), one lane hands the 32 x 32 tile to the TMA unit, which writes full rows to global memory
+          if (p.epi == 0) {
+            const uint32_t buf = epi_smem + (n_groups & 1u) * 2048u;  // two tiles: the previous store may still read
+            if (lane == 0) tma_store_wait_read<1>();
+            __syncwarp();
+            uint32_t o[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              o[j] = pack_bf16(__fmul_rn(__uint_as_float(rc[2 * j]), alpha), __fmul_rn(__uint_as_float(rc[2 * j + 1]), alpha));
+              amax_bits = __vmaxu2(amax_bits, o[j] & 0x7fff7fffu);  // packed magnitudes of the rounded values stored
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {  // 64-byte rows, 64-byte swizzle: 16-byte chunk c of row r sits at c ^ ((r >> 1) & 3)
+              const uint32_t dst = buf + (uint32_t)lane * 64u + (((uint32_t)c ^ (((uint32_t)lane >> 1) & 3u)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[4 * c]), "r"(o[4 * c + 1]),
+                           "r"(o[4 * c + 2]), "r"(o[4 * c + 3])
+                           : "memory");
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
+          } else {
+            const uint32_t buf = epi_smem;  // one 4 KB tile
+            if (lane == 0) tma_store_wait_read<0>();
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {  // 128-byte rows, 128-byte swizzle: chunk c of row r sits at c ^ (r & 7)
+              const uint32_t dst = buf + (uint32_t)lane * 128u + (((uint32_t)c ^ ((uint32_t)lane & 7u)) << 4);
+              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
+                           "f"(__fmul_rn(__uint_as_float(rc[4 * c]), alpha)), "f"(__fmul_rn(__uint_as_float(rc[4 * c + 1]), alpha)),
+                           "f"(__fmul_rn(__uint_as_float(rc[4 * c + 2]), alpha)), "f"(__fmul_rn(__uint_as_float(rc[4 * c + 3]), alpha))
+                           : "memory");
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
+          }
+          ++n_groups;
+          continue;
+        }
+        // ---- FP32 read-modify-write: row-wise (lane = row) into the padded buffer, read back with a lane owning 4
+        // consecutive columns, add the destination values fetched earlier, store coalesced
         float4* wr = reinterpret_cast<float4*>(epi_buf + (uint32_t)lane * EPI_ROW_WORDS);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -412,32 +476,17 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         }
         __syncwarp();
         const float* rd = epi_buf + sub_row * EPI_ROW_WORDS + sub_col;
-        if (p.epi == 0) {
-          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
+        float* dst = reinterpret_cast<float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
 #pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const float4 v = *reinterpret_cast<const float4*>(rd + it * 4 * EPI_ROW_WORDS);
-            const uint32_t o0 = pack_bf16(v.x, v.y), o1 = pack_bf16(v.z, v.w);
-            // magnitude of the rounded values actually stored, as FP32 bit patterns (bf16 bits << 16)
-            amax_bits = max(amax_bits, max(max((o0 << 16) & 0x7fffffffu, o0 & 0x7fff0000u),
-                                           max((o1 << 16) & 0x7fffffffu, o1 & 0x7fff0000u)));
-            *reinterpret_cast<uint2*>(dst + (size_t)(it * 4) * p.ldo) = make_uint2(o0, o1);
-          }
-        } else {
-          float* dst = reinterpret_cast<float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
-#pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            float4 v = *reinterpret_cast<const float4*>(rd + it * 4 * EPI_ROW_WORDS);
-            if (p.epi == 2) {
-              v.x = __fadd_rn(oc[it].x, v.x);
-              v.y = __fadd_rn(oc[it].y, v.y);
-              v.z = __fadd_rn(oc[it].z, v.z);
-              v.w = __fadd_rn(oc[it].w, v.w);
-            }
-            *reinterpret_cast<float4*>(dst + (size_t)(it * 4) * p.ldo) = v;
-          }
-          if (p.epi == 2 && (uint32_t)ch + 2 < nch) load_old(ch + 2, oc);  // this block's values are consumed: refill
+        for (int it = 0; it < 8; ++it) {
+          float4 v = *reinterpret_cast<const float4*>(rd + it * 4 * EPI_ROW_WORDS);
+          v.x = __fadd_rn(oc[it].x, v.x);
+          v.y = __fadd_rn(oc[it].y, v.y);
+          v.z = __fadd_rn(oc[it].z, v.z);
+          v.w = __fadd_rn(oc[it].w, v.w);
+          *reinterpret_cast<float4*>(dst + (size_t)(it * 4) * p.ldo) = v;
         }
+        if ((uint32_t)ch + 2 < nch) load_old(ch + 2, oc);  // this block's values are consumed: refill
         __syncwarp();  // the buffer is rewritten by the next block
       }
       // accumulator drained: hand it back to the MMA warp
@@ -448,11 +497,13 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         else mbar_arrive(tempty_bar(acc));
       }
       if (p.epi == 0 && p.amax_bits) {
-        const uint32_t w = __reduce_max_sync(0xffffffffu, amax_bits);
+        // two packed bf16 magnitudes -> FP32 bit pattern of the larger
+        const uint32_t w = __reduce_max_sync(0xffffffffu, max(amax_bits & 0xffffu, amax_bits >> 16) << 16);
         if (lane == 0 && w) atomicMax(p.amax_bits, w);
       }
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
+    if (lane == 0) tma_store_wait_all();  // this warp's bulk stores have reached global memory
     if (p.commit.st) {
       // every epilogue thread of every CTA gets here (also after a timeout); the last CTA commits the scale state
       if (last_block(&p.commit.st->ticket, gridDim.x, etid, last_flag, epi_bar_sync))

@@ -70,6 +70,7 @@ struct AccumParams {
 struct GemmParams {
   CUtensorMap tmA;             // A [M, Kc] bytes, box 128 x 128, 128-byte swizzle
   CUtensorMap tmB;             // B [N, Kc] bytes, box 128 x gemm_b_box_rows(M)
+  CUtensorMap tmD;             // D [M, N] (bf16 or FP32), box 32 x 32, for the epilogue's bulk stores (epi 0 and 1)
   uint32_t M, N, Kc;
   uint32_t idesc;              // tcgen05 instruction descriptor (formats, majors, shape)
   uint32_t a_mn, b_mn;         // operand given MN-major (as [Kc, M] / [Kc, N] bytes): paired variant only
@@ -89,7 +90,7 @@ struct Launch {
   dim3 grid{1, 1, 1}, block{1, 1, 1};
   uint32_t smem = 0;
   uint32_t nbytes = 0;
-  alignas(64) unsigned char params[384];
+  alignas(64) unsigned char params[640];
   template <class P>
   void set(const P& p) {
     static_assert(sizeof(P) <= sizeof(params), "parameter block too large");

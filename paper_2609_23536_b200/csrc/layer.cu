@@ -71,6 +71,22 @@ int32_t make_map(const DeviceInfo* d, CUtensorMap* map, const void* ptr, uint64_
   return QE_OK;
 }
 
+// Tensor map over the output D [M, N] (row pitch ldo elements) for the epilogue's bulk stores: 32 x 32 boxes; bf16
+// rows of a box are 64 bytes (64-byte swizzle), FP32 rows 128 bytes (128-byte swizzle).
+int32_t make_out_map(const DeviceInfo* d, CUtensorMap* map, const void* ptr, uint64_t M, uint64_t N, uint64_t ldo,
+                     bool fp32) {
+  cuuint64_t gdim[2] = {N, M};
+  cuuint64_t gstride[1] = {ldo * (fp32 ? 4u : 2u)};
+  cuuint32_t box[2] = {32u, 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = d->encode(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                         const_cast<void*>(ptr), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         fp32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(QE_ERR_CUDA, "cuTensorMapEncodeTiled (output) failed with %d", (int)r);
+  return QE_OK;
+}
+
 uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
 bool shape_ok(uint32_t v) { return v >= 256 && v % 128 == 0 && v <= (1u << 20); }
@@ -404,6 +420,7 @@ void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe
   gp.out = y;
   gp.ldo = N;
   gp.epi = 0;
+  make_out_map(L->ctx->dev, &gp.tmD, y, T, N, N, false);
   gp.amax_bits = &L->st->pending_amax[QE_CLASS_Y];
   gp.status = &L->st->status;
   gp.commit = commit_params(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr);  // done by the GEMM's last CTA
@@ -427,6 +444,7 @@ void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::L
   gp.out = dx;
   gp.ldo = K;
   gp.epi = 0;
+  make_out_map(L->ctx->dev, &gp.tmD, dx, T, K, K, false);
   gp.amax_bits = nullptr;
   gp.status = &L->st->status;
   gp.commit = commit_params(L, 1u << QE_CLASS_G, 1, nullptr);  // backward amax/scale updated exactly once, here
@@ -450,6 +468,7 @@ void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp
   gp.ldo = K;
   gp.amax_bits = nullptr;
   gp.status = &L->st->status;
+  make_out_map(L->ctx->dev, &gp.tmD, temp ? temp : dst, N, K, K, true);  // used by the overwrite epilogue
   if (!temp) {
     gp.out = dst;  // direct placement: the epilogue reads, adds and writes the destination itself
     gp.epi = accumulate ? 2 : 1;
@@ -1128,6 +1147,7 @@ int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void*
   gp.out = d;
   gp.ldo = Nn;
   gp.epi = (int32_t)out_kind;
+  if ((st = make_out_map(dev, &gp.tmD, d, M, Nn, Nn, out_kind != 0)) != QE_OK) return st;
   gp.amax_bits = (uint32_t*)amax_dev;
   gp.status = status_dev;
   return launch_on(qe::make_gemm(gp, dev->num_sms), (cudaStream_t)stream);
