@@ -101,10 +101,12 @@ class ClockSampler:
 class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
-    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False):
+    def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False,
+                 group_dw=True):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
+        self.group_dw = group_dw and not staged
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
                               exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
@@ -169,6 +171,13 @@ class Stage:
         t_issue = time.perf_counter()
         for a, m in self.schedule:
             order = range(n) if a == "F" else range(n - 1, -1, -1)
+            if a == "dW" and self.group_dw:  # one call for the microbatch's weight gradients of all linears
+                ordl = list(order)
+                for lo in range(0, n, 16):
+                    idx = ordl[lo:lo + 16]
+                    self.qe.backward_dW_multi([self.layers[i] for i in idx], [tapes[(m, i)] for i in idx], self.grad,
+                                              [self.offsets[i] for i in idx])
+                continue
             for i in order:
                 L = self.layers[i]
                 if a == "F":
@@ -438,6 +447,8 @@ def main():
     ap.add_argument("--step-api", action="store_true",
                     help="qe_step_run: the whole step in one C call (native host loop; ONE graph per step in graph mode; dW not overlapped). "
                          "Default: one C-ABI call per action with dW overlapped on the context's second stream")
+    ap.add_argument("--no-group-dw", dest="group_dw", action="store_false",
+                    help="one qe_backward_dW call per linear instead of qe_backward_dW_multi per microbatch")
     ap.add_argument("--staged", action="store_true", help="copied-gradient comparison path: dW into a temporary, then a copy-add kernel")
     ap.add_argument("--own-stream", action="store_true", help="let the context create its own execution stream (event handoff on every action)")
     args = ap.parse_args()
@@ -470,7 +481,7 @@ def main():
 
     use_step = args.step_api
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
-                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged)
+                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw)
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:
@@ -486,7 +497,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "gradient_path": "staged copy-add" if args.staged else "direct placement", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "gradient_path": "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),

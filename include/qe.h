@@ -221,6 +221,17 @@ int32_t qe_backward_dW(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t 
  * to temp_dev (FP32 [N,K], caller-owned scratch) and then added into the destination by a second kernel. */
 int32_t qe_backward_dW_staged(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t grad_buf_elems,
                               uint64_t offset, float* temp_dev, void* caller_stream);
+/* The W action of Sec. 4.2 for several layers of the stage at once (typically one microbatch's deferred weight
+ * gradients): the same checks, results (bit for bit) and state transitions as qe_backward_dW(layers[i], &tapes[i],
+ * grad_buf_dev, grad_buf_elems, offsets[i], stream) for i = 0..n-1, but the GEMMs of up to four layers share one
+ * kernel launch where each of them can run on the paired-CTA variant (N_i a multiple of 256); the others are
+ * launched one by one inside the same call.  layers[] (host array) distinct and of one context, 1 <= n <=
+ * QE_MAX_MULTI_DW; tapes[] and offsets[] host arrays of n entries.  All n checks are made before anything runs: on
+ * a contract error nothing ran and no layer's state changed.  A bounded wait that expires inside a shared launch
+ * is recorded in the status word of the first layer of that launch. */
+#define QE_MAX_MULTI_DW 16
+int32_t qe_backward_dW_multi(qe_layer* const* layers, const qe_tape* tapes, uint32_t n, float* grad_buf_dev,
+                             uint64_t grad_buf_elems, const uint64_t* offsets, void* caller_stream);
 /* Optimizer boundary: waits for the execution stream, reads the device status word, then applies
  * qe_contract_boundary (bumping the weight version so that the next forward refreshes the cache). */
 int32_t qe_optimizer_boundary(qe_layer*, uint32_t microbatches_expected);
@@ -291,6 +302,7 @@ typedef struct qe_stats {
   uint64_t kernels_launched;   /* kernels of this library enqueued (eager launches + kernel nodes replayed)   */
   double capture_host_ms;      /* host time spent building graphs                                             */
   uint64_t workspace_bytes;    /* sum over live layers                                                        */
+  uint64_t grouped_dw;         /* weight-gradient GEMMs that shared a launch with other layers' (built launches)  */
 } qe_stats;
 int32_t qe_get_stats(const qe_ctx*, qe_stats* out);
 

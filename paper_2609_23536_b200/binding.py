@@ -97,7 +97,7 @@ class qe_stats(C.Structure):
     _fields_ = [
         ("graphs_built", C.c_uint64), ("graph_replays", C.c_uint64), ("eager_launches", C.c_uint64),
         ("handoffs", C.c_uint64), ("node_param_updates", C.c_uint64), ("kernels_launched", C.c_uint64),
-        ("capture_host_ms", C.c_double), ("workspace_bytes", C.c_uint64),
+        ("capture_host_ms", C.c_double), ("workspace_bytes", C.c_uint64), ("grouped_dw", C.c_uint64),
     ]
 
     def asdict(self):
@@ -135,6 +135,8 @@ _SIGNATURES = {
     "qe_backward_dI_host": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
+    "qe_backward_dW_multi": (C.c_int32, [C.POINTER(_P), C.POINTER(qe_tape), C.c_uint32, _P, C.c_uint64,
+                                         C.POINTER(C.c_uint64), _P]),
     "qe_step_run": (C.c_int32, [_P, C.POINTER(_P), C.c_uint32, C.POINTER(qe_step_action), C.c_uint32, C.c_uint32,
                                 C.POINTER(qe_step_io), _P, C.c_uint64, C.POINTER(C.c_uint64), _P, _P]),
     "qe_optimizer_boundary": (C.c_int32, [_P, C.c_uint32]),
@@ -465,6 +467,15 @@ def qe_noalloc_staging_elems() -> int:
 
 
 ACT = {"F": 0, "dI": 1, "dW": 2}
+
+
+def backward_dW_multi(layers, tapes, grad_buf, offsets, stream=None):
+    """qe_backward_dW_multi: the weight gradients of several layers (distinct, one context) in one call."""
+    n = len(layers)
+    hs = (_P * n)(*[L.h for L in layers])
+    ts = (qe_tape * n)(*tapes)
+    offs = (C.c_uint64 * n)(*offsets)
+    _check(lib.qe_backward_dW_multi(hs, ts, n, _ptr(grad_buf), grad_buf.numel(), offs, _stream(stream)))
 
 
 class StepPlan:

@@ -228,9 +228,35 @@ __device__ __forceinline__ void tile_coords(uint32_t tile, uint32_t tiles_m, uin
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory"); }
 
+// ------------------------------------------------------------------------------------------------ problem lookup
+// A launch computes one GEMM, or (grouped launch) up to four independent ones whose tiles are numbered one after the
+// other, so that one set of persistent CTAs packs them into common waves and the launch overhead is paid once.
+struct OneProblem {
+  const GemmParams& p;
+  __device__ __forceinline__ uint32_t total_tiles(uint32_t tile_m) const { return (p.M / tile_m) * ((p.N + BN - 1) / BN); }
+  __device__ __forceinline__ const GemmParams& at(uint32_t tile, uint32_t& local) const {
+    local = tile;
+    return p;
+  }
+  __device__ __forceinline__ const GemmParams& first() const { return p; }
+  __device__ __forceinline__ const CommitParams* commit() const { return &p.commit; }
+};
+struct ProblemGroup {
+  const GemmGroupParams& g;
+  __device__ __forceinline__ uint32_t total_tiles(uint32_t) const { return g.tile_end[g.n - 1]; }
+  __device__ __forceinline__ const GemmParams& at(uint32_t tile, uint32_t& local) const {
+    uint32_t i = 0, base = 0;
+    while (i + 1 < g.n && tile >= g.tile_end[i]) base = g.tile_end[i++];
+    local = tile - base;
+    return g.prob[i];
+  }
+  __device__ __forceinline__ const GemmParams& first() const { return g.prob[0]; }
+  __device__ __forceinline__ const CommitParams* commit() const { return nullptr; }
+};
+
 // ------------------------------------------------------------------------------------------------ kernel
-template <bool TWO>
-__device__ __forceinline__ void gemm_body(const GemmParams& p) {
+template <bool TWO, class PS>
+__device__ __forceinline__ void gemm_body(const PS& ps) {
   using C = Cfg<TWO>;
   constexpr int STAGES = C::STAGES;
   constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES;
@@ -251,16 +277,21 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = TWO ? cluster_ctarank() : 0u;  // position in the CTA pair; rank 0 issues the MMAs
-  const uint32_t tiles_m = p.M / C::TILE_M, tiles_n = (p.N + BN - 1) / BN;
-  const uint32_t num_tiles = tiles_m * tiles_n;
+  const uint32_t num_tiles = ps.total_tiles(C::TILE_M);
   const uint32_t first_tile = blockIdx.x / C::CTAS, tile_step = gridDim.x / C::CTAS;
-  const uint32_t num_kb = p.Kc / BK;
-  const bool m_fastest = p.M <= p.N;
+  uint32_t* const status = ps.first().status;
+// per tile: which problem it belongs to (`p`), its index inside that problem and the problem's tiling
+#define QE_TILE_PROBLEM()                                                                      \
+  uint32_t local_tile;                                                                         \
+  const GemmParams& p = ps.at(tile, local_tile);                                               \
+  const uint32_t tiles_m = p.M / C::TILE_M, tiles_n = (p.N + BN - 1) / BN, num_kb = p.Kc / BK; \
+  const bool m_fastest = p.M <= p.N
 
   if (threadIdx.x == 32) {  // descriptor fetch overlaps the rest of the prologue (and the predecessor's tail)
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
-    if (p.epi != 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmD) : "memory");
+    const GemmParams& q = ps.first();  // (a group's other descriptors are fetched on first use)
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&q.tmA) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&q.tmB) : "memory");
+    if (q.epi != 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&q.tmD) : "memory");
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -305,10 +336,11 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       uint32_t ph = 0;
       bool ok = true;
       for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
+        QE_TILE_PROBLEM();
         uint32_t m0, n0;
-        tile_coords(tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
+        tile_coords(local_tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
         for (uint32_t kb = 0; kb < num_kb; ++kb) {
-          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, ERR_PRODUCER))) break;
+          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status, ERR_PRODUCER))) break;
           const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_BYTES;
           if (TWO) {
             // both CTAs credit the even CTA's barrier, which expects the bytes of the whole pair
@@ -342,11 +374,13 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       uint32_t ph = 0, acc = 0, acc_ph = 0;
       bool ok = true;
       for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
-        if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, ERR_MMA))) break;
+        QE_TILE_PROBLEM();
+        (void)tiles_m; (void)tiles_n; (void)m_fastest;
+        if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, status, ERR_MMA))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * (uint32_t)BN;
         for (uint32_t kb = 0; kb < num_kb; ++kb) {
-          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, p.status, ERR_MMA))) break;
+          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, status, ERR_MMA))) break;
           tc_fence_after();
           const uint32_t a_src = smem_base + s * STAGE_BYTES, b_src = a_src + A_BYTES;
           const uint64_t adesc = make_desc(a_src), bdesc = make_desc(b_src);
@@ -375,14 +409,16 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
     float* epi_buf = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + (uint32_t)(warp - 2) * EPI_BUF_BYTES);
     const uint32_t epi_smem = epi_base + (uint32_t)(warp - 2) * EPI_BUF_BYTES;  // same buffer, shared-space address
     uint32_t n_groups = 0;  // bulk-store groups this warp has committed (buffer parity for the bf16 path)
-    const float alpha = __fmul_rn(*p.alpha_a, *p.alpha_b);
     uint32_t acc = 0, acc_ph = 0;
     bool ok = true;
     const uint32_t tempty_leader0 = TWO ? map_to_cta(tempty_bar(0), 0) : tempty_bar(0);
     const uint32_t tempty_leader1 = TWO ? map_to_cta(tempty_bar(1), 0) : tempty_bar(1);
     for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
+      QE_TILE_PROBLEM();
+      (void)num_kb;
+      const float alpha = __fmul_rn(*p.alpha_a, *p.alpha_b);
       uint32_t m0, n0;
-      tile_coords(tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
+      tile_coords(local_tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
       const uint32_t row = m0 + rank * BM + quad * 32u + (uint32_t)lane;
       const uint32_t col0 = n0 + half * 128u;
       if (p.epi == 2 && col0 < p.N) {
@@ -405,7 +441,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         if (nch > 0) load_old(0, old[0]);
         if (nch > 1) load_old(1, old[1]);
       }
-      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status, ERR_EPILOGUE))) break;
+      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, status, ERR_EPILOGUE))) break;
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN + half * 128u;
       uint32_t amax_bits = 0;
@@ -504,10 +540,11 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
     if (lane == 0) tma_store_wait_all();  // this warp's bulk stores have reached global memory
-    if (p.commit.st) {
+    const CommitParams* cm = ps.commit();
+    if (cm && cm->st) {
       // every epilogue thread of every CTA gets here (also after a timeout); the last CTA commits the scale state
-      if (last_block(&p.commit.st->ticket, gridDim.x, etid, last_flag, epi_bar_sync))
-        commit_classes(p.commit, etid, red, epi_bar_sync);
+      if (last_block(&cm->st->ticket, gridDim.x, etid, last_flag, epi_bar_sync))
+        commit_classes(*cm, etid, red, epi_bar_sync);
     }
   }
 
@@ -523,11 +560,21 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   }
 }
 
-__global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_constant__ GemmParams p) { gemm_body<false>(p); }
+#undef QE_TILE_PROBLEM
+
+__global__ void __launch_bounds__(THREADS, 1) gemm_fp8_kernel(const __grid_constant__ GemmParams p) {
+  gemm_body<false>(OneProblem{p});
+}
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
     gemm_fp8_pair_kernel(const __grid_constant__ GemmParams p) {
-  gemm_body<true>(p);
+  gemm_body<true>(OneProblem{p});
+}
+
+// Up to four independent GEMMs (each eligible for the paired variant) in one launch.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+    gemm_fp8_pair_group_kernel(const __grid_constant__ GemmGroupParams g) {
+  gemm_body<true>(ProblemGroup{g});
 }
 
 }  // namespace
@@ -548,8 +595,32 @@ cudaError_t gemm_prepare() {
   cudaError_t e = cudaFuncSetAttribute((const void*)gemm_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute((const void*)gemm_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute((const void*)gemm_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute((const void*)gemm_fp8_pair_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)SMEM_BYTES);
+}
+
+bool make_gemm_group(const GemmParams* probs, uint32_t n, int num_sms, Launch* out) {
+  if (n < 2 || n > 4) return false;
+  GemmGroupParams g{};
+  uint32_t tiles = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (!gemm_uses_pair(probs[i].M) || probs[i].commit.st) return false;  // paired variant only, no commit tail
+    tiles += (probs[i].M / 256u) * ((probs[i].N + BN - 1) / BN);
+    g.tile_end[i] = tiles;
+    g.prob[i] = probs[i];
+  }
+  g.n = n;
+  Launch l;
+  l.func = (const void*)gemm_fp8_pair_group_kernel;
+  const uint32_t ctas = 2u * tiles, cap = (uint32_t)num_sms & ~1u;
+  l.grid = dim3(ctas < cap ? ctas : cap, 1, 1);
+  l.block = dim3(THREADS, 1, 1);
+  l.smem = SMEM_BYTES;
+  l.set(g);
+  *out = l;
+  return true;
 }
 
 Launch make_gemm(const GemmParams& p, int num_sms) {

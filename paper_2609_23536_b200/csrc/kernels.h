@@ -84,13 +84,21 @@ struct GemmParams {
   CommitParams commit;         // performed by the last CTA to finish (commit.st != null)
 };
 
+// Up to four independent GEMMs computed by one launch: tiles are numbered problem after problem.
+struct GemmGroupParams {
+  uint32_t n;
+  uint32_t tile_end[4];        // cumulative tile counts (256 x 256 tiles)
+  uint32_t pad[11];
+  GemmParams prob[4];
+};
+
 // One launch, self-contained.
 struct Launch {
   const void* func = nullptr;
   dim3 grid{1, 1, 1}, block{1, 1, 1};
   uint32_t smem = 0;
   uint32_t nbytes = 0;
-  alignas(64) unsigned char params[640];
+  alignas(64) unsigned char params[2304];
   template <class P>
   void set(const P& p) {
     static_assert(sizeof(P) <= sizeof(params), "parameter block too large");
@@ -105,6 +113,9 @@ Launch make_amax_pass1(const AmaxParams& p);
 Launch make_amax_pass2(const AmaxParams& p);
 Launch make_accumulate(const AccumParams& p);
 Launch make_gemm(const GemmParams& p, int num_sms);
+// One launch for n = 2..4 GEMMs; false if the group cannot be formed (a problem needs the single-CTA variant or a
+// commit tail), in which case the caller launches them one by one.
+bool make_gemm_group(const GemmParams* probs, uint32_t n, int num_sms, Launch* out);
 cudaError_t gemm_prepare();  // opt in to the dynamic shared memory the GEMM needs (once per device)
 uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M, bool a_mn = false, bool b_mn = false);
 bool gemm_uses_pair(uint32_t M);

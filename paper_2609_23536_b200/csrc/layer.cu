@@ -451,8 +451,9 @@ void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::L
   ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
 }
 
-// dst = first element of the layer's gradient slice; temp != null selects the copied-gradient comparison path
-void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp, std::vector<qe::Launch>& ls) {
+// The weight-gradient GEMM of slot p; dst = first element of the layer's gradient slice, temp != null makes it
+// write the temporary instead (copied-gradient comparison path).
+qe::GemmParams dW_gemm(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   qe::GemmParams gp{};
   const bool mn = L->GqT[p] == nullptr;  // Gq [T,N] and Xq [T,K] themselves, read as MN-major operands
@@ -472,11 +473,17 @@ void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp
   if (!temp) {
     gp.out = dst;  // direct placement: the epilogue reads, adds and writes the destination itself
     gp.epi = accumulate ? 2 : 1;
-    ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
   } else {
     gp.out = temp;
     gp.epi = 1;
-    ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
+  }
+  return gp;
+}
+
+void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp, std::vector<qe::Launch>& ls) {
+  const uint32_t K = L->cfg.K, N = L->cfg.N;
+  ls.push_back(qe::make_gemm(dW_gemm(L, p, dst, accumulate, temp), L->ctx->dev->num_sms));
+  if (temp) {
     qe::AccumParams ap{};
     ap.dst = (float4*)dst;
     ap.src = (const float4*)temp;
@@ -485,6 +492,40 @@ void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp
     ls.push_back(qe::make_accumulate(ap));
   }
 }
+
+// Weight-gradient GEMMs of different layers that follow one another share one launch where the kernel allows it
+// (all on the paired variant): the persistent CTAs pack their tiles into common waves and the launch is paid once.
+// The layers' gradient slices are disjoint (destination registry), so the GEMMs are independent.
+struct DWBatch {
+  qe::GemmParams gp[4];
+  qe_layer* layer[4];
+  uint32_t n = 0;
+  bool has(const qe_layer* L) const {
+    for (uint32_t i = 0; i < n; ++i)
+      if (layer[i] == L) return true;
+    return false;
+  }
+  void flush(qe_ctx* ctx, std::vector<qe::Launch>& ls) {
+    qe::GemmParams paired[4];
+    uint32_t np = 0;
+    for (uint32_t i = 0; i < n; ++i)
+      if (qe::gemm_uses_pair(gp[i].M)) paired[np++] = gp[i];
+    qe::Launch l;
+    const bool grouped = np >= 2 && qe::make_gemm_group(paired, np, ctx->dev->num_sms, &l);
+    if (grouped) {
+      ls.push_back(l);
+      ctx->stats.grouped_dw += np;
+    }
+    for (uint32_t i = 0; i < n; ++i)
+      if (!grouped || !qe::gemm_uses_pair(gp[i].M)) ls.push_back(qe::make_gemm(gp[i], ctx->dev->num_sms));
+    n = 0;
+  }
+  void add(qe_ctx* ctx, qe_layer* L, const qe::GemmParams& g, std::vector<qe::Launch>& ls) {
+    if (n == 4 || has(L)) flush(ctx, ls);  // a layer's own GEMMs accumulate into one slice: never in one launch
+    gp[n] = g;
+    layer[n++] = L;
+  }
+};
 
 }  // namespace
 
@@ -767,6 +808,97 @@ int32_t qe_backward_dW_staged(qe_layer* L, const qe_tape* tape, float* grad, uin
   return backward_dW_impl(L, tape, grad, elems, off, temp, stream);
 }
 
+// Graph of a launch list identified by a hash (whole steps, multi-layer dW calls); rebuilt when the list's length
+// changed under the same key (e.g. no weight refresh this time).
+static ActionGraph* keyed_graph(qe_ctx* ctx, uint64_t key, size_t n_launches) {
+  qe_ctx::StepGraph* sg = nullptr;
+  for (auto* c : ctx->step_graphs)
+    if (c->key == key) sg = c;
+  if (sg && sg->g.launches.size() != n_launches) {
+    destroy_graph(&sg->g);
+    sg->g = ActionGraph();
+  }
+  if (!sg) {
+    sg = new (std::nothrow) qe_ctx::StepGraph();
+    if (!sg) return nullptr;
+    sg->key = key;
+    ctx->step_graphs.push_back(sg);
+  }
+  return &sg->g;
+}
+
+struct Fnv {
+  uint64_t key = 1469598103934665603ull;  // FNV-1a
+  void mix(const void* ptr, size_t n) {
+    const unsigned char* c = (const unsigned char*)ptr;
+    for (size_t i = 0; i < n; ++i) key = (key ^ c[i]) * 1099511628211ull;
+  }
+};
+
+int32_t qe_backward_dW_multi(qe_layer* const* layers, const qe_tape* tapes, uint32_t n, float* grad, uint64_t elems,
+                             const uint64_t* offsets, void* caller_stream) {
+  if (!layers || !tapes || !offsets || n == 0 || n > QE_MAX_MULTI_DW) return fail(QE_ERR_BAD_ARG, "null argument or bad count %u", n);
+  qe_ctx* ctx = layers[0] ? layers[0]->ctx : nullptr;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (!layers[i] || layers[i]->ctx != ctx) return fail(QE_ERR_BAD_ARG, "layer %u is null or belongs to another context", i);
+    for (uint32_t j = 0; j < i; ++j)
+      if (layers[j] == layers[i]) return fail(QE_ERR_BAD_ARG, "layer %u appears twice", i);
+  }
+  // check (every layer, before anything runs) -> run -> commit
+  int32_t acc[QE_MAX_MULTI_DW];
+  int32_t st;
+  for (uint32_t i = 0; i < n; ++i) {
+    const uint64_t slice = (uint64_t)layers[i]->cfg.N * layers[i]->cfg.K;
+    if ((st = qe_contract_dW_check(layers[i]->contract, &tapes[i], (uint64_t)(uintptr_t)grad, elems, offsets[i], slice, &acc[i])) != QE_OK)
+      return st;
+  }
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  cudaStream_t run_on = ctx->exec_stream;
+  if (ctx->dw_stream) {
+    run_on = ctx->dw_stream;
+    QE_CUDA(cudaEventRecord(ctx->ev_dw_in, caller));
+    QE_CUDA(cudaStreamWaitEvent(run_on, ctx->ev_dw_in, 0));
+    for (uint32_t i = 0; i < n; ++i) QE_CUDA(cudaStreamWaitEvent(run_on, layers[i]->ev_di[tapes[i].ref.slot], 0));
+    ctx->stats.handoffs += 1;
+  } else if ((st = handoff_in(ctx, caller)) != QE_OK) {
+    return st;
+  }
+  std::vector<qe::Launch> ls;
+  DWBatch dwb;
+  Fnv h;
+  h.mix("dWmulti", 8);
+  for (uint32_t i = 0; i < n; ++i) {
+    const uint32_t p = tapes[i].ref.slot;
+    dwb.add(ctx, layers[i], dW_gemm(layers[i], p, grad + offsets[i], acc[i], nullptr), ls);
+    h.mix(&layers[i], sizeof(qe_layer*));
+    h.mix(&p, sizeof(p));
+  }
+  dwb.flush(ctx, ls);
+  if (ctx->exec_mode == QE_EXEC_GRAPH) {
+    ActionGraph* g = keyed_graph(ctx, h.key, ls.size());
+    if (!g) return fail(QE_ERR_BAD_ARG, "out of host memory");
+    st = run_action(ctx, g, ls, run_on);
+  } else {
+    for (const qe::Launch& l : ls)
+      if ((st = launch_eager(ctx, l, run_on)) != QE_OK) break;
+  }
+  if (st != QE_OK) return st;
+  if (ctx->dw_stream) {
+    for (uint32_t i = 0; i < n; ++i) {
+      const uint32_t p = tapes[i].ref.slot;
+      QE_CUDA(cudaEventRecord(layers[i]->ev_dw[p], run_on));
+      layers[i]->dw_pending[p] = true;
+    }
+  } else if ((st = handoff_out(ctx, caller)) != QE_OK) {
+    return st;
+  }
+  for (uint32_t i = 0; i < n; ++i) {
+    const uint64_t slice = (uint64_t)layers[i]->cfg.N * layers[i]->cfg.K;
+    if ((st = qe_contract_dW_commit(layers[i]->contract, &tapes[i], (uint64_t)(uintptr_t)grad, offsets[i], slice)) != QE_OK) return st;
+  }
+  return QE_OK;
+}
+
 // ------------------------------------------------------------------------------------------------ whole-step call
 int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, const qe_step_action* actions,
                     uint32_t n_actions, uint32_t M, const qe_step_io* io, float* grad, uint64_t grad_elems,
@@ -785,8 +917,10 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
   ls.reserve(2 * (size_t)n_actions + n_layers);
   int32_t st = QE_OK;
   uint32_t k = 0;
+  DWBatch dwb;
   for (; k < n_actions && st == QE_OK; ++k) {
     const qe_step_action& a = actions[k];
+    if (a.kind != QE_ACT_DW && dwb.n) dwb.flush(ctx, ls);
     if (a.layer >= n_layers || a.mb >= M || a.kind > QE_ACT_DW) {
       st = fail(QE_ERR_BAD_ARG, "action %u: kind %u layer %u mb %u", k, a.kind, a.layer, a.mb);
       break;
@@ -818,10 +952,12 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
       const uint64_t slice = (uint64_t)L->cfg.N * L->cfg.K;
       int32_t acc = 0;
       if ((st = qe_contract_dW_check(L->contract, &tapes[u], (uint64_t)(uintptr_t)grad, grad_elems, offsets[a.layer], slice, &acc)) != QE_OK) break;
-      add_dW(L, tapes[u].ref.slot, grad + offsets[a.layer], acc, temp, ls);
+      if (temp) add_dW(L, tapes[u].ref.slot, grad + offsets[a.layer], acc, temp, ls);
+      else dwb.add(ctx, L, dW_gemm(L, tapes[u].ref.slot, grad + offsets[a.layer], acc, nullptr), ls);
       st = qe_contract_dW_commit(L->contract, &tapes[u], (uint64_t)(uintptr_t)grad, offsets[a.layer], slice);
     }
   }
+  if (dwb.n) dwb.flush(ctx, ls);
   const int32_t check_status = st;
   char saved_msg[512];
   std::snprintf(saved_msg, sizeof(saved_msg), "%s", qe_last_error());
@@ -839,28 +975,13 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
     }
     if (run_status == QE_OK) {
       if (ctx->exec_mode == QE_EXEC_GRAPH && check_status == QE_OK) {
-        uint64_t key = 1469598103934665603ull;  // FNV-1a over the list's identity
-        auto mix = [&key](const void* ptr, size_t n) {
-          const unsigned char* c = (const unsigned char*)ptr;
-          for (size_t i = 0; i < n; ++i) key = (key ^ c[i]) * 1099511628211ull;
-        };
-        mix(layers, sizeof(qe_layer*) * n_layers);
-        mix(actions, sizeof(qe_step_action) * n_actions);
-        mix(&M, sizeof(M));
-        qe_ctx::StepGraph* sg = nullptr;
-        for (auto* c : ctx->step_graphs)
-          if (c->key == key) sg = c;
-        if (sg && sg->g.launches.size() != ls.size()) {  // same list, different kernels (e.g. no weight refresh this time)
-          destroy_graph(&sg->g);
-          sg->g = ActionGraph();
-        }
-        if (!sg) {
-          sg = new (std::nothrow) qe_ctx::StepGraph();
-          if (!sg) return fail(QE_ERR_BAD_ARG, "out of host memory");
-          sg->key = key;
-          ctx->step_graphs.push_back(sg);
-        }
-        run_status = run_action(ctx, &sg->g, ls);
+        Fnv h;  // over the list's identity
+        h.mix(layers, sizeof(qe_layer*) * n_layers);
+        h.mix(actions, sizeof(qe_step_action) * n_actions);
+        h.mix(&M, sizeof(M));
+        ActionGraph* g = keyed_graph(ctx, h.key, ls.size());
+        if (!g) return fail(QE_ERR_BAD_ARG, "out of host memory");
+        run_status = run_action(ctx, g, ls);
       } else {
         for (const qe::Launch& l : ls)
           if ((run_status = launch_eager(ctx, l, ctx->exec_stream)) != QE_OK) break;

@@ -91,7 +91,13 @@ def test_step_call_equals_per_action_calls_bitwise(qe, mode, staged):
         assert state_equal(a, b) and a["device_token"] == b["device_token"]
     st = ctx2.stats()
     assert st["handoffs"] == 2 * 3  # one handshake pair per step instead of per action
-    n_kernels = 3 * len(SHAPES) * (M * ((2 + 2 + 2) if staged else 5) + 1)
+    if staged:
+        n_kernels = 3 * len(SHAPES) * (M * (2 + 2 + 2) + 1)
+        assert st["grouped_dw"] == 0
+    else:
+        # the dW GEMMs of the two layers whose N is a multiple of 256 share one launch per microbatch
+        n_kernels = 3 * (len(SHAPES) * (M * 4 + 1) + M * 2)
+        assert st["grouped_dw"] == 3 * M * 2
     assert st["kernels_launched"] == n_kernels
     if mode == 1:
         assert st["graphs_built"] == 1 and st["graph_replays"] == 3
@@ -118,3 +124,77 @@ def test_step_call_failure_aborts_at_the_failing_action(qe):
     for L in layers:
         L.optimizer_boundary(M)
         assert L.state()["e_W"] == 1
+
+
+MULTI_SHAPES = [(256, 512), (512, 256), (384, 384), (256, 768), (512, 512), (256, 256)]  # five of six can pair
+
+
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+@pytest.mark.parametrize("overlap", [False, True], ids=["inline", "overlapped"])
+def test_dW_multi_equals_per_layer_calls_bitwise(qe, mode, overlap):
+    """One call for a microbatch's weight gradients of all layers (shared launches) against one call per layer."""
+    T, M = 256, 3
+    n = len(MULTI_SHAPES)
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in MULTI_SHAPES])
+    results = []
+    for multi in (False, True):
+        ctx = qe.Context(mode, overlap_dw=overlap)
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, M, inputs.weights("MU", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(MULTI_SHAPES)]
+        grad = torch.full((total,), -3.0, device=DEV)
+        Y = [torch.zeros((T, N), dtype=torch.bfloat16, device=DEV) for K, N in MULTI_SHAPES]
+        dX = [torch.zeros((T, K), dtype=torch.bfloat16, device=DEV) for K, N in MULTI_SHAPES]
+        for step in range(2):
+            tapes = {}
+            for m in range(M):
+                for j, (K, N) in enumerate(MULTI_SHAPES):
+                    tapes[(j, m)] = layers[j].forward(m, step, inputs.activations("MU", 0, step, j, m, T, K).to(DEV), Y[j])
+            for m in range(M):
+                for j, (K, N) in enumerate(MULTI_SHAPES):
+                    layers[j].backward_dI(tapes[(j, m)], inputs.upstream_grads("MU", 0, step, j, m, T, N).to(DEV), dX[j])
+                if multi:
+                    qe.backward_dW_multi(layers, [tapes[(j, m)] for j in range(n)], grad, offs)
+                else:
+                    for j in range(n):
+                        layers[j].backward_dW(tapes[(j, m)], grad, offs[j])
+            for L in layers:
+                L.optimizer_boundary(M)
+        torch.cuda.synchronize()
+        results.append((grad.cpu().numpy().copy(), [L.state() for L in layers], ctx.stats()))
+    (g0, s0, st0), (g1, s1, st1) = results
+    assert np.array_equal(g0.view(np.uint32), g1.view(np.uint32))
+    assert not np.any(g1 == -3.0)  # every slice was overwritten by its first microbatch
+    for a, b in zip(s0, s1):
+        assert state_equal(a, b)
+    assert st0["grouped_dw"] == 0 and st1["grouped_dw"] == 2 * M * 5
+    # per microbatch: 4 + 1 GEMMs share two launches, the layer with N = 384 runs alone
+    assert st0["kernels_launched"] - st1["kernels_launched"] == 2 * M * (n - 3)
+
+
+def test_dW_multi_checks_every_layer_before_anything_runs(qe):
+    T = 256
+    ctx = qe.Context(0)
+    shapes = MULTI_SHAPES[:3]
+    layers = [qe.Layer(ctx, T, K, N, 4, 0, 2, inputs.weights("MV", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(shapes)]
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in shapes])
+    grad = torch.full((total,), 7.0, device=DEV)
+    tapes = []
+    for j, (K, N) in enumerate(shapes):
+        y = torch.zeros((T, N), dtype=torch.bfloat16, device=DEV)
+        dx = torch.zeros((T, K), dtype=torch.bfloat16, device=DEV)
+        tapes.append(layers[j].forward(0, 0, inputs.activations("MV", 0, 0, j, 0, T, K).to(DEV), y))
+        if j != 2:  # the last layer's tape has not had its dI yet
+            layers[j].backward_dI(tapes[j], inputs.upstream_grads("MV", 0, 0, j, 0, T, N).to(DEV), dx)
+    before = [L.state() for L in layers]
+    with pytest.raises(qe.QEError) as e:
+        qe.backward_dW_multi(layers, tapes, grad, offs)
+    assert e.value.code == "ORDER"
+    torch.cuda.synchronize()
+    assert torch.all(grad == 7.0).item()
+    for a, L in zip(before, layers):
+        assert state_equal(a, L.state())
+    with pytest.raises(qe.QEError):
+        qe.backward_dW_multi([layers[0], layers[0]], [tapes[0], tapes[0]], grad, [offs[0], offs[0]])
+    # the first two layers are still consumable
+    qe.backward_dW_multi(layers[:2], tapes[:2], grad, offs[:2])
+    torch.cuda.synchronize()
+    assert not torch.any(grad[: offs[2]] == 7.0).item() and torch.all(grad[offs[2]:] == 7.0).item()
