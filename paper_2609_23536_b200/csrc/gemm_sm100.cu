@@ -3,16 +3,20 @@
 // row-major tensor, read by the tensor cores directly), FP32 accumulation in tensor memory.
 //
 // Structure (one persistent CTA per SM, 320 threads):
-//   warp 0      TMA producer: cp.async.bulk.tensor 2D tiles (128-byte swizzle) into a shared-memory ring (5 stages
-//               of 32 KB in the paired variant, 3 of 48 KB in the single-CTA one)
+//   warp 0      TMA producer: cp.async.bulk.tensor 2D tiles (128-byte swizzle) into a shared-memory ring (6 stages
+//               of 32 KB in the paired variant, 4 of 48 KB in the single-CTA one)
 //   warp 1      allocates tensor memory, then one lane issues tcgen05.mma (128 x 256 x 32 per instruction) and
 //               tcgen05.commit to release ring stages / publish a finished accumulator
 //   warps 2-9   epilogue: tcgen05.ld the 128 x 256 FP32 accumulator (two warps per 32-lane quadrant, 128 columns
-//               each) in 32 x 32 blocks, scale, turn each block through a padded per-warp shared-memory buffer so
-//               that global accesses are coalesced (a lane owns 4 consecutive columns, a warp instruction covers
-//               four 128-byte row segments), and write bf16 (+ max|D| reduced by warp shuffles, one atomicMax per
-//               warp and tile), or FP32 overwrite, or FP32 read-modify-write straight into the destination (direct
-//               gradient placement; the destination tile is prefetched into L2 while the tile's main loop runs)
+//               each) in 32 x 32 blocks, scale, write each block into a swizzled per-warp shared-memory tile and
+//               hand it to the bulk-store unit: a bulk tensor store for bf16 (+ max|D| reduced by warp shuffles,
+//               one atomicMax per warp and tile) and for FP32 overwrite; a bulk tensor reduction (.add) for FP32
+//               accumulation straight into the destination (direct gradient placement): the addition is done in
+//               L2, one per element and launch, and the destination tile is prefetched into L2 while the tile's
+//               main loop runs.  (Like the atomic adds of this architecture the reduction flushes subnormal
+//               FP32 values to zero.)
+//   The launch may also carry up to four independent problems (grouped launch): tiles are numbered problem after
+//   problem and each role looks its tile's problem up, so that one set of persistent CTAs packs them all.
 // When asked to, the last CTA to finish folds the pending amax values into their histories and updates the scales
 // (the commit that ends F and dI), so that no extra launch is needed for it.
 // Two accumulators (2 x 256 tensor-memory columns) let the epilogue of tile i overlap the main loop of tile i+1.
@@ -23,8 +27,9 @@
 // instead of 48 KB), the even CTA issues the MMAs for the pair, tcgen05.commit multicasts stage-free and
 // accumulator-ready arrivals to both CTAs, and each CTA drains its own 128 accumulator rows.  That halves the
 // B-operand shared-memory traffic per SM, which is what bounds the single-CTA variant.  No TMA multicast is used.
-// Each output element is produced by exactly one thread with a fixed contraction order, so results do not depend
-// on the grid size or on how tiles are scheduled (no split-K, no atomics on data).
+// Each output element is produced by exactly one thread with a fixed contraction order and reaches its destination
+// by exactly one store or one addition per launch, so results do not depend on the grid size or on how tiles are
+// scheduled (no split-K; launches that add to the same destination are ordered by their stream).
 //
 // Every wait on an mbarrier is bounded by a clock budget; on expiry the thread ORs an error bit into the status
 // word, raises a CTA-wide abort flag that all other waits observe, and the CTA falls through to its common exit
@@ -42,14 +47,11 @@ constexpr int UMMA_K = 32;
 constexpr uint32_t A_BYTES = BM * BK;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int MAX_STAGES = 6;
-constexpr uint32_t EPI_ROW_WORDS = 36;                       // 32 columns + 4 words of padding: conflict-free both ways
-constexpr uint32_t EPI_BUF_BYTES = 5120;                     // per epilogue warp: the padded 32 x 36-word buffer of the
-                                                             // read-modify-write path (4608 B), or two 2 KB / one 4 KB
-                                                             // swizzled tiles that bulk stores read (1 KB-aligned)
-static_assert(32 * EPI_ROW_WORDS * 4 <= EPI_BUF_BYTES, "epilogue buffer");
+constexpr uint32_t EPI_BUF_BYTES = 4096;                     // per epilogue warp: one FP32 or two bf16 32 x 32 output tiles
+                                                             // (1 KB-aligned, swizzled) that the bulk-store unit reads
 template <bool TWO>
 struct Cfg {
-  static constexpr int STAGES = TWO ? 5 : 3;
+  static constexpr int STAGES = TWO ? 6 : 4;
   static constexpr uint32_t B_ROWS = TWO ? 128 : 256;  // rows of B this CTA loads per stage
   static constexpr uint32_t B_BYTES = B_ROWS * BK;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
@@ -59,8 +61,8 @@ struct Cfg {
 constexpr int THREADS = 320;
 constexpr int EPI_WARPS = 8, EPI_THREADS = EPI_WARPS * 32;
 static_assert(EPI_WARPS == 8, "shared-memory budget below assumes 8 epilogue warps");
-constexpr uint32_t SMEM_BYTES = 5 * (A_BYTES + 128 * BK) + 1024 /*alignment slack*/ + 256 /*barriers, flags*/ +
-                                8 * EPI_BUF_BYTES;  // 160 KB of stages (144 KB for the single-CTA variant)
+constexpr uint32_t SMEM_BYTES = 6 * (A_BYTES + 128 * BK) + 1024 /*alignment slack*/ + 256 /*barriers, flags*/ +
+                                8 * EPI_BUF_BYTES;  // 192 KB of stages in either variant
 constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;  // ~2 s at the maximum SM clock
 
 constexpr uint32_t ERR_PRODUCER = 1u, ERR_MMA = 2u, ERR_EPILOGUE = 4u;
@@ -156,6 +158,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 // Bulk tensor store of a shared-memory tile (issued by one lane), with group tracking.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Bulk tensor reduction: global tile += shared-memory tile, added element by element where the data lives (L2).
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(c0), "r"(c1), "r"(src)
                : "memory");
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -291,7 +300,7 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
     const GemmParams& q = ps.first();  // (a group's other descriptors are fetched on first use)
     asm volatile("prefetch.tensormap [%0];" ::"l"(&q.tmA) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&q.tmB) : "memory");
-    if (q.epi != 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&q.tmD) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&q.tmD) : "memory");
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -406,9 +415,8 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
     const uint32_t quad = (uint32_t)warp & 3u;          // tensor-memory lane quadrant this warp may read
     const uint32_t half = ((uint32_t)warp - 2u) >> 2;   // which 128 of the tile's 256 columns
     const int etid = (int)threadIdx.x - 64;
-    float* epi_buf = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + (uint32_t)(warp - 2) * EPI_BUF_BYTES);
-    const uint32_t epi_smem = epi_base + (uint32_t)(warp - 2) * EPI_BUF_BYTES;  // same buffer, shared-space address
-    uint32_t n_groups = 0;  // bulk-store groups this warp has committed (buffer parity for the bf16 path)
+    const uint32_t epi_smem = epi_base + (uint32_t)(warp - 2) * EPI_BUF_BYTES;  // this warp's two output tiles
+    uint32_t n_groups = 0;  // bulk-store groups this warp has committed (buffer parity)
     uint32_t acc = 0, acc_ph = 0;
     bool ok = true;
     const uint32_t tempty_leader0 = TWO ? map_to_cta(tempty_bar(0), 0) : tempty_bar(0);
@@ -422,31 +430,21 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
       const uint32_t row = m0 + rank * BM + quad * 32u + (uint32_t)lane;
       const uint32_t col0 = n0 + half * 128u;
       if (p.epi == 2 && col0 < p.N) {
-        // read-modify-write: pull this thread's 512 destination bytes towards L2 while the MMAs of the tile run
+        // accumulate: pull this thread's 512 destination bytes into L2, where the reduction will add to them, while
+        // the MMAs of the tile run
         const char* d = reinterpret_cast<const char*>(reinterpret_cast<const float*>(p.out) + (size_t)row * p.ldo + col0);
 #pragma unroll
         for (int j = 0; j < 4; ++j) asm volatile("prefetch.global.L2 [%0];" ::"l"(d + 128 * j));
       }
-      // coalesced view of a 32 x 32 block: this lane owns columns 4*(lane%8)..+3 of rows it*4 + lane/8, it = 0..7
-      const uint32_t blk_row0 = m0 + rank * BM + quad * 32u, sub_row = (uint32_t)lane >> 3, sub_col = ((uint32_t)lane & 7u) * 4u;
+      const uint32_t blk_row0 = m0 + rank * BM + quad * 32u;
       const uint32_t nch = col0 >= p.N ? 0u : min(4u, (p.N - col0) / 32u);  // ragged last column tile; warp-uniform
       uint32_t r[2][32];
-      float4 old[2][8];  // destination values are fetched two blocks ahead (they do not depend on the accumulator)
-      auto load_old = [&](int ch, float4(&o)[8]) {
-        const float* src = reinterpret_cast<const float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col0 + ch * 32u + sub_col;
-#pragma unroll
-        for (int it = 0; it < 8; ++it) o[it] = *reinterpret_cast<const float4*>(src + (size_t)(it * 4) * p.ldo);
-      };
-      if (p.epi == 2) {  // the first two blocks' destination values travel while the tile's MMAs still run
-        if (nch > 0) load_old(0, old[0]);
-        if (nch > 1) load_old(1, old[1]);
-      }
       if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, status, ERR_EPILOGUE))) break;
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((quad * 32u) << 16) + acc * (uint32_t)BN + half * 128u;
       uint32_t amax_bits = 0;
-      // Software pipeline over the warp's four 32 x 32 blocks: the tensor-memory load and (for the read-modify-
-      // write) the destination loads of block ch+1 are in flight while block ch is scaled, turned and written.
+      // Software pipeline over the warp's four 32 x 32 blocks: the tensor-memory load of block ch+1 is in flight
+      // while block ch is scaled, written to shared memory and handed to the bulk-store unit.
       if (nch) tmem_ld32(t_row, r[0]);
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
@@ -455,75 +453,51 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
         tmem_ld_wait();
         if ((uint32_t)ch + 1 < nch) tmem_ld32(t_row + (ch + 1) * 32u, r[(ch + 1) & 1]);
         const uint32_t(&rc)[32] = r[ch & 1];
-        float4(&oc)[8] = old[ch & 1];
-        if (p.epi != 2) {
-          // ---- bf16 / FP32 overwrite: each lane (= row) writes its 32 columns into a swizzled shared-memory tile
-          // (conflict-free), one lane hands the 32 x 32 tile to the TMA unit, which writes full rows to global memory
-          if (p.epi == 0) {
-            const uint32_t buf = epi_smem + (n_groups & 1u) * 2048u;  // two tiles: the previous store may still read
-            if (lane == 0) tma_store_wait_read<1>();
-            __syncwarp();
-            uint32_t o[16];
+        // Each lane (= row) writes its 32 columns into a swizzled shared-memory tile (conflict-free); one lane hands
+        // the 32 x 32 tile to the bulk-store unit, which writes full rows to global memory (bf16, FP32 overwrite) or
+        // adds them to the destination where it lives, in L2 (FP32 accumulate: one addition per element and launch).
+        if (p.epi == 0) {
+          const uint32_t buf = epi_smem + (n_groups & 1u) * 2048u;  // two tiles: the previous store may still read
+          if (lane == 0) tma_store_wait_read<1>();
+          __syncwarp();
+          uint32_t o[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              o[j] = pack_bf16(__fmul_rn(__uint_as_float(rc[2 * j]), alpha), __fmul_rn(__uint_as_float(rc[2 * j + 1]), alpha));
-              amax_bits = __vmaxu2(amax_bits, o[j] & 0x7fff7fffu);  // packed magnitudes of the rounded values stored
-            }
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {  // 64-byte rows, 64-byte swizzle: 16-byte chunk c of row r sits at c ^ ((r >> 1) & 3)
-              const uint32_t dst = buf + (uint32_t)lane * 64u + (((uint32_t)c ^ (((uint32_t)lane >> 1) & 3u)) << 4);
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[4 * c]), "r"(o[4 * c + 1]),
-                           "r"(o[4 * c + 2]), "r"(o[4 * c + 3])
-                           : "memory");
-            }
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
-          } else {
-            const uint32_t buf = epi_smem;  // one 4 KB tile
-            if (lane == 0) tma_store_wait_read<0>();
-            __syncwarp();
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {  // 128-byte rows, 128-byte swizzle: chunk c of row r sits at c ^ (r & 7)
-              const uint32_t dst = buf + (uint32_t)lane * 128u + (((uint32_t)c ^ ((uint32_t)lane & 7u)) << 4);
-              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
-                           "f"(__fmul_rn(__uint_as_float(rc[4 * c]), alpha)), "f"(__fmul_rn(__uint_as_float(rc[4 * c + 1]), alpha)),
-                           "f"(__fmul_rn(__uint_as_float(rc[4 * c + 2]), alpha)), "f"(__fmul_rn(__uint_as_float(rc[4 * c + 3]), alpha))
-                           : "memory");
-            }
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
+          for (int j = 0; j < 16; ++j) {
+            o[j] = pack_bf16(__fmul_rn(__uint_as_float(rc[2 * j]), alpha), __fmul_rn(__uint_as_float(rc[2 * j + 1]), alpha));
+            amax_bits = __vmaxu2(amax_bits, o[j] & 0x7fff7fffu);  // packed magnitudes of the rounded values stored
           }
-          ++n_groups;
-          continue;
-        }
-        // ---- FP32 read-modify-write: row-wise (lane = row) into the padded buffer, read back with a lane owning 4
-        // consecutive columns, add the destination values fetched earlier, store coalesced
-        float4* wr = reinterpret_cast<float4*>(epi_buf + (uint32_t)lane * EPI_ROW_WORDS);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          float4 v;
-          v.x = __fmul_rn(__uint_as_float(rc[4 * j]), alpha);
-          v.y = __fmul_rn(__uint_as_float(rc[4 * j + 1]), alpha);
-          v.z = __fmul_rn(__uint_as_float(rc[4 * j + 2]), alpha);
-          v.w = __fmul_rn(__uint_as_float(rc[4 * j + 3]), alpha);
-          wr[j] = v;
-        }
-        __syncwarp();
-        const float* rd = epi_buf + sub_row * EPI_ROW_WORDS + sub_col;
-        float* dst = reinterpret_cast<float*>(p.out) + (size_t)(blk_row0 + sub_row) * p.ldo + col + sub_col;
+          for (int c = 0; c < 4; ++c) {  // 64-byte rows, 64-byte swizzle: 16-byte chunk c of row r sits at c ^ ((r >> 1) & 3)
+            const uint32_t dst = buf + (uint32_t)lane * 64u + (((uint32_t)c ^ (((uint32_t)lane >> 1) & 3u)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[4 * c]), "r"(o[4 * c + 1]),
+                         "r"(o[4 * c + 2]), "r"(o[4 * c + 3])
+                         : "memory");
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
+        } else {
+          // one tile: waiting for the previous block's store to have read it paces the FP32 traffic, which measured
+          // faster than two tiles in flight per warp
+          const uint32_t buf = epi_smem;
+          if (lane == 0) tma_store_wait_read<0>();
+          __syncwarp();
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          float4 v = *reinterpret_cast<const float4*>(rd + it * 4 * EPI_ROW_WORDS);
-          v.x = __fadd_rn(oc[it].x, v.x);
-          v.y = __fadd_rn(oc[it].y, v.y);
-          v.z = __fadd_rn(oc[it].z, v.z);
-          v.w = __fadd_rn(oc[it].w, v.w);
-          *reinterpret_cast<float4*>(dst + (size_t)(it * 4) * p.ldo) = v;
+          for (int c = 0; c < 8; ++c) {  // 128-byte rows, 128-byte swizzle: chunk c of row r sits at c ^ (r & 7)
+            const uint32_t dst = buf + (uint32_t)lane * 128u + (((uint32_t)c ^ ((uint32_t)lane & 7u)) << 4);
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
+                         "f"(__fmul_rn(__uint_as_float(rc[4 * c]), alpha)), "f"(__fmul_rn(__uint_as_float(rc[4 * c + 1]), alpha)),
+                         "f"(__fmul_rn(__uint_as_float(rc[4 * c + 2]), alpha)), "f"(__fmul_rn(__uint_as_float(rc[4 * c + 3]), alpha))
+                         : "memory");
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (p.epi == 2) tma_reduce_add_2d(&p.tmD, buf, (int)col, (int)blk_row0);
+            else tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
+          }
         }
-        if ((uint32_t)ch + 2 < nch) load_old(ch + 2, oc);  // this block's values are consumed: refill
-        __syncwarp();  // the buffer is rewritten by the next block
+        ++n_groups;
       }
       // accumulator drained: hand it back to the MMA warp
       tc_fence_before();

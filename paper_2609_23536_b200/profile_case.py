@@ -49,7 +49,7 @@ def main():
         work = {"flop": sum(2.0 * M * N * Kc for M, N, Kc, *_ in shapes),
                 "bytes": sum(M * Kc + N * Kc + M * N * (2 if k == 0 else 8) for M, N, Kc, _, k, _, _ in shapes)}
     elif a.case.startswith("gemm"):
-        # gate/up projection: F: [T,H]x[F,H]^T ; dI: [T,F]x[H,F]^T ; dW: [F,T]x[H,T]^T (FP32 read-modify-write)
+        # gate/up projection: F: [T,H]x[F,H]^T ; dI: [T,F]x[H,F]^T ; dW: [F,T]x[H,T]^T (FP32 accumulate)
         M, N, Kc, af, kind, amn, bmn = {"gemm_f": (T, F, H, 0, 0, 0, 0), "gemm_di": (T, H, F, 1, 0, 0, 1),
                                         "gemm_dw": (F, H, T, 1, 2, 1, 1)}[a.case]
         A = torch.randint(0, 120, (Kc, M) if amn else (M, Kc), dtype=torch.uint8, device=dev)
