@@ -203,12 +203,13 @@ int32_t qe_forward(qe_layer*, uint32_t mb, uint64_t gen, const void* x_dev, void
  * dW), dX = bf16((Gq Wq) * sinv_G * sinv_W), commits the gradient amax/scale once. */
 int32_t qe_backward_dI(qe_layer*, const qe_tape*, const void* dy_dev, void* dx_dev, void* caller_stream);
 /* F and dI with HOST buffers (layer created with host_io = 1).  The input is copied host-to-device into the layer's
- * fixed staging buffer on the execution stream after the caller->execution edge (the dynamic-input copy of Sec. 4.4),
- * the action runs on the staging buffers -- in graph mode the graph's addresses therefore never change -- and the output
- * is copied device-to-host before the execution->caller edge, so it is complete for work the caller queues after the
- * call (or after synchronising caller_stream on the host).  Pinned host memory makes the copies asynchronous; y_host /
- * dx_host may be NULL to skip the read-back.  Same checks, state transitions and results as qe_forward /
- * qe_backward_dI. */
+ * fixed staging buffer after the caller->execution edge (the dynamic-input copy of Sec. 4.4), the action runs on
+ * the staging buffers -- in graph mode the graph's addresses therefore never change -- and the output is copied
+ * device-to-host before the execution->caller edge, so it is complete for work the caller queues after the call (or
+ * after synchronising caller_stream on the host).  The two copies run on copy streams of the context, ordered with
+ * the execution stream by events: the upload of a call overlaps the read-back of the call before it (the host link
+ * is full duplex), the kernels wait for both.  Pinned host memory makes the copies asynchronous; y_host / dx_host
+ * may be NULL to skip the read-back.  Same checks, state transitions and results as qe_forward / qe_backward_dI. */
 int32_t qe_forward_host(qe_layer*, uint32_t mb, uint64_t gen, const void* x_host, void* y_host, void* caller_stream,
                         qe_tape* tape_out);
 int32_t qe_backward_dI_host(qe_layer*, const qe_tape*, const void* dy_host, void* dx_host, void* caller_stream);

@@ -111,6 +111,10 @@ struct qe_ctx {
   cudaStream_t dw_stream = nullptr;  // only with QE_CTX_OVERLAP_DW
   cudaEvent_t ev_dw_in = nullptr;
   cudaEvent_t ev_in = nullptr, ev_out = nullptr;
+  // host-buffer calls: copy streams and their events, created by the first such call
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_h2d = nullptr, ev_kernels = nullptr, ev_d2h = nullptr;
+  bool kernels_recorded = false;
   qe_registry* registry = nullptr;
   qe_stats stats{};
   // Layers keep their context alive: it is released when the caller has destroyed it AND its last layer is gone,
@@ -135,6 +139,15 @@ static void ctx_release(qe_ctx* c) {
     cudaStreamSynchronize(c->dw_stream);
     cudaStreamDestroy(c->dw_stream);
     cudaEventDestroy(c->ev_dw_in);
+  }
+  if (c->h2d_stream) {
+    cudaStreamSynchronize(c->h2d_stream);
+    cudaStreamSynchronize(c->d2h_stream);
+    cudaStreamDestroy(c->h2d_stream);
+    cudaStreamDestroy(c->d2h_stream);
+    cudaEventDestroy(c->ev_h2d);
+    cudaEventDestroy(c->ev_kernels);
+    cudaEventDestroy(c->ev_d2h);
   }
   cudaEventDestroy(c->ev_in);
   cudaEventDestroy(c->ev_out);
@@ -294,6 +307,39 @@ int32_t handoff_out(qe_ctx* ctx, cudaStream_t caller) {
   QE_CUDA(cudaEventRecord(ctx->ev_out, ctx->exec_stream));
   QE_CUDA(cudaStreamWaitEvent(caller, ctx->ev_out, 0));
   ctx->stats.handoffs += 1;
+  return QE_OK;
+}
+
+// ---- host-buffer calls.  The upload of an action runs on one copy stream and the read-back of its result on
+// another, so that the upload of action k+1 overlaps the read-back of action k (the host link is full duplex); the
+// kernels stay on the execution stream, which waits for the upload before them and for the read-back after them
+// (a caller that synchronises after the call finds its host buffer complete).
+int32_t host_upload(qe_ctx* ctx, void* dst, const void* src_host, size_t bytes, cudaStream_t caller) {
+  if (!ctx->h2d_stream) {
+    cudaError_t e = cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_h2d, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_kernels, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_d2h, cudaEventDisableTiming);
+    if (e != cudaSuccess) return fail(QE_ERR_CUDA, "copy streams: %s", cudaGetErrorString(e));
+  }
+  // the staging buffer was last read by the kernels of an earlier host-buffer call
+  if (ctx->kernels_recorded) QE_CUDA(cudaStreamWaitEvent(ctx->h2d_stream, ctx->ev_kernels, 0));
+  if (caller != ctx->exec_stream) QE_CUDA(cudaStreamWaitEvent(ctx->h2d_stream, ctx->ev_in, 0));  // recorded by handoff_in
+  QE_CUDA(cudaMemcpyAsync(dst, src_host, bytes, cudaMemcpyHostToDevice, ctx->h2d_stream));
+  QE_CUDA(cudaEventRecord(ctx->ev_h2d, ctx->h2d_stream));
+  QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_h2d, 0));
+  return QE_OK;
+}
+// after the action's kernels: frees the staging input for the next upload and starts the read-back (if any)
+int32_t host_download(qe_ctx* ctx, void* dst_host, const void* src, size_t bytes) {
+  QE_CUDA(cudaEventRecord(ctx->ev_kernels, ctx->exec_stream));
+  ctx->kernels_recorded = true;
+  if (!dst_host) return QE_OK;
+  QE_CUDA(cudaStreamWaitEvent(ctx->d2h_stream, ctx->ev_kernels, 0));
+  QE_CUDA(cudaMemcpyAsync(dst_host, src, bytes, cudaMemcpyDeviceToHost, ctx->d2h_stream));
+  QE_CUDA(cudaEventRecord(ctx->ev_d2h, ctx->d2h_stream));
+  QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_d2h, 0));
   return QE_OK;
 }
 
@@ -699,8 +745,7 @@ static int32_t forward_impl(qe_layer* L, uint32_t mb, uint64_t gen, const void* 
   cudaStream_t caller = (cudaStream_t)caller_stream;
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
-  if (x_host)  // dynamic-input copy, after the caller -> execution edge
-    QE_CUDA(cudaMemcpyAsync(const_cast<void*>(x), x_host, 2ull * T * K, cudaMemcpyHostToDevice, ctx->exec_stream));
+  if (x_host && (st = host_upload(ctx, const_cast<void*>(x), x_host, 2ull * T * K, caller)) != QE_OK) return st;
   if (L->dw_pending[p]) {  // the slot's buffers are still being read by the dW that released it (other stream)
     QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[p], 0));
     L->dw_pending[p] = false;
@@ -713,7 +758,7 @@ static int32_t forward_impl(qe_layer* L, uint32_t mb, uint64_t gen, const void* 
   std::vector<qe::Launch> ls;
   add_forward(L, p, x, y, ls);
   if ((st = run_action(ctx, &L->gF[p], ls)) != QE_OK) return st;  // ... run ...
-  if (y_host) QE_CUDA(cudaMemcpyAsync(y_host, y, 2ull * T * N, cudaMemcpyDeviceToHost, ctx->exec_stream));
+  if (x_host && (st = host_download(ctx, y_host, y, 2ull * T * N)) != QE_OK) return st;
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
   return qe_contract_forward_commit(L->contract, mb, tape_out);  // ... commit
 }
@@ -740,13 +785,12 @@ static int32_t backward_dI_impl(qe_layer* L, const qe_tape* tape, const void* dy
   cudaStream_t caller = (cudaStream_t)caller_stream;
   const uint32_t p = tape->ref.slot, T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
-  if (dy_host)
-    QE_CUDA(cudaMemcpyAsync(const_cast<void*>(dy), dy_host, 2ull * T * N, cudaMemcpyHostToDevice, ctx->exec_stream));
+  if (dy_host && (st = host_upload(ctx, const_cast<void*>(dy), dy_host, 2ull * T * N, caller)) != QE_OK) return st;
   std::vector<qe::Launch> ls;
   add_dI(L, p, dy, dx, ls);
   if ((st = run_action(ctx, &L->gDI[p], ls)) != QE_OK) return st;
   if (ctx->dw_stream) QE_CUDA(cudaEventRecord(L->ev_di[p], ctx->exec_stream));
-  if (dx_host) QE_CUDA(cudaMemcpyAsync(dx_host, dx, 2ull * T * K, cudaMemcpyDeviceToHost, ctx->exec_stream));
+  if (dy_host && (st = host_download(ctx, dx_host, dx, 2ull * T * K)) != QE_OK) return st;
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
   return qe_contract_dI_commit(L->contract, tape);
 }
