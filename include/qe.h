@@ -216,7 +216,7 @@ int32_t qe_backward_dI_host(qe_layer*, const qe_tape*, const void* dy_host, void
 /* dW (Eq. 5) with direct gradient placement (Sec. 3.4).  D = (Gq^T Xq) * sinv_G * sinv_X using the inverse scales
  * snapshotted in the tape; grad_buf_dev[offset + n*K + k] = D (first write of the epoch) or += D (FP32, in place:
  * one round-to-nearest addition per element and call, performed in L2 by a bulk tensor reduction, subnormal values
- * flushed to zero; deterministic, calls ordered by the stream).  No staging copy, no scale-state change. */
+ * kept; deterministic, calls ordered by the stream).  No staging copy, no scale-state change. */
 int32_t qe_backward_dW(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t grad_buf_elems, uint64_t offset,
                        void* caller_stream);
 /* The copied-gradient comparison path of Sec. 3.4: same checks and the same final values, but D is first written

@@ -13,8 +13,7 @@
 //               one atomicMax per warp and tile) and for FP32 overwrite; a bulk tensor reduction (.add) for FP32
 //               accumulation straight into the destination (direct gradient placement): the addition is done in
 //               L2, one per element and launch, and the destination tile is prefetched into L2 while the tile's
-//               main loop runs.  (Like the atomic adds of this architecture the reduction flushes subnormal
-//               FP32 values to zero.)
+//               main loop runs.  The reduction is a plain round-to-nearest FP32 addition (subnormal values kept).
 //   The launch may also carry up to four independent problems (grouped launch): tiles are numbered problem after
 //   problem and each role looks its tile's problem up, so that one set of persistent CTAs packs them all.
 // When asked to, the last CTA to finish folds the pending amax values into their histories and updates the scales

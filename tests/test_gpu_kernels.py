@@ -144,6 +144,23 @@ def test_gemm_integer_inputs_are_bit_exact(qe, M, Nn, Kc):
     assert np.array_equal(Dacc.numpy(), init.numpy() + want.astype(np.float32))
 
 
+def test_gemm_accumulate_keeps_subnormals(qe):
+    # the in-place accumulate is a plain round-to-nearest FP32 addition like the oracle's: subnormal destination
+    # values and subnormal addends are kept, not flushed to zero
+    M, Nn, Kc = 256, 256, 128
+    ones = np.full((M, Kc), 0x38, dtype=np.uint8)  # E4M3 1.0: every dot product is 128
+    init = torch.full((M, Nn), 1e-40)
+    init[0, 0], init[0, 1], init[0, 2] = -1e-40, 1.5, 2e-38
+    tiny = 1e-21  # alpha = 1e-42 in FP32 (subnormal), D = 128 * alpha (subnormal)
+    alpha = np.float32(np.float32(tiny) * np.float32(tiny))
+    want = init.numpy() + np.float32(128.0) * alpha
+    assert 0 < abs(want[1, 1]) < 1.2e-38
+    got, _ = _run_gemm(qe, ones, 0, np.full((Nn, Kc), 0x38, dtype=np.uint8), 0, tiny, tiny, 2, init)
+    assert np.array_equal(got.numpy().view(np.uint32), want.view(np.uint32))
+    zero, _ = _run_gemm(qe, np.zeros((M, Kc), dtype=np.uint8), 0, np.zeros((Nn, Kc), dtype=np.uint8), 0, 1.0, 1.0, 2, init)
+    assert np.array_equal(zero.numpy().view(np.uint32), init.numpy().view(np.uint32))
+
+
 def test_gemm_permutation_weight_moves_columns(qe):
     rng = np.random.default_rng(1)
     M, K = 256, 512
