@@ -198,3 +198,97 @@ def test_dW_multi_checks_every_layer_before_anything_runs(qe):
     qe.backward_dW_multi(layers[:2], tapes[:2], grad, offs[:2])
     torch.cuda.synchronize()
     assert not torch.any(grad[: offs[2]] == 7.0).item() and torch.all(grad[offs[2]:] == 7.0).item()
+
+
+# ------------------------------------------------------------------------------------------ two local chunks
+CHUNK_SHAPES = [[(256, 512), (512, 256)], [(256, 256), (256, 384)]]  # chunk -> its linears (K, N)
+
+
+def _chunk_actions(s, chunk_layers):
+    """(kind, mb, chunk) -> one action per linear of the chunk: forward in order, backward in reverse."""
+    out = []
+    for a, m, c in s:
+        ls = chunk_layers[c]
+        for l in (ls if a == "F" else reversed(ls)):
+            out.append((a, l, m))
+    return out
+
+
+@pytest.mark.parametrize("gen", ["interleaved", "zb_v"])
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_two_chunk_schedules_split_equals_full_and_match_the_oracle(qe, gen, mode):
+    """Two model chunks on the device, each with its own tape pools (Sec. 4.2): the interleaved and V-shaped orders
+    through the whole-step call, against the same F/dI order with immediate dW (bitwise) and against the oracle."""
+    from oracle.layer import OracleLinear
+    from harness import assert_gemm_close, assert_grad_close, state_equal_except_Y
+    from paper_2609_23536_b200.schedules import full_backward_chunks, interleaved_1f1b, peak_live_per_chunk, zb_v
+
+    T, M, steps = 256, 4, 2
+    s = interleaved_1f1b(M, 2, 0, 2, defer=2) if gen == "interleaved" else zb_v(M, 2, 0)
+    flat = [kn for ch in CHUNK_SHAPES for kn in ch]
+    chunk_layers, i = [], 0
+    for ch in CHUNK_SHAPES:
+        chunk_layers.append(list(range(i, i + len(ch))))
+        i += len(ch)
+    chunk_of = [c for c, ls in enumerate(chunk_layers) for _ in ls]
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in flat])
+    P = peak_live_per_chunk(s)
+
+    def tensors(step):
+        X = [[inputs.activations("CK", step, 0, j, m, T, K) for j, (K, N) in enumerate(flat)] for m in range(M)]
+        dY = [[inputs.upstream_grads("CK", step, 0, j, m, T, N) for j, (K, N) in enumerate(flat)] for m in range(M)]
+        return X, dY
+
+    def run_gpu(schedule):
+        ctx = qe.Context(mode)
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, P[chunk_of[j]], inputs.weights("CK", 0, j, N, K).to(DEV), unit=j)
+                  for j, (K, N) in enumerate(flat)]
+        grad = torch.full((total,), 2.0, device=DEV)
+        outs = []
+        for step in range(steps):
+            Xh, dYh = tensors(step)
+            X = [[t.to(DEV) for t in row] for row in Xh]
+            dY = [[t.to(DEV) for t in row] for row in dYh]
+            Y = [[torch.zeros((T, N), dtype=torch.bfloat16, device=DEV) for K, N in flat] for m in range(M)]
+            dX = [[torch.zeros((T, K), dtype=torch.bfloat16, device=DEV) for K, N in flat] for m in range(M)]
+            qe.StepPlan(ctx, layers, _chunk_actions(schedule, chunk_layers), M, X, Y, dY, dX, grad, offs).run()
+            for L in layers:
+                L.optimizer_boundary(M)
+            torch.cuda.synchronize()
+            outs.append(([[inputs.bits(t.cpu()) for t in row] for row in Y], [[inputs.bits(t.cpu()) for t in row] for row in dX],
+                         grad.cpu().numpy().copy()))
+        return outs, [L.state() for L in layers]
+
+    got, st = run_gpu(s)
+    full, st_full = run_gpu(full_backward_chunks(s))
+    for (Y, dX, g), (Y2, dX2, g2) in zip(got, full):
+        for m in range(M):
+            for j in range(len(flat)):
+                assert np.array_equal(Y[m][j], Y2[m][j]) and np.array_equal(dX[m][j], dX2[m][j])
+        assert np.array_equal(g.view(np.uint32), g2.view(np.uint32))
+    for a, b in zip(st, st_full):
+        assert state_equal({**a, "slots": []}, {**b, "slots": []})
+
+    # the oracle, driven by the same two-chunk order
+    orc = [OracleLinear(T, K, N, 4, 0, P[chunk_of[j]], stage=0, unit=j) for j, (K, N) in enumerate(flat)]
+    for j, (K, N) in enumerate(flat):
+        orc[j].set_weight(inputs.bits(inputs.weights("CK", 0, j, N, K)))
+    buf = np.full(total, 2.0, np.float32)
+    for step in range(steps):
+        Xh, dYh = tensors(step)
+        tapes = {}
+        for a, l, m in _chunk_actions(s, chunk_layers):
+            L = orc[l]
+            if a == "F":
+                tapes[(l, m)], Yo = L.forward(m, L.e_W, inputs.bits(Xh[m][l]))
+                assert_gemm_close(got[step][0][m][l], Yo, f"Y step {step} linear {l} mb {m}")
+            elif a == "dI":
+                dXo = L.backward_dI(tapes[(l, m)], inputs.bits(dYh[m][l]))
+                assert_gemm_close(got[step][1][m][l], dXo, f"dX step {step} linear {l} mb {m}")
+            else:
+                L.backward_dW(tapes[(l, m)], buf, offs[l])
+        assert_grad_close(got[step][2], buf, f"main_grad step {step}")
+        for L in orc:
+            L.optimizer_boundary(M)
+    for a, L in zip(st, orc):
+        assert state_equal_except_Y(a, L.state())
