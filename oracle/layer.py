@@ -287,6 +287,71 @@ class OracleLinear:
         s.bits |= DW_BIT
         s.live, s.Xq, s.Gq = False, None, None  # both bits set: release, generation kept
 
+    # ------------------------------------------------------------------ per-microbatch arena (Sec. 3.4, Eq. for A_r)
+    def backward_dW_arena(self, tape: Tape, arena: np.ndarray, layer_off: int, microbatches: int, rows=None) -> None:
+        """The arena as the paper sizes it: one 2-byte view per matrix parameter and configured microbatch
+        (capacity M * sizeof(W)).  Microbatch m writes bf16(D_m) into its own view at
+        arena[layer_off + m*N*K : +N*K]; nothing is accumulated here.  Same checks and state transitions as
+        backward_dW; the bound destination is the layer's whole region of M views."""
+        if self.aborted:
+            raise ContractError("ABORTED")
+        s = self._resolve(tape)
+        if s.bits & DW_BIT:
+            raise ContractError("DUP_CONSUME", "dW already consumed this tape")
+        if not (s.bits & DI_BIT):
+            raise ContractError("ORDER", "dW before dI")
+        n = self.N * self.K
+        mb = tape.key.mb
+        if (
+            not isinstance(arena, np.ndarray)
+            or arena.dtype != np.uint16
+            or arena.ndim != 1
+            or layer_off < 0
+            or layer_off % 8 != 0  # 16-byte alignment, in 2-byte elements
+            or not (1 <= microbatches <= 64)
+            or mb >= microbatches
+            or layer_off + microbatches * n > arena.size
+        ):
+            raise ContractError("DEST")
+        if self.bound_dest is not None and self.bound_dest != (id(arena), layer_off):
+            raise ContractError("DEST", "differs from the destination bound for this epoch")
+        self.registry.check_and_bind(id(self), arena, layer_off, microbatches * n)
+        if self.write_mask >> mb & 1:
+            raise ContractError("DUP_WRITE")
+        if self.write_mask == 0 and mb != 0:
+            raise ContractError("ORDER", "microbatch 0 initialises the accumulation")
+        if s.Xq is not None and s.Gq is not None:
+            G = fp8.decode(s.Gq, fp8.E5M2)
+            if rows is not None:
+                G = G[:, np.asarray(rows)]
+            acc = G.T @ fp8.decode(s.Xq, fp8.E4M3)
+            bits = bf16.round_from_f64(acc * np.float64(s.sinv_G) * np.float64(s.sinv_X))
+            view = arena[layer_off + mb * n : layer_off + (mb + 1) * n].reshape(self.N, self.K)
+            view[slice(None) if rows is None else np.asarray(rows)] = bits
+        self.bound_dest = (id(arena), layer_off)
+        self.write_mask |= 1 << mb
+        s.bits |= DW_BIT
+        s.live, s.Xq, s.Gq = False, None, None
+
+    def arena_finalize(self, arena: np.ndarray, layer_off: int, microbatches: int, buf: np.ndarray, off: int) -> None:
+        """Before the optimizer boundary: the optimizer-visible FP32 gradient is the sum of the layer's M views,
+        added in microbatch order in FP32: buf[off + i] = (...((v_0[i] + v_1[i]) + v_2[i]) ... + v_{M-1}[i]).
+        Every configured microbatch must have written exactly once."""
+        if self.aborted:
+            raise ContractError("ABORTED")
+        n = self.N * self.K
+        if self.write_mask != (1 << microbatches) - 1:
+            raise ContractError("INCOMPLETE", "a microbatch has not written its view")
+        if self.bound_dest != (id(arena), layer_off):
+            raise ContractError("DEST", "not the arena region bound this epoch")
+        if buf.dtype != np.float32 or buf.ndim != 1 or off < 0 or off % 4 != 0 or off + n > buf.size:
+            raise ContractError("DEST")
+        total = bf16.decode(arena[layer_off : layer_off + n]).astype(np.float32)
+        for m in range(1, microbatches):
+            v = bf16.decode(arena[layer_off + m * n : layer_off + (m + 1) * n]).astype(np.float32)
+            total = (total + v).astype(np.float32)
+        buf[off : off + n] = total
+
     # ------------------------------------------------------------------ boundaries
     def optimizer_boundary(self, microbatches_expected: int) -> None:
         if self.aborted:

@@ -1,4 +1,6 @@
 """Pins for the oracle's F / dI / dW state machine (CPU only): invariants of the contract."""
+from fractions import Fraction
+
 import numpy as np
 import pytest
 from hypothesis import given, settings, strategies as st
@@ -375,3 +377,134 @@ def test_resume_from_quiescent_checkpoint_equals_uninterrupted_run():
     got = run(E, bufE, range(3, 8))
     for k in got:
         assert np.array_equal(full[k].view(np.uint8), got[k].view(np.uint8)), k
+
+
+# ------------------------------------------------------------------------------------------ per-microbatch arena
+def _int_layer_run(M, T, K, N, use_arena, seed=5):
+    """Integer-valued X (|x| <= 7) and dY (|g| <= 7), each containing a 7: every scale is a power of two (448/7,
+    57344/7) and every per-microbatch gradient sum_t g x is a small integer, exact in bf16 and FP32."""
+    rng = np.random.default_rng(seed)
+    L = OracleLinear(T, K, N, 4, 0, M)
+    L.set_weight(inputs.bits(inputs.weights("AR", 0, 0, N, K)))
+    n = N * K
+    arena = np.full(16 + M * n, 0x7FC0, np.uint16)  # NaN-filled: an unwritten view would show
+    buf = np.full(8 + n, np.float32(99.0))
+    exact = np.zeros((N, K), np.int64)
+    tapes = []
+    for m in range(M):
+        x = rng.integers(-7, 8, (T, K))
+        g = rng.integers(-7, 8, (T, N))
+        x[0, 0], g[0, 0] = 7, -7
+        exact += g.T @ x
+        import torch
+
+        tape, _ = L.forward(m, L.e_W, inputs.bits(torch.tensor(x, dtype=torch.float32).to(torch.bfloat16)))
+        L.backward_dI(tape, inputs.bits(torch.tensor(g, dtype=torch.float32).to(torch.bfloat16)))
+        tapes.append(tape)
+    for m in range(M):
+        if use_arena:
+            L.backward_dW_arena(tapes[m], arena, 16, M)
+        else:
+            L.backward_dW(tapes[m], buf, 8)
+    if use_arena:
+        L.arena_finalize(arena, 16, M, buf, 8)
+    return L, arena, buf, exact
+
+
+def test_arena_variant_equals_flat_accumulate_and_integer_matmul_when_views_are_exact():
+    M, T, K, N = 4, 4, 8, 16
+    La, arena, buf_a, exact = _int_layer_run(M, T, K, N, True)
+    Lf, _, buf_f, exact_f = _int_layer_run(M, T, K, N, False)
+    assert np.array_equal(exact, exact_f) and np.abs(exact).max() < 2**24
+    assert np.array_equal(buf_a[8:].reshape(N, K), exact.astype(np.float32))
+    assert np.array_equal(buf_a.view(np.uint32), buf_f.view(np.uint32))
+    assert np.all(buf_a[:8] == 99.0)  # nothing outside the slice
+    assert np.all(arena[:16] == 0x7FC0)
+    views = bf16.decode(arena[16:]).reshape(M, N, K)
+    assert np.array_equal(views.sum(axis=0), exact.astype(np.float64))  # every view holds its own microbatch
+    assert not np.array_equal(views[0], views[1])
+    assert state_equal(La.state(), Lf.state())
+    La.optimizer_boundary(M)
+
+
+def _nearest_bf16_by_search(x: Fraction) -> int:
+    """Nearest bf16 code to an exact rational, ties to the even code, by searching all finite codes."""
+    best, best_err = None, None
+    for code in range(0x10000):
+        if (code & 0x7F80) == 0x7F80:
+            continue
+        v = Fraction(float(bf16.decode(np.array([code], np.uint16))[0]))
+        err = abs(v - x)
+        if best is None or err < best_err or (err == best_err and code % 2 == 0 and best % 2 == 1):
+            best, best_err = code, err
+    return best
+
+
+def test_arena_view_is_one_rounding_of_the_exact_gradient_to_bf16():
+    T, K, N = 3, 2, 2
+    L = OracleLinear(T, K, N, 4, 0, 1)
+    L.set_weight(inputs.bits(inputs.weights("AR", 0, 0, N, K)))
+    X = inputs.bits(inputs.activations("AR", 0, 0, 0, 0, T, K))
+    dY = inputs.bits(inputs.upstream_grads("AR", 0, 0, 0, 0, T, N))
+    L.S["X"].scale, L.S["X"].scale_inv = np.float32(3.7), np.float32(1.0) / np.float32(3.7)
+    L.S["G"].scale, L.S["G"].scale_inv = np.float32(811.0), np.float32(1.0) / np.float32(811.0)
+    tape, _ = L.forward(0, L.e_W, X)
+    L.backward_dI(tape, dY)
+    s = L.slots[tape.ref.slot]
+    Gd, Xd = fp8.decode(s.Gq, fp8.E5M2), fp8.decode(s.Xq, fp8.E4M3)
+    sg, sx = Fraction(float(s.sinv_G)), Fraction(float(s.sinv_X))
+    arena = np.zeros(8, np.uint16)
+    L.backward_dW_arena(tape, arena, 0, 1)
+    for n in range(N):
+        for k in range(K):
+            exact = sum(Fraction(float(Gd[t, n])) * Fraction(float(Xd[t, k])) for t in range(T)) * sg * sx
+            assert int(arena[n * K + k]) == _nearest_bf16_by_search(exact), (n, k)
+
+
+def test_arena_finalize_adds_views_in_microbatch_order_in_fp32():
+    L = OracleLinear(1, 1, 8, 4, 0, 3)
+    L.write_mask, n = 0b111, 8
+    one, tiny = 0x3F80, 0x3380  # bf16 1.0 and 2^-24
+    assert bf16.decode(np.array([tiny], np.uint16))[0] == 2.0**-24
+    buf = np.zeros(8, np.float32)
+    for order, want in (((one, tiny, tiny), np.float32(1.0)), ((tiny, tiny, one), np.float32(1.0) + np.float32(2.0**-23))):
+        arena = np.concatenate([np.full(n, c, np.uint16) for c in order])
+        L.bound_dest = (id(arena), 0)
+        L.arena_finalize(arena, 0, 3, buf, 0)
+        assert np.all(buf == want) and want.dtype == np.float32
+
+
+def test_arena_contract_errors():
+    M, T, K, N = 2, 4, 8, 8
+    L, arena, buf, _ = _int_layer_run(M, T, K, N, True)
+    with pytest.raises(ContractError) as e:
+        L.arena_finalize(arena, 24, M, buf, 8)  # not the bound region
+    assert e.value.code == "DEST"
+    L.optimizer_boundary(M)
+    # next epoch: one view missing -> finalize refuses; duplicate write refused; region too small refused
+    import torch
+
+    L.set_weight(inputs.bits(inputs.weights("AR", 1, 0, N, K)))
+    x = inputs.bits(torch.ones((T, K), dtype=torch.bfloat16))
+    g = inputs.bits(torch.ones((T, N), dtype=torch.bfloat16))
+    t0, _ = L.forward(0, L.e_W, x)
+    t1, _ = L.forward(1, L.e_W, x)
+    L.backward_dI(t0, g)
+    L.backward_dI(t1, g)
+    with pytest.raises(ContractError) as e:
+        L.backward_dW_arena(t1, arena, 16, M)
+    assert e.value.code == "ORDER"  # microbatch 0 first
+    with pytest.raises(ContractError) as e:
+        L.backward_dW_arena(t0, arena[: 16 + N * K], 16, M)
+    assert e.value.code == "DEST"
+    L.backward_dW_arena(t0, arena, 16, M)
+    with pytest.raises(ContractError) as e:
+        L.arena_finalize(arena, 16, M, buf, 8)
+    assert e.value.code == "INCOMPLETE"
+    with pytest.raises(ContractError) as e:
+        L.backward_dW_arena(t0, arena, 16, M)
+    assert e.value.code in ("STALE_REF", "DUP_CONSUME", "DUP_WRITE")
+    L.backward_dW_arena(t1, arena, 16, M)
+    L.arena_finalize(arena, 16, M, buf, 8)
+    assert np.all(buf[8:] == 2 * T)
+    L.optimizer_boundary(M)
