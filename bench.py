@@ -102,11 +102,11 @@ class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
     def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False,
-                 group_dw=True):
+                 group_dw=True, arena=False):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
-        self.group_dw = group_dw and not staged
+        self.group_dw = group_dw and not staged and not arena
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
                               exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
@@ -119,6 +119,8 @@ class Stage:
         offs, per_layer = inputs.grad_offsets(lin)
         self.grad = torch.zeros(per_layer * cfg["layers"], dtype=torch.float32, device=device)
         self.temp = torch.empty(max(K * N for _, K, N in lin), dtype=torch.float32, device=device) if staged else None
+        # per-microbatch arena variant: M bf16 views per linear (capacity M * sum of sizeof(W)), summed at the boundary
+        self.arena = torch.empty(M * per_layer * cfg["layers"], dtype=torch.bfloat16, device=device) if arena else None
         for l in range(cfg["layers"]):
             for j, (_, K, N) in enumerate(lin):
                 w = inputs.weights(cfg_name, l, j, N, K).to(device)
@@ -194,10 +196,15 @@ class Stage:
                         self.d2h += self.dXh[m][i].numel() * 2
                     else:
                         L.backward_dI(tapes[(m, i)], self.dY[m][i], self.dX[m][i])
+                elif self.arena is not None:
+                    L.backward_dW_arena(tapes[(m, i)], self.arena, self.cfg["M"] * self.offsets[i], self.cfg["M"])
                 elif self.temp is not None:
                     L.backward_dW_staged(tapes[(m, i)], self.grad, self.offsets[i], self.temp)
                 else:
                     L.backward_dW(tapes[(m, i)], self.grad, self.offsets[i])
+        if self.arena is not None:
+            for i, L in enumerate(self.layers):
+                L.arena_finalize(self.arena, self.cfg["M"] * self.offsets[i], self.cfg["M"], self.grad, self.offsets[i])
         self.issue_s += time.perf_counter() - t_issue  # host time to enqueue the step (before the boundary's sync)
         for L in self.layers:
             L.optimizer_boundary(self.cfg["M"])
@@ -313,7 +320,7 @@ def gemm_roofline(qe, cfg, peaks, device):
     achieved = tot_flops / (tot_ms * 1e-3) / 1e12
     # dram__bytes_read + dram__bytes_write per launch, averaged over the twelve GEMMs of a microbatch, from one ncu
     # capture of `python -m paper_2609_23536_b200.profile_case gemm_microbatch --small` (config-2 shapes only)
-    traffic = 39.8e6 if (T, tuple(cfg["linears"])) == (2048, tuple(inputs.CONFIGS["C2"]["linears"])) else None
+    traffic = 39.6e6 if (T, tuple(cfg["linears"])) == (2048, tuple(inputs.CONFIGS["C2"]["linears"])) else None
     peak = 2.0 * peaks["bf16_burst"]  # FP8 dense = 2 x the bf16 peak (nominal ratio), kernels timed alone -> burst figure
     return {
         "bound": "tensor", "kernel": "gemm_fp8_pair_kernel", "achieved": round(achieved, 1), "peak": round(peak, 1),
@@ -360,6 +367,9 @@ def hbm_kernels(qe, cfg, peaks, device):
     g = torch.zeros(n // 2, device=device)
     t = torch.ones(n // 2, device=device)
     out["accumulate_12B_per_elt"] = timeit(lambda: qe.qe_accumulate(g, t, True), 12 * (n // 2))
+    views = x.view(8, -1)  # 8 bf16 views of 16.8 M elements -> one FP32 gradient
+    dst = torch.empty(views.shape[1], device=device)
+    out["arena_reduce_8_views_20B_per_elt"] = timeit(lambda: qe.qe_arena_reduce(views, 8, dst), 20 * views.shape[1])
     out["peak_GB/s"] = peaks["hbm_gbs"]
     out["peak_source"] = peaks["source"]
     return out
@@ -449,6 +459,8 @@ def main():
                          "Default: one C-ABI call per action with dW overlapped on the context's second stream")
     ap.add_argument("--no-group-dw", dest="group_dw", action="store_false",
                     help="one qe_backward_dW call per linear instead of qe_backward_dW_multi per microbatch")
+    ap.add_argument("--arena", action="store_true",
+                    help="per-microbatch arena variant: dW writes one bf16 view per linear and microbatch, summed into the FP32 buffer before the boundary")
     ap.add_argument("--staged", action="store_true", help="copied-gradient comparison path: dW into a temporary, then a copy-add kernel")
     ap.add_argument("--own-stream", action="store_true", help="let the context create its own execution stream (event handoff on every action)")
     args = ap.parse_args()
@@ -481,7 +493,7 @@ def main():
 
     use_step = args.step_api
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
-                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw)
+                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena)
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:
@@ -497,7 +509,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "gradient_path": "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),

@@ -223,6 +223,23 @@ int32_t qe_backward_dW(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t 
  * to temp_dev (FP32 [N,K], caller-owned scratch) and then added into the destination by a second kernel. */
 int32_t qe_backward_dW_staged(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t grad_buf_elems,
                               uint64_t offset, float* temp_dev, void* caller_stream);
+/* The arena as the paper sizes it (Sec. 3.4; capacity A_r = M * sum of sizeof(W)): one bf16 view per matrix
+ * parameter and configured microbatch.  arena_dev: bf16 elements; the layer's region is
+ * [layer_offset, layer_offset + microbatches * N*K), microbatch m's view starts at layer_offset + m * N*K.
+ * qe_backward_dW_arena: same checks, order rules (microbatch 0 first, each microbatch exactly once, destination =
+ * the layer's region, bound for the epoch and alias-checked against other layers) and state transitions as
+ * qe_backward_dW, but view[n*K + k] = bf16(D) and nothing is accumulated.  layer_offset a multiple of 8.
+ * qe_arena_finalize: before the optimizer boundary, grad_buf_dev[offset + i] = sum over m of view_m[i], added in
+ * FP32 in microbatch order (one kernel, (2M + 4) bytes per element); INCOMPLETE unless every microbatch wrote,
+ * DEST unless the region is the one bound this epoch; changes no contract state.
+ * qe_arena_reduce: that kernel alone (views_dev: M contiguous views of view_elems bf16 each, view_elems a multiple
+ * of 8, 16-byte aligned). */
+int32_t qe_backward_dW_arena(qe_layer*, const qe_tape*, void* arena_dev, uint64_t arena_elems, uint64_t layer_offset,
+                             uint32_t microbatches, void* caller_stream);
+int32_t qe_arena_finalize(qe_layer*, const void* arena_dev, uint64_t arena_elems, uint64_t layer_offset,
+                          uint32_t microbatches, float* grad_buf_dev, uint64_t grad_buf_elems, uint64_t offset,
+                          void* caller_stream);
+int32_t qe_arena_reduce(const void* views_dev, uint64_t view_elems, uint32_t M, float* dst_dev, void* stream);
 /* The W action of Sec. 4.2 for several layers of the stage at once (typically one microbatch's deferred weight
  * gradients): the same checks, results (bit for bit) and state transitions as qe_backward_dW(layers[i], &tapes[i],
  * grad_buf_dev, grad_buf_elems, offsets[i], stream) for i = 0..n-1, but the GEMMs of up to four layers share one

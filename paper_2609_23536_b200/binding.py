@@ -135,6 +135,9 @@ _SIGNATURES = {
     "qe_backward_dI_host": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
+    "qe_backward_dW_arena": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, C.c_uint32, _P]),
+    "qe_arena_finalize": (C.c_int32, [_P, _P, C.c_uint64, C.c_uint64, C.c_uint32, _P, C.c_uint64, C.c_uint64, _P]),
+    "qe_arena_reduce": (C.c_int32, [_P, C.c_uint64, C.c_uint32, _P, _P]),
     "qe_backward_dW_multi": (C.c_int32, [C.POINTER(_P), C.POINTER(qe_tape), C.c_uint32, _P, C.c_uint64,
                                          C.POINTER(C.c_uint64), _P]),
     "qe_step_run": (C.c_int32, [_P, C.POINTER(_P), C.c_uint32, C.POINTER(qe_step_action), C.c_uint32, C.c_uint32,
@@ -348,6 +351,13 @@ class Layer:
     def backward_dW_staged(self, tape, grad_buf, offset, temp, stream=None):
         _check(lib.qe_backward_dW_staged(self.h, C.byref(tape), _ptr(grad_buf), grad_buf.numel(), offset, _ptr(temp), _stream(stream)))
 
+    def backward_dW_arena(self, tape, arena, layer_offset, microbatches, stream=None):
+        _check(lib.qe_backward_dW_arena(self.h, C.byref(tape), _ptr(arena), arena.numel(), layer_offset, microbatches, _stream(stream)))
+
+    def arena_finalize(self, arena, layer_offset, microbatches, grad_buf, offset, stream=None):
+        _check(lib.qe_arena_finalize(self.h, _ptr(arena), arena.numel(), layer_offset, microbatches, _ptr(grad_buf),
+                                     grad_buf.numel(), offset, _stream(stream)))
+
     def optimizer_boundary(self, expected):
         _check(lib.qe_optimizer_boundary(self.h, expected))
 
@@ -467,6 +477,11 @@ def qe_noalloc_staging_elems() -> int:
 
 
 ACT = {"F": 0, "dI": 1, "dW": 2}
+
+
+def qe_arena_reduce(views, M, dst, stream=None):
+    """views: bf16 tensor of M contiguous views; dst: FP32 tensor of one view's size."""
+    _check(lib.qe_arena_reduce(_ptr(views), views.numel() // M, M, _ptr(dst), _stream(stream)))
 
 
 def backward_dW_multi(layers, tapes, grad_buf, offsets, stream=None):

@@ -67,6 +67,15 @@ struct AccumParams {
   int32_t pad;
 };
 
+// Sum of M bf16 views (view m at views + m * view_vec 16-byte vectors) into FP32, added in view order.
+struct ArenaReduceParams {
+  const uint4* views;   // 8 bf16 per vector
+  float4* dst;          // 2 vectors of 4 FP32 per input vector
+  uint64_t view_vec;    // vectors per view (= N*K / 8)
+  uint32_t M;
+  uint32_t pad;
+};
+
 struct GemmParams {
   CUtensorMap tmA;             // A [M, Kc] bytes, box 128 x 128, 128-byte swizzle
   CUtensorMap tmB;             // B [N, Kc] bytes, box 128 x gemm_b_box_rows(M)
@@ -112,6 +121,7 @@ Launch make_commit(const CommitParams& p);
 Launch make_amax_pass1(const AmaxParams& p);
 Launch make_amax_pass2(const AmaxParams& p);
 Launch make_accumulate(const AccumParams& p);
+Launch make_arena_reduce(const ArenaReduceParams& p);
 Launch make_gemm(const GemmParams& p, int num_sms);
 // One launch for n = 2..4 GEMMs; false if the group cannot be formed (a problem needs the single-CTA variant or a
 // commit tail), in which case the caller launches them one by one.

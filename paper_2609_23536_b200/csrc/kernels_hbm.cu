@@ -228,4 +228,56 @@ Launch make_accumulate(const AccumParams& p) {
   return l;
 }
 
+// ------------------------------------------------------------------------------------------------ arena reduction
+// The per-microbatch arena (one bf16 view per matrix parameter and microbatch): the optimizer-visible FP32 gradient
+// is the sum of the M views, added in microbatch order.  (2 M + 4) bytes per element; a thread owns 8 consecutive
+// elements, the loads of four views are in flight at once.
+__device__ __forceinline__ void add_bf16x8(float (&a)[8], const uint4& v) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    a[2 * j] = __fadd_rn(a[2 * j], __uint_as_float(w[j] << 16));
+    a[2 * j + 1] = __fadd_rn(a[2 * j + 1], __uint_as_float(w[j] & 0xffff0000u));
+  }
+}
+
+__global__ void __launch_bounds__(256) arena_reduce_kernel(const __grid_constant__ ArenaReduceParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < p.view_vec; i += stride) {
+    const uint4* src = p.views + i;
+    const uint4 v0 = __ldcs(src);
+    const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
+    float a[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      a[2 * j] = __uint_as_float(w[j] << 16);
+      a[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+    uint32_t m = 1;
+    for (; m + 4 <= p.M; m += 4) {
+      const uint4 x0 = __ldcs(src + (uint64_t)m * p.view_vec), x1 = __ldcs(src + (uint64_t)(m + 1) * p.view_vec);
+      const uint4 x2 = __ldcs(src + (uint64_t)(m + 2) * p.view_vec), x3 = __ldcs(src + (uint64_t)(m + 3) * p.view_vec);
+      add_bf16x8(a, x0);
+      add_bf16x8(a, x1);
+      add_bf16x8(a, x2);
+      add_bf16x8(a, x3);
+    }
+    for (; m < p.M; ++m) add_bf16x8(a, __ldcs(src + (uint64_t)m * p.view_vec));
+    p.dst[2 * i] = make_float4(a[0], a[1], a[2], a[3]);
+    p.dst[2 * i + 1] = make_float4(a[4], a[5], a[6], a[7]);
+  }
+}
+
+Launch make_arena_reduce(const ArenaReduceParams& p) {
+  Launch l;
+  l.func = (const void*)arena_reduce_kernel;
+  const uint64_t blocks = (p.view_vec + 255) / 256;
+  l.grid = dim3((unsigned)(blocks < 148ull * 8 ? (blocks ? blocks : 1) : 148ull * 8), 1, 1);
+  l.block = dim3(256, 1, 1);
+  l.set(p);
+  return l;
+}
+
 }  // namespace qe

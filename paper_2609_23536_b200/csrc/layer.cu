@@ -526,6 +526,15 @@ qe::GemmParams dW_gemm(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, 
   return gp;
 }
 
+// Per-microbatch arena: the same GEMM writes bf16(D) into the microbatch's own view (no accumulation, no amax).
+qe::GemmParams dW_gemm_view(qe_layer* L, uint32_t p, void* view) {
+  qe::GemmParams gp = dW_gemm(L, p, nullptr, 0, nullptr);
+  gp.out = view;
+  gp.epi = 0;
+  make_out_map(L->ctx->dev, &gp.tmD, view, L->cfg.N, L->cfg.K, L->cfg.K, false);
+  return gp;
+}
+
 void add_dW(qe_layer* L, uint32_t p, float* dst, int32_t accumulate, float* temp, std::vector<qe::Launch>& ls) {
   const uint32_t K = L->cfg.K, N = L->cfg.N;
   ls.push_back(qe::make_gemm(dW_gemm(L, p, dst, accumulate, temp), L->ctx->dev->num_sms));
@@ -807,11 +816,13 @@ int32_t qe_backward_dI_host(qe_layer* L, const qe_tape* tape, const void* dy_hos
   return backward_dI_impl(L, tape, L->dy_stage, L->dx_stage, caller_stream, dy_host, dx_host);
 }
 
+// view != null: per-microbatch arena mode; grad / elems / off / slice then describe the layer's whole region of the
+// arena in 4-byte units (what the contract core's destination rules are written in) and view is this microbatch's.
 static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, uint64_t elems, uint64_t off,
-                                float* temp, void* caller_stream) {
+                                float* temp, void* caller_stream, void* view = nullptr, uint64_t region_units = 0) {
   if (!L || !tape) return fail(QE_ERR_BAD_ARG, "null argument");
   const uint32_t K = L->cfg.K, N = L->cfg.N;
-  const uint64_t slice = (uint64_t)N * K;
+  const uint64_t slice = view ? region_units : (uint64_t)N * K;
   int32_t acc = 0;
   int32_t st = qe_contract_dW_check(L->contract, tape, (uint64_t)(uintptr_t)grad, elems, off, slice, &acc);
   if (st != QE_OK) return st;
@@ -830,7 +841,8 @@ static int32_t backward_dW_impl(qe_layer* L, const qe_tape* tape, float* grad, u
     return st;
   }
   std::vector<qe::Launch> ls;
-  add_dW(L, p, grad + off, acc, temp, ls);
+  if (view) ls.push_back(qe::make_gemm(dW_gemm_view(L, p, view), ctx->dev->num_sms));
+  else add_dW(L, p, grad + off, acc, temp, ls);
   st = run_action(ctx, temp ? &L->gDWs[p] : &L->gDW[p], ls, run_on);
   if (st != QE_OK) return st;
   if (ctx->dw_stream) {  // joined at the optimizer boundary and before the slot's next forward
@@ -850,6 +862,49 @@ int32_t qe_backward_dW_staged(qe_layer* L, const qe_tape* tape, float* grad, uin
                               float* temp, void* stream) {
   if (!temp || ((uintptr_t)temp & 15u)) return fail(QE_ERR_BAD_ARG, "temp_dev must be non-null and 16-byte aligned");
   return backward_dW_impl(L, tape, grad, elems, off, temp, stream);
+}
+
+int32_t qe_backward_dW_arena(qe_layer* L, const qe_tape* tape, void* arena, uint64_t arena_elems, uint64_t layer_offset,
+                             uint32_t microbatches, void* stream) {
+  if (!L || !tape || !arena) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (microbatches < 1 || microbatches > QE_MAX_MICROBATCHES) return fail(QE_ERR_BAD_ARG, "microbatches %u", microbatches);
+  const uint64_t n = (uint64_t)L->cfg.N * L->cfg.K;
+  if (layer_offset % 8 || ((uintptr_t)arena & 15u)) return fail(QE_ERR_DEST, "arena region not 16-byte aligned");
+  if (tape->key.mb >= microbatches) return fail(QE_ERR_DEST, "microbatch %u has no view among %u", tape->key.mb, microbatches);
+  uint16_t* view = (uint16_t*)arena + layer_offset + (uint64_t)tape->key.mb * n;
+  // 2-byte elements expressed in the contract core's 4-byte units (n is even: N and K are multiples of 128)
+  return backward_dW_impl(L, tape, (float*)arena, arena_elems / 2, layer_offset / 2, nullptr, stream, view, microbatches * n / 2);
+}
+
+int32_t qe_arena_finalize(qe_layer* L, const void* arena, uint64_t arena_elems, uint64_t layer_offset, uint32_t microbatches,
+                          float* grad, uint64_t grad_elems, uint64_t off, void* caller_stream) {
+  if (!L || !arena || !grad) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (microbatches < 1 || microbatches > QE_MAX_MICROBATCHES) return fail(QE_ERR_BAD_ARG, "microbatches %u", microbatches);
+  const qe_contract* c = L->contract;
+  const uint64_t n = (uint64_t)L->cfg.N * L->cfg.K;
+  if (c->aborted) return fail(QE_ERR_ABORTED, "step aborted; arena unusable for this epoch");
+  const uint64_t want = microbatches == 64 ? ~0ull : ((1ull << microbatches) - 1);
+  if (c->write_mask != want)
+    return fail(QE_ERR_INCOMPLETE, "view write mask %#llx, expected %#llx", (unsigned long long)c->write_mask, (unsigned long long)want);
+  if (!c->has_dest || c->dest_addr != (uint64_t)(uintptr_t)arena || c->dest_off != layer_offset / 2 || layer_offset % 8)
+    return fail(QE_ERR_DEST, "not the arena region bound for this epoch");
+  if (layer_offset > arena_elems || microbatches * n > arena_elems - layer_offset) return fail(QE_ERR_DEST, "region exceeds the arena");
+  if (off > grad_elems || n > grad_elems - off || ((uintptr_t)(grad + off) & 15u)) return fail(QE_ERR_DEST, "gradient slice out of range or misaligned");
+  qe_ctx* ctx = L->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  int32_t st = handoff_in(ctx, caller);
+  if (st != QE_OK) return st;
+  if (ctx->dw_stream) {  // the views were written on the second stream
+    QE_CUDA(cudaEventRecord(ctx->ev_dw_in, ctx->dw_stream));
+    QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_dw_in, 0));
+  }
+  qe::ArenaReduceParams ap{};
+  ap.views = (const uint4*)((const uint16_t*)arena + layer_offset);
+  ap.dst = (float4*)(grad + off);
+  ap.view_vec = n / 8;
+  ap.M = microbatches;
+  if ((st = launch_eager(ctx, qe::make_arena_reduce(ap), ctx->exec_stream)) != QE_OK) return st;
+  return handoff_out(ctx, caller);
 }
 
 // Graph of a launch list identified by a hash (whole steps, multi-layer dW calls); rebuilt when the list's length
@@ -1280,6 +1335,18 @@ int32_t qe_accumulate(float* dst, const float* src, uint64_t n, int32_t accumula
   ap.nvec = n / 4;
   ap.accumulate = accumulate;
   return launch_on(qe::make_accumulate(ap), (cudaStream_t)stream);
+}
+
+int32_t qe_arena_reduce(const void* views, uint64_t view_elems, uint32_t M, float* dst, void* stream) {
+  if (!views || !dst) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (M < 1 || M > QE_MAX_MICROBATCHES) return fail(QE_ERR_BAD_ARG, "M %u", M);
+  if (view_elems == 0 || view_elems % 8 || (((uintptr_t)views | (uintptr_t)dst) & 15u)) return fail(QE_ERR_BAD_ARG, "views of a multiple of 8 elements, 16-byte aligned");
+  qe::ArenaReduceParams ap{};
+  ap.views = (const uint4*)views;
+  ap.dst = (float4*)dst;
+  ap.view_vec = view_elems / 8;
+  ap.M = M;
+  return launch_on(qe::make_arena_reduce(ap), (cudaStream_t)stream);
 }
 
 int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void* b, uint32_t b_fmt, uint32_t b_mn,

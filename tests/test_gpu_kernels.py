@@ -221,3 +221,30 @@ def test_gemm_mn_major_needs_the_paired_variant(qe):
     with pytest.raises(qe.QEError) as e:
         qe.qe_gemm_fp8_ex(A, 0, True, B, 0, False, one, one, D, 1, None, status)
     assert e.value.code == "UNSUPPORTED"
+
+
+# ------------------------------------------------------------------------------------------ arena reduction
+@pytest.mark.parametrize("M,n", [(1, 8), (2, 8 * 300), (5, 8 * 1031), (8, 1 << 20), (64, 8 * 512)])
+def test_arena_reduce_adds_views_in_order(qe, M, n):
+    g = torch.Generator().manual_seed(M * 1000 + n)
+    views = (torch.randn((M, n), generator=g) * torch.logspace(-3, 3, M).unsqueeze(1)).to(torch.bfloat16)
+    want = bf16.decode(inputs.bits(views[0])).astype(np.float32)
+    for m in range(1, M):  # sequential FP32 additions, microbatch order (the oracle's arena_finalize)
+        want = (want + bf16.decode(inputs.bits(views[m])).astype(np.float32)).astype(np.float32)
+    dst = torch.full((n + 4,), 7.0, device=DEV)
+    qe.qe_arena_reduce(views.to(DEV), M, dst[:n])
+    torch.cuda.synchronize()
+    assert np.array_equal(dst[:n].cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert torch.all(dst[n:] == 7.0).item()
+
+
+def test_arena_reduce_order_is_visible_in_the_result(qe):
+    # (1 + 2^-24) + 2^-24 = 1 in FP32 while 2^-24 + 2^-24 + 1 = 1 + 2^-23
+    one, tiny = torch.ones(8, dtype=torch.bfloat16), torch.full((8,), 2.0**-24, dtype=torch.bfloat16)
+    dst = torch.zeros(8, device=DEV)
+    qe.qe_arena_reduce(torch.stack([one, tiny, tiny]).to(DEV), 3, dst)
+    assert torch.all(dst == 1.0).item()
+    qe.qe_arena_reduce(torch.stack([tiny, tiny, one]).to(DEV), 3, dst)
+    assert torch.all(dst == 1.0 + 2.0**-23).item()
+    with pytest.raises(qe.QEError):
+        qe.qe_arena_reduce(torch.zeros((2, 12), dtype=torch.bfloat16, device=DEV), 2, torch.zeros(12, device=DEV))

@@ -446,3 +446,106 @@ def test_limits_longest_history_most_slots_and_microbatches(qe):
     L.optimizer_boundary(64)
     O.optimizer_boundary(64)
     assert L.state()["e_W"] == 1 and L.state()["write_mask"] == 0
+
+
+# ------------------------------------------------------------------------------------------ per-microbatch arena
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+@pytest.mark.parametrize("overlap", [False, True], ids=["inline", "overlapped"])
+def test_arena_variant_against_oracle_and_flat_path(qe, mode, overlap):
+    """One bf16 view per microbatch, summed at finalisation (the arena as the paper sizes it) against the oracle's
+    arena functions; and against the flat accumulate, which it must stay close to (bf16 rounding per microbatch)."""
+    T, K, N, M, H = 256, 256, 512, 4, 4
+    s = sched(M, 2, 1)
+    P = peak_live(s)
+    W = _weights("AR", N, K, 2)
+    get = lambda step, mb: c1_inputs(step, mb, T, K, N, "AR")
+    n = N * K
+    # oracle
+    O = OracleLinear(T, K, N, H, 0, P)
+    o_arena = np.zeros(8 + M * n, np.uint16)
+    o_buf = np.zeros(4 + n, np.float32)
+    # GPU
+    ctx = qe.Context(mode, overlap_dw=overlap)
+    L = qe.Layer(ctx, T, K, N, H, 0, P, inputs.from_bits(W[0]).to(DEV))
+    arena = torch.full((8 + M * n,), float("nan"), dtype=torch.bfloat16, device=DEV)
+    grad = torch.full((4 + n,), -1.0, device=DEV)
+    flat = torch.zeros(n, device=DEV)
+    ctx2 = qe.Context(mode)
+    L2 = qe.Layer(ctx2, T, K, N, H, 0, P, inputs.from_bits(W[0]).to(DEV))
+    for step in range(2):
+        O.set_weight(W[step])
+        for lay in (L, L2):
+            lay.weight.copy_(inputs.from_bits(W[step]).to(DEV))
+        tapes, otapes, tapes2 = {}, {}, {}
+        for a, m in s:
+            X, dY = get(step, m)
+            x, dy = inputs.from_bits(X).to(DEV), inputs.from_bits(dY).to(DEV)
+            if a == "F":
+                otapes[m], _ = O.forward(m, O.e_W, X)
+                tapes[m] = L.forward(m, step, x, torch.empty((T, N), dtype=torch.bfloat16, device=DEV))
+                tapes2[m] = L2.forward(m, step, x, torch.empty((T, N), dtype=torch.bfloat16, device=DEV))
+            elif a == "dI":
+                O.backward_dI(otapes[m], dY)
+                L.backward_dI(tapes[m], dy, torch.empty((T, K), dtype=torch.bfloat16, device=DEV))
+                L2.backward_dI(tapes2[m], dy, torch.empty((T, K), dtype=torch.bfloat16, device=DEV))
+            else:
+                O.backward_dW_arena(otapes[m], o_arena, 8, M)
+                L.backward_dW_arena(tapes[m], arena, 8, M)
+                L2.backward_dW(tapes2[m], flat, 0)
+        O.arena_finalize(o_arena, 8, M, o_buf, 4)
+        L.arena_finalize(arena, 8, M, grad, 4)
+        torch.cuda.synchronize()
+        got_views = inputs.bits(arena.cpu())
+        for m in range(M):
+            assert_gemm_close(got_views[8 + m * n: 8 + (m + 1) * n].reshape(N, K), o_arena[8 + m * n: 8 + (m + 1) * n].reshape(N, K),
+                              f"view step {step} mb {m}")
+        assert np.all(np.isnan(bf16.decode(got_views[:8])))  # nothing before the region
+        g = grad.cpu().numpy()
+        assert np.all(g[:4] == -1.0)
+        assert assert_grad_close(g[4:], o_buf[4:], f"finalised gradient step {step}") < 1e-3
+        # the GPU's own views summed by the oracle's rule give the GPU's gradient bit for bit
+        want = bf16.decode(got_views[8: 8 + n]).astype(np.float32)
+        for m in range(1, M):
+            want = (want + bf16.decode(got_views[8 + m * n: 8 + (m + 1) * n]).astype(np.float32)).astype(np.float32)
+        assert np.array_equal(g[4:].view(np.uint32), want.view(np.uint32))
+        L2.optimizer_boundary(M)
+        # against the flat FP32 accumulate the views lose what bf16 rounding loses: up to 2^-9 relative per view
+        f = flat.cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(g[4:] - f) / np.linalg.norm(f) < 2.0**-8
+        O.optimizer_boundary(M)
+        L.optimizer_boundary(M)
+        assert state_equal_except_Y(L.state(), O.state())
+
+
+def test_arena_variant_contract_errors(qe):
+    T, K, N, M = 256, 256, 256, 2
+    ctx, L = _mk_layer(qe, 0, T, K, N, 4, 0, 2)
+    n = N * K
+    arena = torch.zeros(M * n + 8, dtype=torch.bfloat16, device=DEV)
+    grad = torch.zeros(n, device=DEV)
+    x = torch.ones((T, K), dtype=torch.bfloat16, device=DEV)
+    dy = torch.ones((T, N), dtype=torch.bfloat16, device=DEV)
+    y, dx = torch.empty((T, N), dtype=torch.bfloat16, device=DEV), torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+    t0, t1 = L.forward(0, 0, x, y), L.forward(1, 0, x, y)
+    L.backward_dI(t0, dy, dx)
+    L.backward_dI(t1, dy, dx)
+    for args, code in (((t1, arena, 8, M), "ORDER"), ((t0, arena, 4, M), "DEST"), ((t0, arena[: n + 8], 8, M), "DEST"),
+                       ((t0, arena, 8, 0), "BAD_ARG")):
+        with pytest.raises(qe.QEError) as e:
+            L.backward_dW_arena(*args)
+        assert e.value.code == code
+    L.backward_dW_arena(t0, arena, 8, M)
+    with pytest.raises(qe.QEError) as e:
+        L.arena_finalize(arena, 8, M, grad, 0)
+    assert e.value.code == "INCOMPLETE"
+    with pytest.raises(qe.QEError) as e:
+        L.backward_dW_arena(t1, arena, 0, M)  # another region than the one bound this epoch
+    assert e.value.code == "DEST"
+    L.backward_dW_arena(t1, arena, 8, M)
+    with pytest.raises(qe.QEError) as e:
+        L.arena_finalize(arena, 0, M, grad, 0)
+    assert e.value.code == "DEST"
+    L.arena_finalize(arena, 8, M, grad, 0)
+    torch.cuda.synchronize()
+    L.optimizer_boundary(M)
+    assert L.state()["e_W"] == 1
