@@ -102,11 +102,12 @@ class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
     def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False,
-                 group_dw=True, arena=False):
+                 group_dw=True, arena=False, chain=False):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
         self.group_dw = group_dw and not staged and not arena
+        self.chain = chain
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
                               exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
@@ -126,6 +127,15 @@ class Stage:
                 w = inputs.weights(cfg_name, l, j, N, K).to(device)
                 self.layers.append(qe.Layer(self.ctx, T, K, N, cfg["H"], cfg["margin"], P, w, stage=0, unit=l * len(lin) + j, host_io=host_io))
                 self.offsets.append(l * per_layer + offs[j])
+        # groups of directly chainable linears (next K == this N, T and N multiples of 256), at most 16 long
+        self.groups = []
+        for i, L in enumerate(self.layers):
+            fits = (self.groups and len(self.groups[-1]) < 16 and self.layers[self.groups[-1][-1]].N == L.K
+                    and L.N % 256 == 0 and L.T % 256 == 0 and self.layers[self.groups[-1][-1]].N % 256 == 0)
+            if chain and fits:
+                self.groups[-1].append(i)
+            else:
+                self.groups.append([i])
         # distinct synthetic tensors per (microbatch, linear); drawn on the host once, outside any timed region
         g = torch.Generator(device="cpu")
         g.manual_seed(inputs.seed_for(cfg_name, "bench"))
@@ -173,6 +183,16 @@ class Stage:
         t_issue = time.perf_counter()
         for a, m in self.schedule:
             order = range(n) if a == "F" else range(n - 1, -1, -1)
+            if self.chain and a != "dW" and not host_io:
+                # the linears as directly chained groups of up to 16 (FP8 hand-off: one cast per group and direction)
+                for g in (self.groups if a == "F" else reversed(self.groups)):
+                    ls = [self.layers[i] for i in g]
+                    if a == "F":
+                        for i, t in zip(g, self.qe.forward_chain(ls, m, self.epoch, self.X[m][g[0]], self.Y[m][g[-1]])):
+                            tapes[(m, i)] = t
+                    else:
+                        self.qe.backward_dI_chain(ls, [tapes[(m, i)] for i in g], self.dY[m][g[-1]], self.dX[m][g[0]])
+                continue
             if a == "dW" and self.group_dw:  # one call for the microbatch's weight gradients of all linears
                 ordl = list(order)
                 for lo in range(0, n, 16):
@@ -459,6 +479,9 @@ def main():
                          "Default: one C-ABI call per action with dW overlapped on the context's second stream")
     ap.add_argument("--no-group-dw", dest="group_dw", action="store_false",
                     help="one qe_backward_dW call per linear instead of qe_backward_dW_multi per microbatch")
+    ap.add_argument("--chain", action="store_true",
+                    help="treat consecutive linears whose shapes fit (K of the next = N of this) as directly chained: "
+                         "qe_forward_chain / qe_backward_dI_chain with FP8 hand-off (config C5)")
     ap.add_argument("--arena", action="store_true",
                     help="per-microbatch arena variant: dW writes one bf16 view per linear and microbatch, summed into the FP32 buffer before the boundary")
     ap.add_argument("--staged", action="store_true", help="copied-gradient comparison path: dW into a temporary, then a copy-add kernel")
@@ -493,7 +516,7 @@ def main():
 
     use_step = args.step_api
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
-                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena)
+                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain)
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:
@@ -509,7 +532,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "chained_fp8_handoff": bool(args.chain), "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),

@@ -223,6 +223,23 @@ int32_t qe_backward_dW(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t 
  * to temp_dev (FP32 [N,K], caller-owned scratch) and then added into the destination by a second kernel. */
 int32_t qe_backward_dW_staged(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t grad_buf_elems,
                               uint64_t offset, float* temp_dev, void* caller_stream);
+/* FP8 hand-off between directly chained linears (layers[i+1] consumes layers[i]'s output: same T,
+ * K_{i+1} = N_i; host array of n <= QE_MAX_CHAIN distinct layers of one context).  qe_forward_chain runs F of every
+ * layer for microbatch mb: x_dev bf16 [T, K_0] in, y_dev bf16 [T, N_{n-1}] out, tapes_out[n].  The output of
+ * layers[i] (i < n-1) is never stored as bf16: its forward GEMM's epilogue rounds it to bf16, takes max|Y| of the
+ * rounded values (committed as layers[i]'s Y amax and layers[i+1]'s X amax), multiplies by layers[i+1]'s current X
+ * scale in FP32 and converts to E4M3 straight into layers[i+1]'s tape slot, with that layer's inverse-scale
+ * snapshot -- exactly the bytes and state that qe_forward(layers[i]) followed by qe_forward(layers[i+1]) on the
+ * bf16 tensor would have produced, without the cast kernel and its 3 bytes per element.  qe_backward_dI_chain is
+ * the same in the backward direction (tapes[] in layer order): dy_dev bf16 [T, N_{n-1}] in, dx_dev bf16 [T, K_0]
+ * out, each input gradient handed to the layer before it as E5M2 with that layer's G scale.  Every layer's contract
+ * check is made before anything runs; dW of each layer follows through qe_backward_dW / _multi as usual.
+ * UNSUPPORTED when a receiving layer keeps transposed FP8 copies (T and N multiples of 256 are required). */
+#define QE_MAX_CHAIN 16
+int32_t qe_forward_chain(qe_layer* const* layers, uint32_t n, uint32_t mb, uint64_t gen, const void* x_dev,
+                         void* y_dev, void* caller_stream, qe_tape* tapes_out);
+int32_t qe_backward_dI_chain(qe_layer* const* layers, const qe_tape* tapes, uint32_t n, const void* dy_dev,
+                             void* dx_dev, void* caller_stream);
 /* The arena as the paper sizes it (Sec. 3.4; capacity A_r = M * sum of sizeof(W)): one bf16 view per matrix
  * parameter and configured microbatch.  arena_dev: bf16 elements; the layer's region is
  * [layer_offset, layer_offset + microbatches * N*K), microbatch m's view starts at layer_offset + m * N*K.

@@ -135,6 +135,8 @@ _SIGNATURES = {
     "qe_backward_dI_host": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
+    "qe_forward_chain": (C.c_int32, [C.POINTER(_P), C.c_uint32, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
+    "qe_backward_dI_chain": (C.c_int32, [C.POINTER(_P), C.POINTER(qe_tape), C.c_uint32, _P, _P, _P]),
     "qe_backward_dW_arena": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, C.c_uint32, _P]),
     "qe_arena_finalize": (C.c_int32, [_P, _P, C.c_uint64, C.c_uint64, C.c_uint32, _P, C.c_uint64, C.c_uint64, _P]),
     "qe_arena_reduce": (C.c_int32, [_P, C.c_uint64, C.c_uint32, _P, _P]),
@@ -477,6 +479,27 @@ def qe_noalloc_staging_elems() -> int:
 
 
 ACT = {"F": 0, "dI": 1, "dW": 2}
+
+
+def forward_chain(layers, mb, gen, x, y, stream=None):
+    """qe_forward_chain: F of directly chained linears with FP8 hand-off; returns one tape per layer."""
+    n = len(layers)
+    hs = (_P * n)(*[L.h for L in layers])
+    tapes = (qe_tape * n)()
+    _check(lib.qe_forward_chain(hs, n, mb, gen, _ptr(x), _ptr(y), _stream(stream), tapes))
+    out = []
+    for t in tapes:  # copies that outlive the ctypes array
+        c = qe_tape()
+        C.memmove(C.byref(c), C.byref(t), C.sizeof(qe_tape))
+        out.append(c)
+    return out
+
+
+def backward_dI_chain(layers, tapes, dy, dx, stream=None):
+    n = len(layers)
+    hs = (_P * n)(*[L.h for L in layers])
+    ts = (qe_tape * n)(*tapes)
+    _check(lib.qe_backward_dI_chain(hs, ts, n, _ptr(dy), _ptr(dx), _stream(stream)))
 
 
 def qe_arena_reduce(views, M, dst, stream=None):

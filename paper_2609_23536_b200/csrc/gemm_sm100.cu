@@ -34,6 +34,7 @@
 // word, raises a CTA-wide abort flag that all other waits observe, and the CTA falls through to its common exit
 // where tensor memory is released.
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 
 #include "commit.cuh"
 #include "kernels.h"
@@ -336,6 +337,10 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
   // operands, scales and the destination may come from it, so wait for it here.
   grid_dep_wait();
   grid_dep_launch();
+  if (blockIdx.x == 0 && threadIdx.x == 64) {  // FP8 hand-off: the consumer's tape snapshot of its inverse scale
+    const GemmParams& q = ps.first();
+    if (q.epi == 3 && q.sinv_dst) *q.sinv_dst = *q.sinv_src;
+  }
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -475,6 +480,41 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
           fence_async_smem();
           __syncwarp();
           if (lane == 0) tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
+        } else if (p.epi == 3) {
+          // FP8 hand-off to the consuming linear: round to bf16 (the value that linear would have read), take its
+          // magnitude for the amax, multiply by the consumer's scale in FP32 and convert -- the consumer's cast
+          // kernel, applied to registers.  32 bytes per row; two 1 KB tiles per warp.
+          const uint32_t buf = epi_smem + (n_groups & 1u) * 1024u;
+          if (lane == 0) tma_store_wait_read<1>();
+          __syncwarp();
+          const float qs = *p.out_scale;
+          uint32_t q[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            uint32_t w[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              w[h] = pack_bf16(__fmul_rn(__uint_as_float(rc[4 * j + 2 * h]), alpha), __fmul_rn(__uint_as_float(rc[4 * j + 2 * h + 1]), alpha));
+              amax_bits = __vmaxu2(amax_bits, w[h] & 0x7fff7fffu);
+            }
+            const float2 f01 = make_float2(__fmul_rn(__uint_as_float(w[0] << 16), qs), __fmul_rn(__uint_as_float(w[0] & 0xffff0000u), qs));
+            const float2 f23 = make_float2(__fmul_rn(__uint_as_float(w[1] << 16), qs), __fmul_rn(__uint_as_float(w[1] & 0xffff0000u), qs));
+            const uint32_t lo = p.out_fmt == 0 ? __nv_cvt_float2_to_fp8x2(f01, __NV_SATFINITE, __NV_E4M3)
+                                               : __nv_cvt_float2_to_fp8x2(f01, __NV_SATFINITE, __NV_E5M2);
+            const uint32_t hi = p.out_fmt == 0 ? __nv_cvt_float2_to_fp8x2(f23, __NV_SATFINITE, __NV_E4M3)
+                                               : __nv_cvt_float2_to_fp8x2(f23, __NV_SATFINITE, __NV_E5M2);
+            q[j] = lo | (hi << 16);
+          }
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const uint32_t dst = buf + (uint32_t)lane * 32u + ((uint32_t)c << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(q[4 * c]), "r"(q[4 * c + 1]),
+                         "r"(q[4 * c + 2]), "r"(q[4 * c + 3])
+                         : "memory");
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) tma_store_2d(&p.tmD, buf, (int)col, (int)blk_row0);
         } else {
           // one tile: waiting for the previous block's store to have read it paces the FP32 traffic, which measured
           // faster than two tiles in flight per warp
@@ -505,10 +545,13 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
         if (TWO) mbar_arrive_cluster(acc ? tempty_leader1 : tempty_leader0);  // the MMA issuer waits in the even CTA
         else mbar_arrive(tempty_bar(acc));
       }
-      if (p.epi == 0 && p.amax_bits) {
+      if ((p.epi == 0 || p.epi == 3) && (p.amax_bits || p.amax_bits2)) {
         // two packed bf16 magnitudes -> FP32 bit pattern of the larger
         const uint32_t w = __reduce_max_sync(0xffffffffu, max(amax_bits & 0xffffu, amax_bits >> 16) << 16);
-        if (lane == 0 && w) atomicMax(p.amax_bits, w);
+        if (lane == 0 && w) {
+          if (p.amax_bits) atomicMax(p.amax_bits, w);
+          if (p.amax_bits2) atomicMax(p.amax_bits2, w);
+        }
       }
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }

@@ -79,7 +79,7 @@ struct ArenaReduceParams {
 struct GemmParams {
   CUtensorMap tmA;             // A [M, Kc] bytes, box 128 x 128, 128-byte swizzle
   CUtensorMap tmB;             // B [N, Kc] bytes, box 128 x gemm_b_box_rows(M)
-  CUtensorMap tmD;             // D [M, N] (bf16 or FP32), box 32 x 32, for the epilogue's bulk stores (epi 0 and 1)
+  CUtensorMap tmD;             // D [M, N] (bf16, FP32 or FP8 bytes), box 32 x 32, for the epilogue's bulk stores
   uint32_t M, N, Kc;
   uint32_t idesc;              // tcgen05 instruction descriptor (formats, majors, shape)
   uint32_t a_mn, b_mn;         // operand given MN-major (as [Kc, M] / [Kc, N] bytes): paired variant only
@@ -87,8 +87,17 @@ struct GemmParams {
   const float* alpha_b;
   void* out;                   // bf16 or FP32 [M, N], row pitch ldo elements
   uint32_t ldo;
-  int32_t epi;                 // 0 bf16 (+amax), 1 FP32 overwrite, 2 FP32 accumulate
+  int32_t epi;                 // 0 bf16 (+amax), 1 FP32 overwrite, 2 FP32 accumulate, 3 FP8 hand-off (below)
   uint32_t* amax_bits;         // or null
+  // epi 3: the bf16-rounded result is not stored; it is quantised for the consuming linear as that linear's own
+  // cast kernel would have done: q = fp8(fp32(bf16(D)) * *out_scale), max|bf16(D)| also into *amax_bits2, and
+  // *sinv_dst = *sinv_src (the consumer's tape snapshot)
+  const float* out_scale;
+  int32_t out_fmt;             // 0 = E4M3, 1 = E5M2
+  uint32_t pad0;
+  uint32_t* amax_bits2;        // or null
+  const float* sinv_src;
+  float* sinv_dst;
   uint32_t* status;
   CommitParams commit;         // performed by the last CTA to finish (commit.st != null)
 };
@@ -107,7 +116,7 @@ struct Launch {
   dim3 grid{1, 1, 1}, block{1, 1, 1};
   uint32_t smem = 0;
   uint32_t nbytes = 0;
-  alignas(64) unsigned char params[2304];
+  alignas(64) unsigned char params[2560];
   template <class P>
   void set(const P& p) {
     static_assert(sizeof(P) <= sizeof(params), "parameter block too large");

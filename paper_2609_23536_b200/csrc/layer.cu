@@ -87,6 +87,19 @@ int32_t make_out_map(const DeviceInfo* d, CUtensorMap* map, const void* ptr, uin
   return QE_OK;
 }
 
+// Tensor map over FP8 bytes D [M, N] (row pitch ld bytes) for the hand-off epilogue: 32-byte x 32-row boxes, no swizzle.
+int32_t make_out_map_u8(const DeviceInfo* d, CUtensorMap* map, const void* ptr, uint64_t M, uint64_t N, uint64_t ld) {
+  cuuint64_t gdim[2] = {N, M};
+  cuuint64_t gstride[1] = {ld};
+  cuuint32_t box[2] = {32u, 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = d->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(QE_ERR_CUDA, "cuTensorMapEncodeTiled (FP8 output) failed with %d", (int)r);
+  return QE_OK;
+}
+
 uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
 bool shape_ok(uint32_t v) { return v >= 256 && v % 128 == 0 && v <= (1u << 20); }
@@ -451,9 +464,13 @@ void add_refresh(qe_layer* L, std::vector<qe::Launch>& ls) {
                             QE_E4M3, 1u << QE_CLASS_W));
 }
 
-void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe::Launch>& ls) {
+// FP8 hand-off between directly chained linears: the forward GEMM of `L` emits its output as the E4M3 input of
+// `next` (quantised with next's current X scale, straight into next's tape slot pn, with next's X amax and
+// inverse-scale snapshot), so `next` needs no cast kernel; x == null means L's own input was deposited that way.
+void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe::Launch>& ls, qe_layer* next = nullptr,
+                 uint32_t pn = 0) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
-  ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
+  if (x) ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
   qe::GemmParams gp{};
   gp.tmA = L->tmXq_A[p];
   gp.tmB = L->tmWq_B;
@@ -463,19 +480,33 @@ void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe
   gp.idesc = qe::gemm_idesc(QE_E4M3, QE_E4M3, T);
   gp.alpha_a = &L->st->slot_sinv_X[p];
   gp.alpha_b = &L->st->cache_sinv_W;
-  gp.out = y;
   gp.ldo = N;
-  gp.epi = 0;
-  make_out_map(L->ctx->dev, &gp.tmD, y, T, N, N, false);
+  if (next) {
+    gp.out = next->Xq[pn];
+    gp.epi = 3;
+    make_out_map_u8(L->ctx->dev, &gp.tmD, next->Xq[pn], T, N, N);
+    gp.out_scale = &next->st->scale[QE_CLASS_X];
+    gp.out_fmt = QE_E4M3;
+    gp.amax_bits2 = &next->st->pending_amax[QE_CLASS_X];
+    gp.sinv_src = &next->st->scale_inv[QE_CLASS_X];
+    gp.sinv_dst = &next->st->slot_sinv_X[pn];
+  } else {
+    gp.out = y;
+    gp.epi = 0;
+    make_out_map(L->ctx->dev, &gp.tmD, y, T, N, N, false);
+  }
   gp.amax_bits = &L->st->pending_amax[QE_CLASS_Y];
   gp.status = &L->st->status;
   gp.commit = commit_params(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr);  // done by the GEMM's last CTA
   ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
 }
 
-void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::Launch>& ls) {
+// Hand-off in the backward direction: the input gradient of `L` is the output gradient of the linear before it
+// (`prev`), emitted as E5M2 with prev's G scale into prev's tape slot pp; dy == null: L's own dY came that way.
+void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::Launch>& ls, qe_layer* prev = nullptr,
+            uint32_t pp = 0) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
-  ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
+  if (dy) ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
   qe::GemmParams gp{};
   const bool b_mn = L->WqT == nullptr;  // no transposed weight copy: Wq [N,K] is B in MN-major form
   gp.tmA = L->tmGq_A[p];
@@ -487,10 +518,21 @@ void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::L
   gp.b_mn = b_mn;
   gp.alpha_a = &L->st->slot_sinv_G[p];
   gp.alpha_b = &L->st->cache_sinv_W;
-  gp.out = dx;
   gp.ldo = K;
-  gp.epi = 0;
-  make_out_map(L->ctx->dev, &gp.tmD, dx, T, K, K, false);
+  if (prev) {
+    gp.out = prev->Gq[pp];
+    gp.epi = 3;
+    make_out_map_u8(L->ctx->dev, &gp.tmD, prev->Gq[pp], T, K, K);
+    gp.out_scale = &prev->st->scale[QE_CLASS_G];
+    gp.out_fmt = QE_E5M2;
+    gp.amax_bits2 = &prev->st->pending_amax[QE_CLASS_G];
+    gp.sinv_src = &prev->st->scale_inv[QE_CLASS_G];
+    gp.sinv_dst = &prev->st->slot_sinv_G[pp];
+  } else {
+    gp.out = dx;
+    gp.epi = 0;
+    make_out_map(L->ctx->dev, &gp.tmD, dx, T, K, K, false);
+  }
   gp.amax_bits = nullptr;
   gp.status = &L->st->status;
   gp.commit = commit_params(L, 1u << QE_CLASS_G, 1, nullptr);  // backward amax/scale updated exactly once, here
@@ -995,6 +1037,105 @@ int32_t qe_backward_dW_multi(qe_layer* const* layers, const qe_tape* tapes, uint
     const uint64_t slice = (uint64_t)layers[i]->cfg.N * layers[i]->cfg.K;
     if ((st = qe_contract_dW_commit(layers[i]->contract, &tapes[i], (uint64_t)(uintptr_t)grad, offsets[i], slice)) != QE_OK) return st;
   }
+  return QE_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ chained linears
+static int32_t check_chain(qe_layer* const* layers, uint32_t n) {
+  if (!layers || n == 0 || n > QE_MAX_CHAIN) return fail(QE_ERR_BAD_ARG, "null argument or bad chain length %u", n);
+  for (uint32_t i = 0; i < n; ++i) {
+    if (!layers[i] || layers[i]->ctx != layers[0]->ctx) return fail(QE_ERR_BAD_ARG, "layer %u is null or belongs to another context", i);
+    for (uint32_t j = 0; j < i; ++j)
+      if (layers[j] == layers[i]) return fail(QE_ERR_BAD_ARG, "layer %u appears twice", i);
+    if (i && (layers[i]->cfg.T != layers[0]->cfg.T || layers[i]->cfg.K != layers[i - 1]->cfg.N))
+      return fail(QE_ERR_SHAPE, "layer %u does not take layer %u's output ([%u, %u] after [%u, %u])", i, i - 1, layers[i]->cfg.T,
+                  layers[i]->cfg.K, layers[i - 1]->cfg.T, layers[i - 1]->cfg.N);
+  }
+  // a deposited FP8 tensor is the row-major one only: every layer that receives one must run without transposed copies
+  for (uint32_t i = 0; i < n; ++i)
+    if ((i > 0 && layers[i]->XqT[0]) || (i + 1 < n && layers[i]->GqT[0]))
+      return fail(QE_ERR_UNSUPPORTED, "layer %u keeps transposed FP8 copies (T and N must be multiples of 256 for the hand-off)", i);
+  return QE_OK;
+}
+
+static int32_t run_keyed(qe_ctx* ctx, uint64_t key, const std::vector<qe::Launch>& ls) {
+  if (ctx->exec_mode == QE_EXEC_GRAPH) {
+    ActionGraph* g = keyed_graph(ctx, key, ls.size());
+    if (!g) return fail(QE_ERR_BAD_ARG, "out of host memory");
+    return run_action(ctx, g, ls);
+  }
+  for (const qe::Launch& l : ls) {
+    int32_t st = launch_eager(ctx, l, ctx->exec_stream);
+    if (st != QE_OK) return st;
+  }
+  return QE_OK;
+}
+
+int32_t qe_forward_chain(qe_layer* const* layers, uint32_t n, uint32_t mb, uint64_t gen, const void* x, void* y,
+                         void* caller_stream, qe_tape* tapes_out) {
+  int32_t st = check_chain(layers, n);
+  if (st != QE_OK) return st;
+  if (!x || !y || !tapes_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (((uintptr_t)x | (uintptr_t)y) & 15u) return fail(QE_ERR_BAD_ARG, "x and y must be 16-byte aligned");
+  int32_t refresh[QE_MAX_CHAIN];
+  uint32_t p[QE_MAX_CHAIN];
+  for (uint32_t i = 0; i < n; ++i)  // every layer's check before anything runs
+    if ((st = qe_contract_forward_check(layers[i]->contract, mb, gen, &refresh[i], &p[i])) != QE_OK) return st;
+  qe_ctx* ctx = layers[0]->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  std::vector<qe::Launch> ls;
+  Fnv h;
+  h.mix("Fchain", 7);
+  for (uint32_t i = 0; i < n; ++i) {
+    qe_layer* L = layers[i];
+    if (L->dw_pending[p[i]]) {
+      QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[p[i]], 0));
+      L->dw_pending[p[i]] = false;
+    }
+    if (refresh[i]) add_refresh(L, ls);
+    h.mix(&layers[i], sizeof(qe_layer*));
+    h.mix(&p[i], sizeof(uint32_t));
+    h.mix(&refresh[i], sizeof(int32_t));
+  }
+  for (uint32_t i = 0; i < n; ++i) {
+    const bool last = i + 1 == n;
+    add_forward(layers[i], p[i], i == 0 ? x : nullptr, last ? y : nullptr, ls, last ? nullptr : layers[i + 1], last ? 0 : p[i + 1]);
+  }
+  if ((st = run_keyed(ctx, h.key, ls)) != QE_OK) return st;
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  for (uint32_t i = 0; i < n; ++i)
+    if ((st = qe_contract_forward_commit(layers[i]->contract, mb, &tapes_out[i])) != QE_OK) return st;
+  return QE_OK;
+}
+
+int32_t qe_backward_dI_chain(qe_layer* const* layers, const qe_tape* tapes, uint32_t n, const void* dy, void* dx,
+                             void* caller_stream) {
+  int32_t st = check_chain(layers, n);
+  if (st != QE_OK) return st;
+  if (!tapes || !dy || !dx) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (((uintptr_t)dy | (uintptr_t)dx) & 15u) return fail(QE_ERR_BAD_ARG, "dy and dx must be 16-byte aligned");
+  for (uint32_t i = 0; i < n; ++i)
+    if ((st = qe_contract_dI_check(layers[i]->contract, &tapes[i])) != QE_OK) return st;
+  qe_ctx* ctx = layers[0]->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  std::vector<qe::Launch> ls;
+  Fnv h;
+  h.mix("Bchain", 7);
+  for (uint32_t k = n; k-- > 0;) {  // last linear first
+    const uint32_t pk = tapes[k].ref.slot;
+    add_dI(layers[k], pk, k + 1 == n ? dy : nullptr, k == 0 ? dx : nullptr, ls, k ? layers[k - 1] : nullptr,
+           k ? tapes[k - 1].ref.slot : 0);
+    h.mix(&layers[k], sizeof(qe_layer*));
+    h.mix(&pk, sizeof(uint32_t));
+  }
+  if ((st = run_keyed(ctx, h.key, ls)) != QE_OK) return st;
+  if (ctx->dw_stream)
+    for (uint32_t i = 0; i < n; ++i) QE_CUDA(cudaEventRecord(layers[i]->ev_di[tapes[i].ref.slot], ctx->exec_stream));
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  for (uint32_t i = 0; i < n; ++i)
+    if ((st = qe_contract_dI_commit(layers[i]->contract, &tapes[i])) != QE_OK) return st;
   return QE_OK;
 }
 
