@@ -1,7 +1,8 @@
 // Amax-history reduction and scale update as a device function, shared by the standalone commit kernel and by the
 // tails of the quantise and GEMM kernels (where the last block to finish performs it, saving a launch).
 //   hist[c][count mod H] = amax;  scale_c = fp8_max / max(hist[c]) / 2^margin;  scale_inv_c = 1 / scale_c
-// 256 threads take part: 64 per tensor class, all four classes in parallel, one barrier.  The maximum is taken on
+// 256 threads take part: 64 per tensor class, all four classes in parallel, one barrier.  The ring's maximum is kept
+// beside it so that a commit usually reads one entry instead of H.  The maximum is taken on
 // the bit patterns of the non-negative FP32 entries, which orders them like their values and lets a NaN or Inf
 // entry surface as "not finite" (scale then stays as it was, like for an all-zero window).
 #pragma once
@@ -29,8 +30,15 @@ __device__ __forceinline__ void commit_classes(const CommitParams& p, int tid, u
   if (active) {
     cnt = __ldcg(&st->count[c]);
     newest = p.amax_override ? (__float_as_uint(__ldcg(p.amax_override)) & 0x7fffffffu) : __ldcg(&st->pending_amax[c]);
+    const uint32_t wmax = __ldcg(&st->wmax[c]);  // maximum of the ring as it stands
     pos = cnt % p.H;
-    for (uint32_t i = g; i < p.H; i += 64) m = max(m, i == pos ? newest : __ldcg(h + i));
+    const uint32_t evicted = __ldcg(h + pos);
+    // The new maximum is known without reading the ring unless the entry that leaves was the maximum and the one
+    // that enters is smaller: only then is the ring scanned (exactly the same value either way).
+    if (newest >= wmax) m = newest;
+    else if (evicted < wmax) m = wmax;
+    else
+      for (uint32_t i = g; i < p.H; i += 64) m = max(m, i == pos ? newest : __ldcg(h + i));
   }
   m = __reduce_max_sync(0xffffffffu, m);
   if ((tid & 31) == 0) red[tid >> 5] = m;
@@ -40,6 +48,7 @@ __device__ __forceinline__ void commit_classes(const CommitParams& p, int tid, u
     h[pos] = newest;
     st->count[c] = cnt + 1;
     st->pending_amax[c] = 0;
+    st->wmax[c] = m;
     if (m != 0 && m < 0x7f800000u) {
       const float fp8_max = c == 2 ? 57344.0f : 448.0f;  // class 2 = gradients (E5M2), others E4M3
       float s = __fmul_rn(__fdiv_rn(fp8_max, __uint_as_float(m)), p.pow2_neg_margin);

@@ -22,7 +22,8 @@ struct DevState {
   float slot_sinv_X[64];       // inverse scales snapshotted when X_m / dY_m were quantised (per tape slot)
   float slot_sinv_G[64];
   uint32_t ticket;             // "last CTA" counter of the kernel whose tail performs the commit; self-resetting
-  uint32_t pad[43];            // header is 768 bytes; history rings [4][H] follow
+  uint32_t wmax[4];            // bit pattern of max(history ring) per class, kept by the commit (derived state)
+  uint32_t pad[39];            // header is 768 bytes; history rings [4][H] follow
 };
 static_assert(sizeof(DevState) == 768, "DevState layout");
 

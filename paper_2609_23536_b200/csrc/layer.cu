@@ -1407,6 +1407,11 @@ int32_t qe_state_load(qe_layer* L, const void* host_in, uint64_t bytes) {
     h.scale_inv[c] = hd.scale_inv[c];
     h.count[c] = hd.count[c];
     h.pending_amax[c] = 0;
+    // derived state: the maximum of the restored ring (bit patterns of non-negative values order like the values)
+    const uint32_t* ring = reinterpret_cast<const uint32_t*>((const char*)host_in + sizeof(hd)) + (size_t)c * hd.H;
+    uint32_t m = 0;
+    for (uint32_t i = 0; i < hd.H; ++i) m = ring[i] > m ? ring[i] : m;
+    h.wmax[c] = m;
   }
   h.cache_sinv_W = 0.0f;  // cache contents are rebuilt by the first forward
   QE_CUDA(cudaMemcpy(L->st, &h, sizeof(h), cudaMemcpyHostToDevice));
