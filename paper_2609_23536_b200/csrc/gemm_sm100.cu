@@ -155,6 +155,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
+}
+
 // Bulk tensor store of a shared-memory tile (issued by one lane), with group tracking.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
@@ -333,8 +337,22 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
   if (TWO) cluster_sync_all();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // Everything above (barriers, tensor memory) touched no global data and may overlap the previous kernel's tail;
-  // operands, scales and the destination may come from it, so wait for it here.
+  if (warp == 0 && lane == 0 && first_tile < num_tiles) {
+    // While the predecessor drains: pull the first ring-full of B tiles of this CTA's first tile towards L2.  A
+    // prefetch moves no data into the SM, so it is harmless even if the predecessor is still writing that operand.
+    const uint32_t tile = first_tile;
+    QE_TILE_PROBLEM();
+    uint32_t m0, n0;
+    tile_coords(local_tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
+    const int rb = (int)(n0 + (TWO ? rank * C::B_ROWS : 0u));
+    for (uint32_t kb = 0; kb < num_kb && kb < (uint32_t)STAGES; ++kb) {
+      const int ka = (int)(kb * BK);
+      if (p.b_mn) tma_prefetch_2d(&p.tmB, rb, ka);
+      else tma_prefetch_2d(&p.tmB, ka, rb);
+    }
+  }
+  // Everything above (barriers, tensor memory) touched no data a predecessor produces and may overlap the previous
+  // kernel's tail; operands, scales and the destination may come from it, so wait for it here.
   grid_dep_wait();
   grid_dep_launch();
   if (blockIdx.x == 0 && threadIdx.x == 64) {  // FP8 hand-off: the consumer's tape snapshot of its inverse scale
@@ -555,13 +573,14 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
       }
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
-    if (lane == 0) tma_store_wait_all();  // this warp's bulk stores have reached global memory
     const CommitParams* cm = ps.commit();
     if (cm && cm->st) {
-      // every epilogue thread of every CTA gets here (also after a timeout); the last CTA commits the scale state
+      // every epilogue thread of every CTA gets here (also after a timeout); the last CTA commits the scale state.
+      // The commit needs the amax atomics only, so it runs while this CTA's last bulk stores are still draining.
       if (last_block(&cm->st->ticket, gridDim.x, etid, last_flag, epi_bar_sync))
         commit_classes(*cm, etid, red, epi_bar_sync);
     }
+    if (lane == 0) tma_store_wait_all();  // this warp's bulk stores have reached global memory
   }
 
   tc_fence_before();
