@@ -102,12 +102,13 @@ class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
     def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False,
-                 group_dw=True, arena=False, chain=False):
+                 group_dw=True, arena=False, chain=False, pair_f_di=True):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
         self.group_dw = group_dw and not staged and not arena
         self.chain = chain
+        self.pair_f_di = pair_f_di and not chain and not host_io
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
                               exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
@@ -181,8 +182,26 @@ class Stage:
         tapes = {}
         n = len(self.layers)
         t_issue = time.perf_counter()
-        for a, m in self.schedule:
+        skip = False
+        for k, (a, m) in enumerate(self.schedule):
+            if skip:  # this dI went out together with the forward before it
+                skip = False
+                continue
             order = range(n) if a == "F" else range(n - 1, -1, -1)
+            if (self.pair_f_di and not host_io and a == "F" and k + 1 < len(self.schedule) and self.schedule[k + 1][0] == "dI"):
+                # steady state: a forward unit and an input-gradient unit are both at hand; F of linear i goes out
+                # with dI of linear n-1-i (the two chains are independent), one shared GEMM launch per pair
+                mb_b = self.schedule[k + 1][1]
+                for i in range(n):
+                    j = n - 1 - i
+                    if i == j:
+                        tapes[(m, i)] = self.layers[i].forward(m, self.epoch, self.X[m][i], self.Y[m][i])
+                        self.layers[j].backward_dI(tapes[(mb_b, j)], self.dY[mb_b][j], self.dX[mb_b][j])
+                    else:
+                        tapes[(m, i)] = self.qe.forward_dI_pair(self.layers[i], m, self.epoch, self.X[m][i], self.Y[m][i],
+                                                                 self.layers[j], tapes[(mb_b, j)], self.dY[mb_b][j], self.dX[mb_b][j])
+                skip = True
+                continue
             if self.chain and a != "dW" and not host_io:
                 # the linears as directly chained groups of up to 16 (FP8 hand-off: one cast per group and direction)
                 for g in (self.groups if a == "F" else reversed(self.groups)):
@@ -479,6 +498,8 @@ def main():
                          "Default: one C-ABI call per action with dW overlapped on the context's second stream")
     ap.add_argument("--no-group-dw", dest="group_dw", action="store_false",
                     help="one qe_backward_dW call per linear instead of qe_backward_dW_multi per microbatch")
+    ap.add_argument("--no-pair-f-di", dest="pair_f_di", action="store_false",
+                    help="never issue a forward and the input gradient that follows it in the schedule as qe_forward_dI_pair calls")
     ap.add_argument("--chain", action="store_true",
                     help="treat consecutive linears whose shapes fit (K of the next = N of this) as directly chained: "
                          "qe_forward_chain / qe_backward_dI_chain with FP8 hand-off (config C5)")
@@ -516,7 +537,7 @@ def main():
 
     use_step = args.step_api
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
-                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain)
+                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain, pair_f_di=args.pair_f_di)
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:
@@ -532,7 +553,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "chained_fp8_handoff": bool(args.chain), "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "chained_fp8_handoff": bool(args.chain), "f_with_next_dI": "one shared GEMM launch per (F of linear i, dI of linear n-1-i)" if (args.pair_f_di and not args.chain and not args.step_api) else "separate", "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),

@@ -223,6 +223,15 @@ int32_t qe_backward_dW(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t 
  * to temp_dev (FP32 [N,K], caller-owned scratch) and then added into the destination by a second kernel. */
 int32_t qe_backward_dW_staged(qe_layer*, const qe_tape*, float* grad_buf_dev, uint64_t grad_buf_elems,
                               uint64_t offset, float* temp_dev, void* caller_stream);
+/* F of one layer and dI of another in one call (Sec. 4.2: in the steady state of a split-backward schedule a stage
+ * holds a forward unit and an input-gradient unit at once; their chains through the layers are independent).  The
+ * same checks, results (bit for bit) and state transitions as qe_forward(layer_f, mb, gen, x_dev, y_dev, stream,
+ * tape_out) followed by qe_backward_dI(layer_b, tape_b, dy_dev, dx_dev, stream), with the two GEMMs in one kernel
+ * launch where both can run on the paired-CTA variant (T a multiple of 256).  layer_f != layer_b, one context.  Both
+ * checks are made before anything runs: on a contract error nothing ran and neither layer's state changed. */
+int32_t qe_forward_dI_pair(qe_layer* layer_f, uint32_t mb, uint64_t gen, const void* x_dev, void* y_dev,
+                           qe_tape* tape_out, qe_layer* layer_b, const qe_tape* tape_b, const void* dy_dev,
+                           void* dx_dev, void* caller_stream);
 /* FP8 hand-off between directly chained linears (layers[i+1] consumes layers[i]'s output: same T,
  * K_{i+1} = N_i; host array of n <= QE_MAX_CHAIN distinct layers of one context).  qe_forward_chain runs F of every
  * layer for microbatch mb: x_dev bf16 [T, K_0] in, y_dev bf16 [T, N_{n-1}] out, tapes_out[n].  The output of
@@ -339,6 +348,7 @@ typedef struct qe_stats {
   double capture_host_ms;      /* host time spent building graphs                                             */
   uint64_t workspace_bytes;    /* sum over live layers                                                        */
   uint64_t grouped_dw;         /* weight-gradient GEMMs that shared a launch with other layers' (built launches)  */
+  uint64_t paired_f_di;        /* forward / input-gradient GEMM pairs that shared a launch                     */
 } qe_stats;
 int32_t qe_get_stats(const qe_ctx*, qe_stats* out);
 

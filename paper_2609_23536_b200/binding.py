@@ -97,7 +97,7 @@ class qe_stats(C.Structure):
     _fields_ = [
         ("graphs_built", C.c_uint64), ("graph_replays", C.c_uint64), ("eager_launches", C.c_uint64),
         ("handoffs", C.c_uint64), ("node_param_updates", C.c_uint64), ("kernels_launched", C.c_uint64),
-        ("capture_host_ms", C.c_double), ("workspace_bytes", C.c_uint64), ("grouped_dw", C.c_uint64),
+        ("capture_host_ms", C.c_double), ("workspace_bytes", C.c_uint64), ("grouped_dw", C.c_uint64), ("paired_f_di", C.c_uint64),
     ]
 
     def asdict(self):
@@ -135,6 +135,7 @@ _SIGNATURES = {
     "qe_backward_dI_host": (C.c_int32, [_P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
+    "qe_forward_dI_pair": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, C.POINTER(qe_tape), _P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_forward_chain": (C.c_int32, [C.POINTER(_P), C.c_uint32, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
     "qe_backward_dI_chain": (C.c_int32, [C.POINTER(_P), C.POINTER(qe_tape), C.c_uint32, _P, _P, _P]),
     "qe_backward_dW_arena": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, C.c_uint32, _P]),
@@ -479,6 +480,14 @@ def qe_noalloc_staging_elems() -> int:
 
 
 ACT = {"F": 0, "dI": 1, "dW": 2}
+
+
+def forward_dI_pair(layer_f, mb, gen, x, y, layer_b, tape_b, dy, dx, stream=None):
+    """qe_forward_dI_pair: F of layer_f and dI of layer_b (another layer) in one call; returns layer_f's tape."""
+    t = qe_tape()
+    _check(lib.qe_forward_dI_pair(layer_f.h, mb, gen, _ptr(x), _ptr(y), C.byref(t), layer_b.h, C.byref(tape_b),
+                                  _ptr(dy), _ptr(dx), _stream(stream)))
+    return t
 
 
 def forward_chain(layers, mb, gen, x, y, stream=None):

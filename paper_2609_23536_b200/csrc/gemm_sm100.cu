@@ -252,7 +252,8 @@ struct OneProblem {
     return p;
   }
   __device__ __forceinline__ const GemmParams& first() const { return p; }
-  __device__ __forceinline__ const CommitParams* commit() const { return &p.commit; }
+  __device__ __forceinline__ uint32_t count() const { return 1; }
+  __device__ __forceinline__ const CommitParams& commit(uint32_t) const { return p.commit; }
 };
 struct ProblemGroup {
   const GemmGroupParams& g;
@@ -264,7 +265,8 @@ struct ProblemGroup {
     return g.prob[i];
   }
   __device__ __forceinline__ const GemmParams& first() const { return g.prob[0]; }
-  __device__ __forceinline__ const CommitParams* commit() const { return nullptr; }
+  __device__ __forceinline__ uint32_t count() const { return g.n; }
+  __device__ __forceinline__ const CommitParams& commit(uint32_t i) const { return g.prob[i].commit; }
 };
 
 // ------------------------------------------------------------------------------------------------ kernel
@@ -573,12 +575,18 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
       }
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
-    const CommitParams* cm = ps.commit();
-    if (cm && cm->st) {
-      // every epilogue thread of every CTA gets here (also after a timeout); the last CTA commits the scale state.
-      // The commit needs the amax atomics only, so it runs while this CTA's last bulk stores are still draining.
-      if (last_block(&cm->st->ticket, gridDim.x, etid, last_flag, epi_bar_sync))
-        commit_classes(*cm, etid, red, epi_bar_sync);
+    // Every epilogue thread of every CTA gets here (also after a timeout); the last CTA commits the scale state of
+    // every problem that asks for it.  The commit needs the amax atomics only, so it runs while this CTA's last
+    // bulk stores are still draining.
+    uint32_t* ticket = nullptr;
+    for (uint32_t i = 0; i < ps.count(); ++i)
+      if (!ticket && ps.commit(i).st) ticket = &ps.commit(i).st->ticket;
+    if (ticket && last_block(ticket, gridDim.x, etid, last_flag, epi_bar_sync)) {
+      for (uint32_t i = 0; i < ps.count(); ++i) {
+        if (!ps.commit(i).st) continue;
+        commit_classes(ps.commit(i), etid, red, epi_bar_sync);
+        epi_bar_sync();  // the reduction words are reused by the next problem's commit
+      }
     }
     if (lane == 0) tma_store_wait_all();  // this warp's bulk stores have reached global memory
   }
@@ -641,7 +649,7 @@ bool make_gemm_group(const GemmParams* probs, uint32_t n, int num_sms, Launch* o
   GemmGroupParams g{};
   uint32_t tiles = 0;
   for (uint32_t i = 0; i < n; ++i) {
-    if (!gemm_uses_pair(probs[i].M) || probs[i].commit.st) return false;  // paired variant only, no commit tail
+    if (!gemm_uses_pair(probs[i].M)) return false;  // paired variant only
     tiles += (probs[i].M / 256u) * ((probs[i].N + BN - 1) / BN);
     g.tile_end[i] = tiles;
     g.prob[i] = probs[i];

@@ -133,8 +133,8 @@ Launch make_amax_pass2(const AmaxParams& p);
 Launch make_accumulate(const AccumParams& p);
 Launch make_arena_reduce(const ArenaReduceParams& p);
 Launch make_gemm(const GemmParams& p, int num_sms);
-// One launch for n = 2..4 GEMMs; false if the group cannot be formed (a problem needs the single-CTA variant or a
-// commit tail), in which case the caller launches them one by one.
+// One launch for n = 2..4 GEMMs (each may carry its own commit tail); false if the group cannot be formed (a problem
+// needs the single-CTA variant), in which case the caller launches them one by one.
 bool make_gemm_group(const GemmParams* probs, uint32_t n, int num_sms, Launch* out);
 cudaError_t gemm_prepare();  // opt in to the dynamic shared memory the GEMM needs (once per device)
 uint32_t gemm_idesc(int a_fmt, int b_fmt, uint32_t M, bool a_mn = false, bool b_mn = false);

@@ -467,8 +467,9 @@ void add_refresh(qe_layer* L, std::vector<qe::Launch>& ls) {
 // FP8 hand-off between directly chained linears: the forward GEMM of `L` emits its output as the E4M3 input of
 // `next` (quantised with next's current X scale, straight into next's tape slot pn, with next's X amax and
 // inverse-scale snapshot), so `next` needs no cast kernel; x == null means L's own input was deposited that way.
+// gemm_out != null: the GEMM is handed back instead of being queued (the caller puts it into a shared launch).
 void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe::Launch>& ls, qe_layer* next = nullptr,
-                 uint32_t pn = 0) {
+                 uint32_t pn = 0, qe::GemmParams* gemm_out = nullptr) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   if (x) ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
   qe::GemmParams gp{};
@@ -498,13 +499,14 @@ void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe
   gp.amax_bits = &L->st->pending_amax[QE_CLASS_Y];
   gp.status = &L->st->status;
   gp.commit = commit_params(L, (1u << QE_CLASS_X) | (1u << QE_CLASS_Y), 1, nullptr);  // done by the GEMM's last CTA
-  ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
+  if (gemm_out) *gemm_out = gp;
+  else ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
 }
 
 // Hand-off in the backward direction: the input gradient of `L` is the output gradient of the linear before it
 // (`prev`), emitted as E5M2 with prev's G scale into prev's tape slot pp; dy == null: L's own dY came that way.
 void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::Launch>& ls, qe_layer* prev = nullptr,
-            uint32_t pp = 0) {
+            uint32_t pp = 0, qe::GemmParams* gemm_out = nullptr) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
   if (dy) ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
   qe::GemmParams gp{};
@@ -536,7 +538,8 @@ void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::L
   gp.amax_bits = nullptr;
   gp.status = &L->st->status;
   gp.commit = commit_params(L, 1u << QE_CLASS_G, 1, nullptr);  // backward amax/scale updated exactly once, here
-  ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
+  if (gemm_out) *gemm_out = gp;
+  else ls.push_back(qe::make_gemm(gp, L->ctx->dev->num_sms));
 }
 
 // The weight-gradient GEMM of slot p; dst = first element of the layer's gradient slice, temp != null makes it
@@ -1137,6 +1140,55 @@ int32_t qe_backward_dI_chain(qe_layer* const* layers, const qe_tape* tapes, uint
   for (uint32_t i = 0; i < n; ++i)
     if ((st = qe_contract_dI_commit(layers[i]->contract, &tapes[i])) != QE_OK) return st;
   return QE_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ F and dI together
+// In the steady state of a split-backward schedule a stage holds a forward unit (microbatch m + k) and an input-
+// gradient unit (microbatch m) at the same time.  Their chains through the layers are independent, so F of layer i
+// and dI of layer j (two different layers) can share one GEMM launch: one fixed cost and common waves.
+int32_t qe_forward_dI_pair(qe_layer* Lf, uint32_t mb, uint64_t gen, const void* x, void* y, qe_tape* tape_out,
+                           qe_layer* Lb, const qe_tape* tape_b, const void* dy, void* dx, void* caller_stream) {
+  if (!Lf || !Lb || !x || !y || !tape_out || !tape_b || !dy || !dx) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (Lf == Lb || Lf->ctx != Lb->ctx) return fail(QE_ERR_BAD_ARG, "the two layers must be different layers of one context");
+  if (((uintptr_t)x | (uintptr_t)y | (uintptr_t)dy | (uintptr_t)dx) & 15u) return fail(QE_ERR_BAD_ARG, "tensors must be 16-byte aligned");
+  int32_t refresh = 0;
+  uint32_t p = 0;
+  int32_t st = qe_contract_forward_check(Lf->contract, mb, gen, &refresh, &p);  // both checks before anything runs
+  if (st != QE_OK) return st;
+  if ((st = qe_contract_dI_check(Lb->contract, tape_b)) != QE_OK) return st;
+  qe_ctx* ctx = Lf->ctx;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  const uint32_t pb = tape_b->ref.slot;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (Lf->dw_pending[p]) {
+    QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, Lf->ev_dw[p], 0));
+    Lf->dw_pending[p] = false;
+  }
+  std::vector<qe::Launch> ls;
+  if (refresh) add_refresh(Lf, ls);
+  qe::GemmParams g[2];
+  add_forward(Lf, p, x, y, ls, nullptr, 0, &g[0]);  // queues the two casts, hands the two GEMMs back
+  add_dI(Lb, pb, dy, dx, ls, nullptr, 0, &g[1]);
+  qe::Launch shared;
+  if (qe::make_gemm_group(g, 2, ctx->dev->num_sms, &shared)) {
+    ls.push_back(shared);
+    ctx->stats.paired_f_di += 1;
+  } else {  // a shape that needs the single-CTA variant: one after the other
+    ls.push_back(qe::make_gemm(g[0], ctx->dev->num_sms));
+    ls.push_back(qe::make_gemm(g[1], ctx->dev->num_sms));
+  }
+  Fnv h;
+  h.mix("FdI", 4);
+  h.mix(&Lf, sizeof(Lf));
+  h.mix(&Lb, sizeof(Lb));
+  h.mix(&p, sizeof(p));
+  h.mix(&pb, sizeof(pb));
+  h.mix(&refresh, sizeof(refresh));
+  if ((st = run_keyed(ctx, h.key, ls)) != QE_OK) return st;
+  if (ctx->dw_stream) QE_CUDA(cudaEventRecord(Lb->ev_di[pb], ctx->exec_stream));
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  if ((st = qe_contract_forward_commit(Lf->contract, mb, tape_out)) != QE_OK) return st;
+  return qe_contract_dI_commit(Lb->contract, tape_b);
 }
 
 // ------------------------------------------------------------------------------------------------ whole-step call

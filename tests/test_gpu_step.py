@@ -292,3 +292,82 @@ def test_two_chunk_schedules_split_equals_full_and_match_the_oracle(qe, gen, mod
             L.optimizer_boundary(M)
     for a, L in zip(st, orc):
         assert state_equal_except_Y(a, L.state())
+
+
+# ------------------------------------------------------------------------------------------ F and dI in one call
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+@pytest.mark.parametrize("overlap", [False, True], ids=["inline", "overlapped-dW"])
+def test_forward_dI_pair_equals_separate_calls_bitwise(qe, mode, overlap):
+    """Steady state of a split-backward schedule: F(m + 2) of linear i together with dI(m) of linear n-1-i."""
+    T, M = 256, 5
+    shapes = [(256, 512), (512, 256), (384, 384), (256, 768)]  # F and dI GEMMs have M = T = 256: all take the paired variant
+    n = len(shapes)
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in shapes])
+    s = sched(M, 2, 2)
+    results = []
+    for paired in (False, True):
+        ctx = qe.Context(mode, overlap_dw=overlap)
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, peak_live(s), inputs.weights("PR", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(shapes)]
+        grad = torch.full((total,), 1.5, device=DEV)
+        Y = [[torch.zeros((T, N), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        dX = [[torch.zeros((T, K), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        for step in range(2):
+            X = [[inputs.activations("PR", step, 0, j, m, T, K).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+            dY = [[inputs.upstream_grads("PR", step, 0, j, m, T, N).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+            tapes, skip = {}, False
+            for k, (a, m) in enumerate(s):
+                if skip:
+                    skip = False
+                    continue
+                if paired and a == "F" and k + 1 < len(s) and s[k + 1][0] == "dI":
+                    mb = s[k + 1][1]
+                    for i in range(n):
+                        j = n - 1 - i
+                        tapes[(m, i)] = qe.forward_dI_pair(layers[i], m, step, X[m][i], Y[m][i], layers[j], tapes[(mb, j)], dY[mb][j], dX[mb][j])
+                    skip = True
+                elif a == "F":
+                    for i in range(n):
+                        tapes[(m, i)] = layers[i].forward(m, step, X[m][i], Y[m][i])
+                elif a == "dI":
+                    for j in range(n - 1, -1, -1):
+                        layers[j].backward_dI(tapes[(m, j)], dY[m][j], dX[m][j])
+                else:
+                    qe.backward_dW_multi(layers, [tapes[(m, j)] for j in range(n)], grad, offs)
+            for L in layers:
+                L.optimizer_boundary(M)
+        torch.cuda.synchronize()
+        results.append(([inputs.bits(t.cpu()) for row in Y for t in row], [inputs.bits(t.cpu()) for row in dX for t in row],
+                        grad.cpu().numpy().copy(), [L.state() for L in layers], ctx.stats()))
+    a, b = results
+    for u, v in zip(a[0] + a[1], b[0] + b[1]):
+        assert np.array_equal(u, v)
+    assert np.array_equal(a[2].view(np.uint32), b[2].view(np.uint32))
+    for u, v in zip(a[3], b[3]):
+        assert state_equal(u, v) and u["device_token"] == v["device_token"]
+    n_pairs = sum(1 for k, (x, m) in enumerate(s) if x == "F" and k + 1 < len(s) and s[k + 1][0] == "dI")
+    assert n_pairs == 3
+    # every (i, n-1-i) pair shares a launch: one GEMM launch less per pair
+    assert b[4]["paired_f_di"] == 2 * n_pairs * n and a[4]["paired_f_di"] == 0
+    assert a[4]["kernels_launched"] - b[4]["kernels_launched"] == 2 * n_pairs * n
+
+
+def test_forward_dI_pair_checks_both_before_anything_runs(qe):
+    T = 256
+    ctx = qe.Context(0)
+    A = qe.Layer(ctx, T, 256, 512, 4, 0, 2, inputs.weights("PR", 0, 0, 512, 256).to(DEV), unit=0)
+    B = qe.Layer(ctx, T, 512, 256, 4, 0, 2, inputs.weights("PR", 0, 1, 256, 512).to(DEV), unit=1)
+    xa, ya = torch.zeros((T, 256), dtype=torch.bfloat16, device=DEV), torch.zeros((T, 512), dtype=torch.bfloat16, device=DEV)
+    xb, yb = torch.zeros((T, 512), dtype=torch.bfloat16, device=DEV), torch.zeros((T, 256), dtype=torch.bfloat16, device=DEV)
+    tb = B.forward(0, 0, xb, yb)
+    B.backward_dI(tb, yb, xb)
+    before = (A.state(), B.state())
+    with pytest.raises(qe.QEError) as e:  # B's tape already had its dI: A's forward must not run either
+        qe.forward_dI_pair(A, 0, 0, xa, ya, B, tb, yb, xb)
+    assert e.value.code == "DUP_CONSUME"
+    assert state_equal(before[0], A.state()) and state_equal(before[1], B.state())
+    with pytest.raises(qe.QEError) as e:
+        qe.forward_dI_pair(A, 0, 0, xa, ya, A, tb, yb, xb)
+    assert e.value.code == "BAD_ARG"
+    tb1 = B.forward(1, 0, xb, yb)
+    ta = qe.forward_dI_pair(A, 0, 0, xa, ya, B, tb1, yb, xb)
+    assert A.state()["token"] == 1 and B.state()["token"] == 4 and ta.key.mb == 0
