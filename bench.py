@@ -102,13 +102,14 @@ class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
     def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False,
-                 group_dw=True, arena=False, chain=False, pair_f_di=True):
+                 group_dw=True, arena=False, chain=False, pair_f_di=True, together=True):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
         self.group_dw = group_dw and not staged and not arena
         self.chain = chain
         self.pair_f_di = pair_f_di and not chain and not host_io
+        self.together = together and self.pair_f_di and not staged and not arena
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
                               exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
@@ -182,25 +183,38 @@ class Stage:
         tapes = {}
         n = len(self.layers)
         t_issue = time.perf_counter()
-        skip = False
+        skip = 0
         for k, (a, m) in enumerate(self.schedule):
-            if skip:  # this dI went out together with the forward before it
-                skip = False
+            if skip:  # this dI (and dW) went out together with the forward before it
+                skip -= 1
                 continue
             order = range(n) if a == "F" else range(n - 1, -1, -1)
             if (self.pair_f_di and not host_io and a == "F" and k + 1 < len(self.schedule) and self.schedule[k + 1][0] == "dI"):
                 # steady state: a forward unit and an input-gradient unit are both at hand; F of linear i goes out
                 # with dI of linear n-1-i (the two chains are independent), one shared GEMM launch per pair
                 mb_b = self.schedule[k + 1][1]
+                # ... and a deferred weight-gradient unit too, when the schedule has one next: its GEMM for linear i
+                # joins the same launch (qe_run_together), no second stream needed
+                mb_w = self.schedule[k + 2][1] if (self.together and k + 2 < len(self.schedule) and self.schedule[k + 2][0] == "dW") else None
                 for i in range(n):
                     j = n - 1 - i
+                    if mb_w is not None and i != j:
+                        acts = [("F", self.layers[i], m, self.epoch, self.X[m][i], self.Y[m][i]),
+                                ("dI", self.layers[j], tapes[(mb_b, j)], self.dY[mb_b][j], self.dX[mb_b][j]),
+                                ("dW", self.layers[i], tapes[(mb_w, i)], self.offsets[i])]
+                        tapes[(m, i)] = self.qe.run_together(self.ctx, acts, self.grad)[0]
+                        continue
                     if i == j:
                         tapes[(m, i)] = self.layers[i].forward(m, self.epoch, self.X[m][i], self.Y[m][i])
                         self.layers[j].backward_dI(tapes[(mb_b, j)], self.dY[mb_b][j], self.dX[mb_b][j])
                     else:
                         tapes[(m, i)] = self.qe.forward_dI_pair(self.layers[i], m, self.epoch, self.X[m][i], self.Y[m][i],
                                                                  self.layers[j], tapes[(mb_b, j)], self.dY[mb_b][j], self.dX[mb_b][j])
-                skip = True
+                skip = 1
+                if mb_w is not None:
+                    skip = 2
+                    if n % 2:  # the middle linear went out alone above: its weight gradient too
+                        self.layers[n // 2].backward_dW(tapes[(mb_w, n // 2)], self.grad, self.offsets[n // 2])
                 continue
             if self.chain and a != "dW" and not host_io:
                 # the linears as directly chained groups of up to 16 (FP8 hand-off: one cast per group and direction)
@@ -500,6 +514,8 @@ def main():
                     help="one qe_backward_dW call per linear instead of qe_backward_dW_multi per microbatch")
     ap.add_argument("--no-pair-f-di", dest="pair_f_di", action="store_false",
                     help="never issue a forward and the input gradient that follows it in the schedule as qe_forward_dI_pair calls")
+    ap.add_argument("--no-together", dest="together", action="store_false",
+                    help="keep the deferred dW out of the shared F + dI launches (it then goes to the second stream)")
     ap.add_argument("--chain", action="store_true",
                     help="treat consecutive linears whose shapes fit (K of the next = N of this) as directly chained: "
                          "qe_forward_chain / qe_backward_dI_chain with FP8 hand-off (config C5)")
@@ -537,7 +553,7 @@ def main():
 
     use_step = args.step_api
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
-                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain, pair_f_di=args.pair_f_di)
+                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain, pair_f_di=args.pair_f_di, together=args.together)
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:

@@ -232,6 +232,29 @@ int32_t qe_backward_dW_staged(qe_layer*, const qe_tape*, float* grad_buf_dev, ui
 int32_t qe_forward_dI_pair(qe_layer* layer_f, uint32_t mb, uint64_t gen, const void* x_dev, void* y_dev,
                            qe_tape* tape_out, qe_layer* layer_b, const qe_tape* tape_b, const void* dy_dev,
                            void* dx_dev, void* caller_stream);
+/* Several independent actions in one call (the general form of qe_forward_dI_pair and qe_backward_dW_multi): in
+ * the steady state of a split-backward schedule a stage holds a forward unit, an input-gradient unit and a deferred
+ * weight-gradient unit at once (Sec. 4.2), none of which depends on another.  The result -- outputs, gradient
+ * buffer, scale state, tapes -- is bit for bit that of issuing the actions one after the other in the order given;
+ * all GEMMs that can run on the paired-CTA variant share one kernel launch (forward and input-gradient tiles
+ * first, weight-gradient tiles after them).  1 <= n <= QE_MAX_TOGETHER; at most one
+ * action of a kind per layer; a dW action's tape must already have had its dI (ORDER otherwise, also when that dI
+ * is part of the same call).  Every check is made before anything runs: on a contract error nothing ran and no
+ * state changed.  Everything runs on the execution stream (weight gradients issued earlier on the context's second
+ * stream are waited for). */
+#define QE_MAX_TOGETHER 4
+typedef struct qe_action {
+  uint32_t kind;          /* QE_ACT_F, QE_ACT_DI or QE_ACT_DW                                                */
+  uint32_t mb;            /* F: microbatch                                                                   */
+  uint64_t gen;           /* F: the caller's view of the weight version                                      */
+  qe_layer* layer;
+  const void* in_dev;     /* F: x bf16 [T,K]; dI: dy bf16 [T,N]; dW: unused                                  */
+  void* out_dev;          /* F: y bf16 [T,N]; dI: dx bf16 [T,K]; dW: unused                                  */
+  qe_tape* tape;          /* F: receives the tape; dI, dW: the tape to consume                               */
+  uint64_t grad_offset;   /* dW: element offset of the layer's slice in grad_buf_dev                         */
+} qe_action;
+int32_t qe_run_together(qe_ctx*, qe_action* actions, uint32_t n, float* grad_buf_dev, uint64_t grad_buf_elems,
+                        void* caller_stream);
 /* FP8 hand-off between directly chained linears (layers[i+1] consumes layers[i]'s output: same T,
  * K_{i+1} = N_i; host array of n <= QE_MAX_CHAIN distinct layers of one context).  qe_forward_chain runs F of every
  * layer for microbatch mb: x_dev bf16 [T, K_0] in, y_dev bf16 [T, N_{n-1}] out, tapes_out[n].  The output of

@@ -106,6 +106,15 @@ class qe_stats(C.Structure):
 
 # every symbol include/qe.h declares, with its signature
 _P = C.c_void_p
+
+
+class qe_action(C.Structure):
+    _fields_ = [
+        ("kind", C.c_uint32), ("mb", C.c_uint32), ("gen", C.c_uint64), ("layer", _P), ("in_dev", _P), ("out_dev", _P),
+        ("tape", C.POINTER(qe_tape)), ("grad_offset", C.c_uint64),
+    ]
+
+
 _SIGNATURES = {
     "qe_registry_create": (C.c_int32, [C.POINTER(_P)]),
     "qe_registry_destroy": (C.c_int32, [_P]),
@@ -136,6 +145,7 @@ _SIGNATURES = {
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
     "qe_forward_dI_pair": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, C.POINTER(qe_tape), _P, C.POINTER(qe_tape), _P, _P, _P]),
+    "qe_run_together": (C.c_int32, [_P, C.POINTER(qe_action), C.c_uint32, _P, C.c_uint64, _P]),
     "qe_forward_chain": (C.c_int32, [C.POINTER(_P), C.c_uint32, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
     "qe_backward_dI_chain": (C.c_int32, [C.POINTER(_P), C.POINTER(qe_tape), C.c_uint32, _P, _P, _P]),
     "qe_backward_dW_arena": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, C.c_uint32, _P]),
@@ -488,6 +498,28 @@ def forward_dI_pair(layer_f, mb, gen, x, y, layer_b, tape_b, dy, dx, stream=None
     _check(lib.qe_forward_dI_pair(layer_f.h, mb, gen, _ptr(x), _ptr(y), C.byref(t), layer_b.h, C.byref(tape_b),
                                   _ptr(dy), _ptr(dx), _stream(stream)))
     return t
+
+
+def run_together(ctx, actions, grad_buf=None, stream=None):
+    """qe_run_together.  actions: ("F", layer, mb, gen, x, y) | ("dI", layer, tape, dy, dx) | ("dW", layer, tape, offset).
+    Returns the tapes of the F actions, in order."""
+    n = len(actions)
+    arr = (qe_action * n)()
+    new_tapes = []
+    for i, a in enumerate(actions):
+        if a[0] == "F":
+            _, L, mb, gen, x, y = a
+            t = qe_tape()
+            new_tapes.append(t)
+            arr[i] = qe_action(ACT["F"], mb, gen, L.h, _ptr(x), _ptr(y), C.pointer(t), 0)
+        elif a[0] == "dI":
+            _, L, tape, dy, dx = a
+            arr[i] = qe_action(ACT["dI"], 0, 0, L.h, _ptr(dy), _ptr(dx), C.pointer(tape), 0)
+        else:
+            _, L, tape, off = a
+            arr[i] = qe_action(ACT["dW"], 0, 0, L.h, None, None, C.pointer(tape), off)
+    _check(lib.qe_run_together(ctx.h, arr, n, _ptr(grad_buf), grad_buf.numel() if grad_buf is not None else 0, _stream(stream)))
+    return new_tapes
 
 
 def forward_chain(layers, mb, gen, x, y, stream=None):

@@ -1191,6 +1191,103 @@ int32_t qe_forward_dI_pair(qe_layer* Lf, uint32_t mb, uint64_t gen, const void* 
   return qe_contract_dI_commit(Lb->contract, tape_b);
 }
 
+// ------------------------------------------------------------------------------------------------ independent actions
+int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, void* caller_stream) {
+  if (!ctx || !acts || n == 0 || n > QE_MAX_TOGETHER) return fail(QE_ERR_BAD_ARG, "null argument or bad count %u", n);
+  bool any_dw = false;
+  for (uint32_t i = 0; i < n; ++i) {
+    const qe_action& a = acts[i];
+    if (a.kind > QE_ACT_DW || !a.layer || a.layer->ctx != ctx || !a.tape) return fail(QE_ERR_BAD_ARG, "action %u: bad kind, layer or tape", i);
+    if (a.kind != QE_ACT_DW && (!a.in_dev || !a.out_dev || (((uintptr_t)a.in_dev | (uintptr_t)a.out_dev) & 15u)))
+      return fail(QE_ERR_BAD_ARG, "action %u: input / output null or misaligned", i);
+    for (uint32_t j = 0; j < i; ++j)
+      if (acts[j].layer == a.layer && acts[j].kind == a.kind) return fail(QE_ERR_BAD_ARG, "actions %u and %u: same kind on the same layer", j, i);
+    any_dw |= a.kind == QE_ACT_DW;
+  }
+  if (any_dw && !grad) return fail(QE_ERR_BAD_ARG, "gradient buffer is null");
+  // check (every action, before anything runs) -> run -> commit
+  int32_t refresh[QE_MAX_TOGETHER] = {}, acc[QE_MAX_TOGETHER] = {};
+  uint32_t slot[QE_MAX_TOGETHER] = {};
+  int32_t st;
+  for (uint32_t i = 0; i < n; ++i) {
+    const qe_action& a = acts[i];
+    qe_layer* L = a.layer;
+    if (a.kind == QE_ACT_F) {
+      st = qe_contract_forward_check(L->contract, a.mb, a.gen, &refresh[i], &slot[i]);
+    } else if (a.kind == QE_ACT_DI) {
+      st = qe_contract_dI_check(L->contract, a.tape);
+      slot[i] = a.tape->ref.slot;
+    } else {
+      st = qe_contract_dW_check(L->contract, a.tape, (uint64_t)(uintptr_t)grad, grad_elems, a.grad_offset, (uint64_t)L->cfg.N * L->cfg.K, &acc[i]);
+      slot[i] = a.tape->ref.slot;
+    }
+    if (st != QE_OK) return st;
+  }
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (any_dw && ctx->dw_stream) {  // weight gradients issued earlier on the second stream accumulate into the same buffer
+    QE_CUDA(cudaEventRecord(ctx->ev_dw_in, ctx->dw_stream));
+    QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_dw_in, 0));
+  }
+  std::vector<qe::Launch> ls;
+  qe::GemmParams g[QE_MAX_TOGETHER];
+  uint32_t ng = 0, n_chain = 0, n_dw = 0;
+  Fnv h;
+  h.mix("together", 9);
+  for (int pass = 0; pass < 2; ++pass) {  // F and dI first (others wait for them), the weight gradients' tiles after theirs
+    for (uint32_t i = 0; i < n; ++i) {
+      const qe_action& a = acts[i];
+      qe_layer* L = a.layer;
+      if ((a.kind == QE_ACT_DW) != (pass == 1)) continue;
+      qe::GemmParams gp;
+      if (a.kind == QE_ACT_F) {
+        if (L->dw_pending[slot[i]]) {
+          QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[slot[i]], 0));
+          L->dw_pending[slot[i]] = false;
+        }
+        if (refresh[i]) add_refresh(L, ls);
+        add_forward(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp);
+      } else if (a.kind == QE_ACT_DI) {
+        add_dI(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp);
+      } else {
+        gp = dW_gemm(L, slot[i], grad + a.grad_offset, acc[i], nullptr);
+      }
+      if (qe::gemm_uses_pair(gp.M)) {
+        g[ng++] = gp;
+        (a.kind == QE_ACT_DW ? n_dw : n_chain) += 1;
+      } else {
+        ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));  // single-CTA variant: a launch of its own
+      }
+      h.mix(&a.kind, sizeof(a.kind));
+      h.mix(&a.layer, sizeof(a.layer));
+      h.mix(&slot[i], sizeof(uint32_t));
+      h.mix(&refresh[i], sizeof(int32_t));
+    }
+  }
+  qe::Launch shared;
+  if (ng >= 2 && qe::make_gemm_group(g, ng, ctx->dev->num_sms, &shared)) {
+    ls.push_back(shared);
+    ctx->stats.grouped_dw += n_dw;
+    ctx->stats.paired_f_di += n_chain >= 1 ? 1 : 0;
+  } else {
+    for (uint32_t i = 0; i < ng; ++i) ls.push_back(qe::make_gemm(g[i], ctx->dev->num_sms));
+  }
+  if ((st = run_keyed(ctx, h.key, ls)) != QE_OK) return st;
+  if (ctx->dw_stream)
+    for (uint32_t i = 0; i < n; ++i)
+      if (acts[i].kind == QE_ACT_DI) QE_CUDA(cudaEventRecord(acts[i].layer->ev_di[slot[i]], ctx->exec_stream));
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  for (uint32_t i = 0; i < n; ++i) {
+    const qe_action& a = acts[i];
+    qe_layer* L = a.layer;
+    if (a.kind == QE_ACT_F) st = qe_contract_forward_commit(L->contract, a.mb, a.tape);
+    else if (a.kind == QE_ACT_DI) st = qe_contract_dI_commit(L->contract, a.tape);
+    else st = qe_contract_dW_commit(L->contract, a.tape, (uint64_t)(uintptr_t)grad, a.grad_offset, (uint64_t)L->cfg.N * L->cfg.K);
+    if (st != QE_OK) return st;
+  }
+  return QE_OK;
+}
+
 // ------------------------------------------------------------------------------------------------ whole-step call
 int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, const qe_step_action* actions,
                     uint32_t n_actions, uint32_t M, const qe_step_io* io, float* grad, uint64_t grad_elems,

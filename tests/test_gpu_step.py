@@ -371,3 +371,89 @@ def test_forward_dI_pair_checks_both_before_anything_runs(qe):
     tb1 = B.forward(1, 0, xb, yb)
     ta = qe.forward_dI_pair(A, 0, 0, xa, ya, B, tb1, yb, xb)
     assert A.state()["token"] == 1 and B.state()["token"] == 4 and ta.key.mb == 0
+
+
+# ------------------------------------------------------------------------------------------ independent actions together
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_run_together_equals_one_action_after_the_other_bitwise(qe, mode):
+    """F(m + 2) of linear i, dI(m) of linear n-1-i and the deferred dW(m - 1) of linear i in one call each."""
+    T, M = 256, 6
+    shapes = [(256, 512), (512, 256), (384, 384), (256, 768)]
+    n = len(shapes)
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in shapes])
+    s = sched(M, 2, 1)  # F0 F1 | F2 dI0 | F3 dI1 dW0 | ... : triples from the third round on
+    results = []
+    for together in (False, True):
+        ctx = qe.Context(mode)
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, peak_live(s), inputs.weights("TG", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(shapes)]
+        grad = torch.full((total,), -2.5, device=DEV)
+        Y = [[torch.zeros((T, N), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        dX = [[torch.zeros((T, K), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        for step in range(2):
+            X = [[inputs.activations("TG", step, 0, j, m, T, K).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+            dY = [[inputs.upstream_grads("TG", step, 0, j, m, T, N).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+            tapes, skip, k = {}, 0, 0
+            while k < len(s):
+                a, m = s[k]
+                triple = together and a == "F" and k + 2 < len(s) and s[k + 1][0] == "dI" and s[k + 2][0] == "dW"
+                if triple:
+                    mb, mw = s[k + 1][1], s[k + 2][1]
+                    for i in range(n):
+                        j = n - 1 - i
+                        acts = [("F", layers[i], m, step, X[m][i], Y[m][i]), ("dI", layers[j], tapes[(mb, j)], dY[mb][j], dX[mb][j]),
+                                ("dW", layers[i], tapes[(mw, i)], offs[i])]
+                        tapes[(m, i)] = qe.run_together(ctx, acts, grad)[0]
+                    k += 3
+                    continue
+                if a == "F":
+                    for i in range(n):
+                        tapes[(m, i)] = layers[i].forward(m, step, X[m][i], Y[m][i])
+                elif a == "dI":
+                    for j in range(n - 1, -1, -1):
+                        layers[j].backward_dI(tapes[(m, j)], dY[m][j], dX[m][j])
+                else:
+                    for i in range(n):
+                        layers[i].backward_dW(tapes[(m, i)], grad, offs[i])
+                k += 1
+            for L in layers:
+                L.optimizer_boundary(M)
+        torch.cuda.synchronize()
+        results.append(([inputs.bits(t.cpu()) for row in Y for t in row], [inputs.bits(t.cpu()) for row in dX for t in row],
+                        grad.cpu().numpy().copy(), [L.state() for L in layers], ctx.stats()))
+    a, b = results
+    for u, v in zip(a[0] + a[1], b[0] + b[1]):
+        assert np.array_equal(u, v)
+    assert np.array_equal(a[2].view(np.uint32), b[2].view(np.uint32))
+    assert not np.any(b[2] == -2.5)
+    for u, v in zip(a[3], b[3]):
+        assert state_equal({**u, "slots": []}, {**v, "slots": []}) and u["device_token"] == v["device_token"]
+    n_triples = sum(1 for k in range(len(s) - 2) if s[k][0] == "F" and s[k + 1][0] == "dI" and s[k + 2][0] == "dW")
+    assert n_triples == 3
+    # per triple call three GEMM launches became one, except for the 384-wide linear whose dW takes the single-CTA variant
+    assert a[4]["kernels_launched"] - b[4]["kernels_launched"] == 2 * n_triples * (2 * n - 1)
+    assert b[4]["grouped_dw"] == 2 * n_triples * (n - 1)
+
+
+def test_run_together_is_all_or_nothing(qe):
+    T = 256
+    ctx = qe.Context(0)
+    A = qe.Layer(ctx, T, 256, 512, 4, 0, 2, inputs.weights("TG", 0, 0, 512, 256).to(DEV), unit=0)
+    B = qe.Layer(ctx, T, 512, 256, 4, 0, 2, inputs.weights("TG", 0, 1, 256, 512).to(DEV), unit=1)
+    grad = torch.full((2 * 512 * 256,), float("nan"), device=DEV)
+    xa, ya = torch.ones((T, 256), dtype=torch.bfloat16, device=DEV), torch.zeros((T, 512), dtype=torch.bfloat16, device=DEV)
+    xb, yb = torch.ones((T, 512), dtype=torch.bfloat16, device=DEV), torch.zeros((T, 256), dtype=torch.bfloat16, device=DEV)
+    tb = B.forward(0, 0, xb, yb)
+    before = (A.state(), B.state())
+    # B's dW in the same call as its dI: ORDER, and A's forward must not have run
+    with pytest.raises(qe.QEError) as e:
+        qe.run_together(ctx, [("F", A, 0, 0, xa, ya), ("dI", B, tb, yb, xb), ("dW", B, tb, 512 * 256)], grad)
+    assert e.value.code == "ORDER"
+    torch.cuda.synchronize()
+    assert state_equal(before[0], A.state()) and state_equal(before[1], B.state()) and torch.all(torch.isnan(grad)).item()
+    with pytest.raises(qe.QEError) as e:
+        qe.run_together(ctx, [("F", A, 0, 0, xa, ya), ("F", A, 1, 0, xa, ya)], grad)
+    assert e.value.code == "BAD_ARG"
+    (ta,) = qe.run_together(ctx, [("F", A, 0, 0, xa, ya), ("dI", B, tb, yb, xb)])
+    qe.run_together(ctx, [("dI", A, ta, ya, xa), ("dW", B, tb, 512 * 256)], grad)
+    torch.cuda.synchronize()
+    assert not torch.any(torch.isnan(grad[512 * 256:])).item() and torch.all(torch.isnan(grad[: 512 * 256])).item()
