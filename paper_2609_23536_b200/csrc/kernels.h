@@ -51,6 +51,12 @@ struct QuantParams {
 };
 
 
+struct QuantPairParams {
+  QuantParams q[2];            // neither carries a commit tail
+  uint32_t blocks0;            // blocks of the first cast
+  uint32_t pad[3];
+};
+
 struct AmaxParams {
   const uint4* x;              // bf16, 8 per vector
   uint64_t nvec;
@@ -127,6 +133,7 @@ struct Launch {
 };
 
 Launch make_quantize(const QuantParams& p);
+Launch make_quantize_pair(const QuantParams& a, const QuantParams& b);
 Launch make_commit(const CommitParams& p);
 Launch make_amax_pass1(const AmaxParams& p);
 Launch make_amax_pass2(const AmaxParams& p);

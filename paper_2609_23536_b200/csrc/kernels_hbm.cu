@@ -57,16 +57,15 @@ __device__ __forceinline__ void transpose4x4(const uint32_t a0, const uint32_t a
 // bytes of every output row of the transposed copy).
 constexpr int kQuantThreads = 256;
 
+// One block's share (256 rows x 64 columns at block coordinates bx, by) of a cast; wmax: 8 shared words.
 template <int FMT>
-__global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_constant__ QuantParams p) {
+__device__ __forceinline__ void quantize_block(const QuantParams& p, uint32_t bx, uint32_t by, uint32_t* wmax) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rb = lane >> 3, cv = lane & 7;
-  const uint32_t row0 = blockIdx.y * 256u + warp * 32u + rb * 8u;
-  const uint32_t col0 = blockIdx.x * 64u + cv * 8u;
-  grid_dep_wait();  // the scale (and possibly x) come from earlier kernels
-  grid_dep_launch();
+  const uint32_t row0 = by * 256u + warp * 32u + rb * 8u;
+  const uint32_t col0 = bx * 64u + cv * 8u;
   const float scale = *p.scale;
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && p.sinv_dst) *p.sinv_dst = *p.sinv_src;
+  if (bx == 0 && by == 0 && threadIdx.x == 0 && p.sinv_dst) *p.sinv_dst = *p.sinv_src;
 
   uint32_t m = 0;
   if (row0 < p.rows) {  // warp-uniform up to rb; rows is a multiple of 8 so a thread's 8 rows are all in or out
@@ -98,8 +97,6 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_co
       }
     }
   }
-  __shared__ uint32_t wmax[kQuantThreads / 32];
-  __shared__ uint32_t last_flag;
   if (p.amax_bits) {
     const uint32_t w = warp_max_u32(packed_to_f32bits(m));
     if (lane == 0) wmax[warp] = w;
@@ -111,11 +108,46 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_co
       if (b) atomicMax(p.amax_bits, b);
     }
   }
+}
+
+template <int FMT>
+__global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_constant__ QuantParams p) {
+  __shared__ uint32_t wmax[kQuantThreads / 32];
+  __shared__ uint32_t last_flag;
+  grid_dep_wait();  // the scale (and possibly x) come from earlier kernels
+  grid_dep_launch();
+  quantize_block<FMT>(p, blockIdx.x, blockIdx.y, wmax);
   if (p.commit.st) {  // the last block to finish folds the new amax into the history and updates the scale
     auto sync = [] { __syncthreads(); };
     if (last_block(&p.commit.st->ticket, gridDim.x * gridDim.y, threadIdx.x, &last_flag, sync))
       commit_classes(p.commit, threadIdx.x, wmax, sync);
   }
+}
+
+// Two independent casts in one launch (the X of a forward unit and the dY of an input-gradient unit that go out
+// together): blocks [0, blocks0) work on the first, the rest on the second.  No commit tails.
+__global__ void __launch_bounds__(kQuantThreads) quantize_pair_kernel(const __grid_constant__ QuantPairParams pp) {
+  __shared__ uint32_t wmax[kQuantThreads / 32];
+  grid_dep_wait();
+  grid_dep_launch();
+  const uint32_t which = blockIdx.x >= pp.blocks0 ? 1u : 0u;
+  const QuantParams& p = pp.q[which];
+  const uint32_t b = blockIdx.x - (which ? pp.blocks0 : 0u), bxn = p.cols / 64u;
+  if (p.fmt == 0) quantize_block<0>(p, b % bxn, b / bxn, wmax);
+  else quantize_block<1>(p, b % bxn, b / bxn, wmax);
+}
+
+Launch make_quantize_pair(const QuantParams& a, const QuantParams& b) {
+  QuantPairParams pp{};
+  pp.q[0] = a;
+  pp.q[1] = b;
+  pp.blocks0 = (a.cols / 64) * ((a.rows + 255) / 256);
+  Launch l;
+  l.func = (const void*)quantize_pair_kernel;
+  l.grid = dim3(pp.blocks0 + (b.cols / 64) * ((b.rows + 255) / 256), 1, 1);
+  l.block = dim3(kQuantThreads, 1, 1);
+  l.set(pp);
+  return l;
 }
 
 Launch make_quantize(const QuantParams& p) {

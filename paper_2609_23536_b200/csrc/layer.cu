@@ -439,8 +439,8 @@ qe::CommitParams commit_params(qe_layer* L, uint32_t mask, uint32_t bump, const 
 }
 
 // commit_mask != 0: the kernel's last block also commits those classes (used for the weight refresh)
-qe::Launch quant_launch(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uint32_t rows, uint32_t cols, int cls,
-                        float* sinv_dst, int fmt, uint32_t commit_mask = 0) {
+qe::QuantParams quant_params(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uint32_t rows, uint32_t cols, int cls,
+                             float* sinv_dst, int fmt, uint32_t commit_mask = 0) {
   qe::QuantParams qp{};
   qp.x = (const uint16_t*)x;
   qp.q = q;
@@ -453,7 +453,11 @@ qe::Launch quant_launch(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uin
   qp.amax_bits = &L->st->pending_amax[cls];
   qp.fmt = fmt;
   if (commit_mask) qp.commit = commit_params(L, commit_mask, 0, nullptr);
-  return qe::make_quantize(qp);
+  return qp;
+}
+qe::Launch quant_launch(qe_layer* L, const void* x, uint8_t* q, uint8_t* qT, uint32_t rows, uint32_t cols, int cls,
+                        float* sinv_dst, int fmt, uint32_t commit_mask = 0) {
+  return qe::make_quantize(quant_params(L, x, q, qT, rows, cols, cls, sinv_dst, fmt, commit_mask));
 }
 
 
@@ -469,9 +473,10 @@ void add_refresh(qe_layer* L, std::vector<qe::Launch>& ls) {
 // inverse-scale snapshot), so `next` needs no cast kernel; x == null means L's own input was deposited that way.
 // gemm_out != null: the GEMM is handed back instead of being queued (the caller puts it into a shared launch).
 void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe::Launch>& ls, qe_layer* next = nullptr,
-                 uint32_t pn = 0, qe::GemmParams* gemm_out = nullptr) {
+                 uint32_t pn = 0, qe::GemmParams* gemm_out = nullptr, qe::QuantParams* cast_out = nullptr) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
-  if (x) ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
+  if (x && cast_out) *cast_out = quant_params(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3);
+  else if (x) ls.push_back(quant_launch(L, x, L->Xq[p], L->XqT[p], T, K, QE_CLASS_X, &L->st->slot_sinv_X[p], QE_E4M3));
   qe::GemmParams gp{};
   gp.tmA = L->tmXq_A[p];
   gp.tmB = L->tmWq_B;
@@ -506,9 +511,10 @@ void add_forward(qe_layer* L, uint32_t p, const void* x, void* y, std::vector<qe
 // Hand-off in the backward direction: the input gradient of `L` is the output gradient of the linear before it
 // (`prev`), emitted as E5M2 with prev's G scale into prev's tape slot pp; dy == null: L's own dY came that way.
 void add_dI(qe_layer* L, uint32_t p, const void* dy, void* dx, std::vector<qe::Launch>& ls, qe_layer* prev = nullptr,
-            uint32_t pp = 0, qe::GemmParams* gemm_out = nullptr) {
+            uint32_t pp = 0, qe::GemmParams* gemm_out = nullptr, qe::QuantParams* cast_out = nullptr) {
   const uint32_t T = L->cfg.T, K = L->cfg.K, N = L->cfg.N;
-  if (dy) ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
+  if (dy && cast_out) *cast_out = quant_params(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2);
+  else if (dy) ls.push_back(quant_launch(L, dy, L->Gq[p], L->GqT[p], T, N, QE_CLASS_G, &L->st->slot_sinv_G[p], QE_E5M2));
   qe::GemmParams gp{};
   const bool b_mn = L->WqT == nullptr;  // no transposed weight copy: Wq [N,K] is B in MN-major form
   gp.tmA = L->tmGq_A[p];
@@ -1167,8 +1173,10 @@ int32_t qe_forward_dI_pair(qe_layer* Lf, uint32_t mb, uint64_t gen, const void* 
   std::vector<qe::Launch> ls;
   if (refresh) add_refresh(Lf, ls);
   qe::GemmParams g[2];
-  add_forward(Lf, p, x, y, ls, nullptr, 0, &g[0]);  // queues the two casts, hands the two GEMMs back
-  add_dI(Lb, pb, dy, dx, ls, nullptr, 0, &g[1]);
+  qe::QuantParams c[2];
+  add_forward(Lf, p, x, y, ls, nullptr, 0, &g[0], &c[0]);  // hands the casts and the GEMMs back
+  add_dI(Lb, pb, dy, dx, ls, nullptr, 0, &g[1], &c[1]);
+  ls.push_back(qe::make_quantize_pair(c[0], c[1]));  // both casts in one launch
   qe::Launch shared;
   if (qe::make_gemm_group(g, 2, ctx->dev->num_sms, &shared)) {
     ls.push_back(shared);
@@ -1231,7 +1239,9 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
   }
   std::vector<qe::Launch> ls;
   qe::GemmParams g[QE_MAX_TOGETHER];
-  uint32_t ng = 0, n_chain = 0, n_dw = 0;
+  qe::QuantParams casts[QE_MAX_TOGETHER];
+  std::vector<qe::GemmParams> singles;
+  uint32_t ng = 0, n_chain = 0, n_dw = 0, n_casts = 0;
   Fnv h;
   h.mix("together", 9);
   for (int pass = 0; pass < 2; ++pass) {  // F and dI first (others wait for them), the weight gradients' tiles after theirs
@@ -1246,9 +1256,9 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
           L->dw_pending[slot[i]] = false;
         }
         if (refresh[i]) add_refresh(L, ls);
-        add_forward(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp);
+        add_forward(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp, &casts[n_casts++]);
       } else if (a.kind == QE_ACT_DI) {
-        add_dI(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp);
+        add_dI(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp, &casts[n_casts++]);
       } else {
         gp = dW_gemm(L, slot[i], grad + a.grad_offset, acc[i], nullptr);
       }
@@ -1256,7 +1266,7 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
         g[ng++] = gp;
         (a.kind == QE_ACT_DW ? n_dw : n_chain) += 1;
       } else {
-        ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));  // single-CTA variant: a launch of its own
+        singles.push_back(gp);  // single-CTA variant: a launch of its own
       }
       h.mix(&a.kind, sizeof(a.kind));
       h.mix(&a.layer, sizeof(a.layer));
@@ -1264,6 +1274,9 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
       h.mix(&refresh[i], sizeof(int32_t));
     }
   }
+  for (uint32_t i = 0; i + 1 < n_casts; i += 2) ls.push_back(qe::make_quantize_pair(casts[i], casts[i + 1]));  // casts two by two
+  if (n_casts & 1u) ls.push_back(qe::make_quantize(casts[n_casts - 1]));
+  for (const qe::GemmParams& gp : singles) ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
   qe::Launch shared;
   if (ng >= 2 && qe::make_gemm_group(g, ng, ctx->dev->num_sms, &shared)) {
     ls.push_back(shared);

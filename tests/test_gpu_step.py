@@ -348,7 +348,7 @@ def test_forward_dI_pair_equals_separate_calls_bitwise(qe, mode, overlap):
     assert n_pairs == 3
     # every (i, n-1-i) pair shares a launch: one GEMM launch less per pair
     assert b[4]["paired_f_di"] == 2 * n_pairs * n and a[4]["paired_f_di"] == 0
-    assert a[4]["kernels_launched"] - b[4]["kernels_launched"] == 2 * n_pairs * n
+    assert a[4]["kernels_launched"] - b[4]["kernels_launched"] == 2 * n_pairs * n * 2  # one GEMM and one cast launch less per pair
 
 
 def test_forward_dI_pair_checks_both_before_anything_runs(qe):
@@ -430,7 +430,7 @@ def test_run_together_equals_one_action_after_the_other_bitwise(qe, mode):
     n_triples = sum(1 for k in range(len(s) - 2) if s[k][0] == "F" and s[k + 1][0] == "dI" and s[k + 2][0] == "dW")
     assert n_triples == 3
     # per triple call three GEMM launches became one, except for the 384-wide linear whose dW takes the single-CTA variant
-    assert a[4]["kernels_launched"] - b[4]["kernels_launched"] == 2 * n_triples * (2 * n - 1)
+    assert a[4]["kernels_launched"] - b[4]["kernels_launched"] == 2 * n_triples * (2 * n - 1 + n)  # ... and the two casts became one
     assert b[4]["grouped_dw"] == 2 * n_triples * (n - 1)
 
 
