@@ -322,7 +322,7 @@ def gemm_roofline(qe, cfg, peaks, device):
     one = torch.ones(1, dtype=torch.float32, device=device)
     status = torch.zeros(1, dtype=torch.int32, device=device)
     tot_flops = tot_ms = 0.0
-    per = {}
+    per, per_shape_ms = {}, {}
     for name, M_, N_, Kc, af, amn, bmn, kind in shapes:
         nset = max(2, int(160e6 // (M_ * Kc + N_ * Kc + M_ * N_ * (2 if kind == 0 else 8))) + 1)
         nset = min(nset, 24)
@@ -344,10 +344,58 @@ def gemm_roofline(qe, cfg, peaks, device):
         fl = 2.0 * M_ * N_ * Kc
         tot_flops += fl
         tot_ms += ms
+        per_shape_ms[(name, M_, N_, Kc)] = ms
         per.setdefault(name, [0.0, 0.0])
         per[name][0] += fl
         per[name][1] += ms
         del A, B, D
+    assert status.item() == 0
+    # ... and the same twelve GEMMs in the launches the layer path issues in its steady state: F of linear i with dI
+    # of linear n-1-i in one launch each, the weight gradients of all linears in one launch
+    lin = cfg["linears"]
+    nl = len(lin)
+    groups = []
+    for i in range(nl):
+        j = nl - 1 - i
+        (_, Ki, Ni), (_, Kj, Nj) = lin[i], lin[j]
+        groups.append([("F", T, Ni, Ki, 0, 0, 0, 0), ("dI", T, Kj, Nj, 1, 0, 1, 0)] if i != j else [("F", T, Ni, Ki, 0, 0, 0, 0)])
+        if i == j:
+            groups.append([("dI", T, Kj, Nj, 1, 0, 1, 0)])
+    for lo in range(0, nl, 4):
+        groups.append([("dW", N, K, T, 1, 1, 1, 2) for _, K, N in lin[lo:lo + 4]])
+    g_flops = g_ms = 0.0
+    g_launches = 0
+    for grp in groups:
+        if any(M_ % 256 for _, M_, *_ in grp) or len(grp) < 2:  # shapes that cannot share a launch: one by one (timed above)
+            for name, M_, N_, Kc, *_ in grp:
+                g_flops += 2.0 * M_ * N_ * Kc
+            g_ms += sum(per_shape_ms[(name, M_, N_, Kc)] for name, M_, N_, Kc, *_ in grp)
+            g_launches += len(grp)
+            continue
+        nbytes = sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if kind == 0 else 8) for _, M_, N_, Kc, _, _, _, kind in grp)
+        nset = min(max(2, int(160e6 // nbytes) + 1), 12)
+        sets = []
+        for _ in range(nset):
+            ps = []
+            for name, M_, N_, Kc, af, amn, bmn, kind in grp:
+                ps.append((torch.randint(0, 120, (Kc, M_) if amn else (M_, Kc), dtype=torch.uint8, device=device), af, amn,
+                           torch.randint(0, 120, (Kc, N_) if bmn else (N_, Kc), dtype=torch.uint8, device=device), 0, bmn, one, one,
+                           torch.zeros((M_, N_), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=device), kind, None))
+            sets.append(ps)
+        for ps in sets:
+            qe.qe_gemm_fp8_group(ps, status)
+        torch.cuda.synchronize()
+        reps = 3 * nset
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for r in range(reps):
+            qe.qe_gemm_fp8_group(sets[r % nset], status)
+        e1.record()
+        torch.cuda.synchronize()
+        g_ms += e0.elapsed_time(e1) / reps
+        g_flops += sum(2.0 * M_ * N_ * Kc for _, M_, N_, Kc, *_ in grp)
+        g_launches += 1
+        del sets
     assert status.item() == 0
     lib = None
     try:  # context only: the vendor library's FP8 GEMM (cuBLASLt through torch._scaled_mm) on the forward shapes
@@ -370,19 +418,23 @@ def gemm_roofline(qe, cfg, peaks, device):
         lib = round(lf / (lm * 1e-3) / 1e12, 1)
     except Exception as e:  # noqa: BLE001
         lib = "unavailable: " + str(e)[:80]
-    achieved = tot_flops / (tot_ms * 1e-3) / 1e12
-    # dram__bytes_read + dram__bytes_write per launch, averaged over the twelve GEMMs of a microbatch, from one ncu
-    # capture of `python -m paper_2609_23536_b200.profile_case gemm_microbatch --small` (config-2 shapes only)
-    traffic = 39.6e6 if (T, tuple(cfg["linears"])) == (2048, tuple(inputs.CONFIGS["C2"]["linears"])) else None
+    single = tot_flops / (tot_ms * 1e-3) / 1e12
+    achieved = g_flops / (g_ms * 1e-3) / 1e12
+    # dram__bytes_read + dram__bytes_write per launch, averaged over the five launches of a microbatch, from one ncu
+    # capture of `python -m paper_2609_23536_b200.profile_case gemm_microbatch_grouped --small` (config-2 shapes only)
+    # (five launches: 445.0 MB read + 159.6 MB written)
+    traffic = 120.9e6 if (T, tuple(cfg["linears"])) == (2048, tuple(inputs.CONFIGS["C2"]["linears"])) and g_launches == 5 else None
     peak = 2.0 * peaks["bf16_burst"]  # FP8 dense = 2 x the bf16 peak (nominal ratio), kernels timed alone -> burst figure
     return {
-        "bound": "tensor", "kernel": "gemm_fp8_pair_kernel", "achieved": round(achieved, 1), "peak": round(peak, 1),
+        "bound": "tensor", "kernel": "gemm_fp8_pair_group_kernel (F + dI pairs, grouped dW: the launches of the steady state)",
+        "achieved": round(achieved, 1), "peak": round(peak, 1),
         "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": traffic,
-        "algorithmic_bytes_per_launch": round(sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if k == 0 else 8) for _, M_, N_, Kc, _, _, _, k in shapes) / len(shapes)),
-        "flop_per_launch": round(tot_flops / len(shapes)), "launches_timed": len(shapes), "peak_source": peaks["source"] + " bf16 burst x2",
+        "algorithmic_bytes_per_launch": round(sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if k == 0 else 8) for _, M_, N_, Kc, _, _, _, k in shapes) / g_launches),
+        "flop_per_launch": round(g_flops / g_launches), "launches_timed": g_launches, "peak_source": peaks["source"] + " bf16 burst x2",
         "frac_of_nominal_4500": round(achieved / 4500.0, 4),
+        "one_problem_per_launch_tflops": round(single, 1),
         "per_action_tflops": {k: round(v[0] / (v[1] * 1e-3) / 1e12, 1) for k, v in per.items()},
-        "gemm_ms_per_microbatch": round(tot_ms, 4),
+        "gemm_ms_per_microbatch": round(g_ms, 4),
         "vendor_library_fp8_forward_tflops_same_shapes": lib,
     }
 
@@ -569,7 +621,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action", "chained_fp8_handoff": bool(args.chain), "f_with_next_dI": "one shared GEMM launch per (F of linear i, dI of linear n-1-i)" if (args.pair_f_di and not args.chain and not args.step_api) else "separate", "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action; a forward and the input gradient (and deferred dW) that follow it in the schedule go out linear by linear through qe_forward_dI_pair / qe_run_together" if args.pair_f_di else "one C-ABI call per action", "chained_fp8_handoff": bool(args.chain), "f_with_next_dI": "one shared GEMM launch per (F of linear i, dI of linear n-1-i)" if (args.pair_f_di and not args.chain and not args.step_api) else "separate", "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),

@@ -407,6 +407,22 @@ int32_t qe_gemm_fp8_ex(const void* a_dev, uint32_t a_format, uint32_t a_mn, cons
                        const float* alpha_b_dev, void* d_dev, uint32_t out_kind, float* amax_dev, uint32_t* status_dev,
                        void* stream);
 
+/* Two to four independent FP8 GEMMs in ONE kernel launch (the launch shape the layer uses for F + dI pairs and for
+ * the weight gradients of a microbatch): the persistent CTAs work through the problems' tiles one problem after the
+ * other, so the launch cost is paid once and partial waves are shared.  Each problem as in qe_gemm_fp8_ex; every M
+ * must be a multiple of 256 (QE_ERR_UNSUPPORTED otherwise); outputs must not overlap.  descs: host array. */
+typedef struct qe_gemm_desc {
+  const void* a_dev;
+  const void* b_dev;
+  void* d_dev;
+  const float* alpha_a_dev;
+  const float* alpha_b_dev;
+  float* amax_dev;        /* out_kind 0 only; may be NULL */
+  uint32_t a_format, a_mn, b_format, b_mn;
+  uint32_t M, Nn, Kc, out_kind;
+} qe_gemm_desc;
+int32_t qe_gemm_fp8_group(const qe_gemm_desc* descs, uint32_t n, uint32_t* status_dev, void* stream);
+
 /* (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
  * The copied-gradient step without any allocation: D = (A . B^T) * *alpha_a_dev * *alpha_b_dev is written to a
  * staging area that is built into the library (a fixed device array of qe_noalloc_staging_elems() = 2^20 FP32

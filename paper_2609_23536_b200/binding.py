@@ -108,6 +108,14 @@ class qe_stats(C.Structure):
 _P = C.c_void_p
 
 
+class qe_gemm_desc(C.Structure):
+    _fields_ = [
+        ("a_dev", _P), ("b_dev", _P), ("d_dev", _P), ("alpha_a_dev", _P), ("alpha_b_dev", _P), ("amax_dev", _P),
+        ("a_format", C.c_uint32), ("a_mn", C.c_uint32), ("b_format", C.c_uint32), ("b_mn", C.c_uint32),
+        ("M", C.c_uint32), ("Nn", C.c_uint32), ("Kc", C.c_uint32), ("out_kind", C.c_uint32),
+    ]
+
+
 class qe_action(C.Structure):
     _fields_ = [
         ("kind", C.c_uint32), ("mb", C.c_uint32), ("gen", C.c_uint64), ("layer", _P), ("in_dev", _P), ("out_dev", _P),
@@ -145,6 +153,7 @@ _SIGNATURES = {
     "qe_backward_dW": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P]),
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
     "qe_forward_dI_pair": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, C.POINTER(qe_tape), _P, C.POINTER(qe_tape), _P, _P, _P]),
+    "qe_gemm_fp8_group": (C.c_int32, [C.POINTER(qe_gemm_desc), C.c_uint32, _P, _P]),
     "qe_run_together": (C.c_int32, [_P, C.POINTER(qe_action), C.c_uint32, _P, C.c_uint64, _P]),
     "qe_forward_chain": (C.c_int32, [C.POINTER(_P), C.c_uint32, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
     "qe_backward_dI_chain": (C.c_int32, [C.POINTER(_P), C.POINTER(qe_tape), C.c_uint32, _P, _P, _P]),
@@ -498,6 +507,18 @@ def forward_dI_pair(layer_f, mb, gen, x, y, layer_b, tape_b, dy, dx, stream=None
     _check(lib.qe_forward_dI_pair(layer_f.h, mb, gen, _ptr(x), _ptr(y), C.byref(t), layer_b.h, C.byref(tape_b),
                                   _ptr(dy), _ptr(dx), _stream(stream)))
     return t
+
+
+def qe_gemm_fp8_group(problems, status, stream=None):
+    """problems: 2..4 tuples (a, a_format, a_mn, b, b_format, b_mn, alpha_a, alpha_b, d, out_kind, amax or None);
+    shapes are taken from the tensors (MN-major operands are [Kc, rows])."""
+    n = len(problems)
+    arr = (qe_gemm_desc * n)()
+    for i, (a, af, amn, b, bf, bmn, sa, sb, d, kind, amax) in enumerate(problems):
+        M, Nn = d.shape
+        Kc = a.shape[0] if amn else a.shape[1]
+        arr[i] = qe_gemm_desc(_ptr(a), _ptr(b), _ptr(d), _ptr(sa), _ptr(sb), _ptr(amax), af, int(amn), bf, int(bmn), M, Nn, Kc, kind)
+    _check(lib.qe_gemm_fp8_group(arr, n, _ptr(status), _stream(stream)))
 
 
 def run_together(ctx, actions, grad_buf=None, stream=None):

@@ -1657,9 +1657,10 @@ int32_t qe_arena_reduce(const void* views, uint64_t view_elems, uint32_t M, floa
   return launch_on(qe::make_arena_reduce(ap), (cudaStream_t)stream);
 }
 
-int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void* b, uint32_t b_fmt, uint32_t b_mn,
-                       uint32_t M, uint32_t Nn, uint32_t Kc, const float* alpha_a, const float* alpha_b, void* d,
-                       uint32_t out_kind, float* amax_dev, uint32_t* status_dev, void* stream) {
+// Validates one standalone GEMM and fills its parameter block.
+static int32_t standalone_gemm(DeviceInfo* dev, const void* a, uint32_t a_fmt, uint32_t a_mn, const void* b, uint32_t b_fmt,
+                               uint32_t b_mn, uint32_t M, uint32_t Nn, uint32_t Kc, const float* alpha_a, const float* alpha_b,
+                               void* d, uint32_t out_kind, float* amax_dev, uint32_t* status_dev, qe::GemmParams* out) {
   if (!a || !b || !alpha_a || !alpha_b || !d || !status_dev) return fail(QE_ERR_BAD_ARG, "null argument");
   if (a_fmt > QE_E5M2 || b_fmt > QE_E5M2 || out_kind > 2 || a_mn > 1 || b_mn > 1) return fail(QE_ERR_BAD_ARG, "bad enum");
   if (!shape_ok(M) && M != 128) return fail(QE_ERR_SHAPE, "M=%u", M);
@@ -1667,9 +1668,7 @@ int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void*
   if ((a_mn || b_mn) && !qe::gemm_uses_pair(M))
     return fail(QE_ERR_UNSUPPORTED, "MN-major operands need M to be a multiple of 256 (paired-CTA variant), M=%u", M);
   if ((((uintptr_t)a | (uintptr_t)b | (uintptr_t)d) & 15u)) return fail(QE_ERR_BAD_ARG, "misaligned pointer");
-  DeviceInfo* dev = nullptr;
-  int32_t st = current_device_info(&dev);
-  if (st != QE_OK) return st;
+  int32_t st;
   qe::GemmParams gp{};
   // contraction-major operand: [rows, Kc]; MN-major operand: [Kc, rows] with a 128 x 128 box
   st = a_mn ? make_map(dev, &gp.tmA, a, Kc, M, 128) : make_map(dev, &gp.tmA, a, M, Kc, 128);
@@ -1690,7 +1689,38 @@ int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void*
   if ((st = make_out_map(dev, &gp.tmD, d, M, Nn, Nn, out_kind != 0)) != QE_OK) return st;
   gp.amax_bits = (uint32_t*)amax_dev;
   gp.status = status_dev;
+  *out = gp;
+  return QE_OK;
+}
+
+int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void* b, uint32_t b_fmt, uint32_t b_mn,
+                       uint32_t M, uint32_t Nn, uint32_t Kc, const float* alpha_a, const float* alpha_b, void* d,
+                       uint32_t out_kind, float* amax_dev, uint32_t* status_dev, void* stream) {
+  DeviceInfo* dev = nullptr;
+  int32_t st = current_device_info(&dev);
+  if (st != QE_OK) return st;
+  qe::GemmParams gp;
+  if ((st = standalone_gemm(dev, a, a_fmt, a_mn, b, b_fmt, b_mn, M, Nn, Kc, alpha_a, alpha_b, d, out_kind, amax_dev, status_dev, &gp)) != QE_OK) return st;
   return launch_on(qe::make_gemm(gp, dev->num_sms), (cudaStream_t)stream);
+}
+
+int32_t qe_gemm_fp8_group(const qe_gemm_desc* descs, uint32_t n, uint32_t* status_dev, void* stream) {
+  if (!descs || !status_dev) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (n < 2 || n > 4) return fail(QE_ERR_BAD_ARG, "a group holds 2 to 4 problems, got %u", n);
+  DeviceInfo* dev = nullptr;
+  int32_t st = current_device_info(&dev);
+  if (st != QE_OK) return st;
+  qe::GemmParams gp[4];
+  for (uint32_t i = 0; i < n; ++i) {
+    const qe_gemm_desc& q = descs[i];
+    if (!qe::gemm_uses_pair(q.M)) return fail(QE_ERR_UNSUPPORTED, "problem %u: M=%u is not a multiple of 256", i, q.M);
+    if ((st = standalone_gemm(dev, q.a_dev, q.a_format, q.a_mn, q.b_dev, q.b_format, q.b_mn, q.M, q.Nn, q.Kc, q.alpha_a_dev,
+                              q.alpha_b_dev, q.d_dev, q.out_kind, q.amax_dev, status_dev, &gp[i])) != QE_OK)
+      return st;
+  }
+  qe::Launch l;
+  if (!qe::make_gemm_group(gp, n, dev->num_sms, &l)) return fail(QE_ERR_UNSUPPORTED, "the problems cannot share a launch");
+  return launch_on(l, (cudaStream_t)stream);
 }
 
 int32_t qe_gemm_fp8(const void* a, uint32_t a_fmt, const void* b, uint32_t b_fmt, uint32_t M, uint32_t Nn, uint32_t Kc,

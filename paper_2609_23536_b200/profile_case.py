@@ -1,6 +1,6 @@
 """Small single-kernel cases for profiling (ncu) and quick timing.
 
-    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|gemm_microbatch|quantize|quantize_t|amax|accumulate [--reps N]
+    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|gemm_microbatch|gemm_microbatch_grouped|quantize|quantize_t|amax|accumulate [--reps N]
 
 Each case holds well under 2 GB on the device, uses operands larger than the 126 MB L2 where DRAM traffic is
 the question, does 2 warm-up launches and then `reps` launches, and prints the CUDA-event time per launch.
@@ -29,7 +29,29 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     T, H, F = (2048, 2048, 11264) if a.small else (4096, 4096, 28672)
     work = None
-    if a.case == "gemm_microbatch":
+    if a.case == "gemm_microbatch_grouped":
+        # the same twelve GEMMs in the five launches of the layer's steady state: F of linear i with dI of linear
+        # 3-i (four launches), then the four weight gradients in one launch
+        lin = ((H, 6144), (H, H), (H, F), (F // 2, H))
+
+        def prob(M, N, Kc, af, kind, amn, bmn):
+            return (torch.randint(0, 120, (Kc, M) if amn else (M, Kc), dtype=torch.uint8, device=dev), af, amn,
+                    torch.randint(0, 120, (Kc, N) if bmn else (N, Kc), dtype=torch.uint8, device=dev), 0, bmn, one, one,
+                    torch.zeros((M, N), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=dev), kind, None)
+
+        launches = []
+        for i in range(4):
+            (Ki, Ni), (Kj, Nj) = lin[i], lin[3 - i]
+            launches.append([prob(T, Ni, Ki, 0, 0, 0, 0), prob(T, Kj, Nj, 1, 0, 0, 1)])
+        launches.append([prob(N, K, T, 1, 2, 1, 1) for K, N in lin])
+
+        def fn():
+            for ps in launches:
+                qe.qe_gemm_fp8_group(ps, status)
+
+        work = {"flop": sum(6.0 * T * K * N for K, N in lin),
+                "bytes": sum(T * K + N * K + 2 * T * N + T * N + N * K + 2 * T * K + T * N + T * K + 8 * N * K for K, N in lin)}
+    elif a.case == "gemm_microbatch":
         # the twelve GEMMs (F, dI, dW of four linears) one microbatch of the Llama-style block launches, in order
         shapes = []
         # operand majors as the layer uses them: F both contraction-major; dI takes Wq [N,K] as an MN-major B;

@@ -248,3 +248,43 @@ def test_arena_reduce_order_is_visible_in_the_result(qe):
     assert torch.all(dst == 1.0 + 2.0**-23).item()
     with pytest.raises(qe.QEError):
         qe.qe_arena_reduce(torch.zeros((2, 12), dtype=torch.bfloat16, device=DEV), 2, torch.zeros(12, device=DEV))
+
+
+# ------------------------------------------------------------------------------------------ several problems per launch
+def test_gemm_group_equals_single_launches_bitwise(qe):
+    """Four different problems (formats, operand majors, epilogues, ragged N) in one launch against one launch each."""
+    rng = np.random.default_rng(77)
+    one = torch.ones(1, device=DEV)
+    half = torch.full((1,), 0.5, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    specs = [  # (M, N, Kc, a_fmt, a_mn, b_mn, out_kind)
+        (256, 640, 512, 0, 0, 0, 0),      # forward-like, bf16 + amax, N not a multiple of 256
+        (512, 256, 1280, 1, 0, 1, 0),     # input-gradient-like: E5M2 x E4M3, MN-major B
+        (768, 512, 256, 1, 1, 1, 2),      # weight-gradient-like: both MN-major, FP32 accumulate
+        (256, 256, 128, 0, 0, 0, 1),      # FP32 overwrite, a single K block
+    ]
+    probs_single, probs_group, outs = [], [], []
+    for M, N, Kc, af, amn, bmn, kind in specs:
+        A = torch.from_numpy(rng.integers(0, 120, (Kc, M) if amn else (M, Kc), dtype=np.uint8)).to(DEV)
+        B = torch.from_numpy(rng.integers(0, 120, (Kc, N) if bmn else (N, Kc), dtype=np.uint8)).to(DEV)
+        init = torch.randn((M, N), device=DEV)
+        d1 = init.to(torch.bfloat16) if kind == 0 else init.clone()
+        d2 = d1.clone()
+        am1, am2 = torch.zeros(1, device=DEV), torch.zeros(1, device=DEV)
+        qe.qe_gemm_fp8_ex(A, af, bool(amn), B, 0, bool(bmn), one, half, d1, kind, am1 if kind == 0 else None, status)
+        probs_group.append((A, af, amn, B, 0, bmn, one, half, d2, kind, am2 if kind == 0 else None))
+        outs.append((d1, d2, am1, am2, kind))
+    qe.qe_gemm_fp8_group(probs_group, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for d1, d2, am1, am2, kind in outs:
+        assert torch.equal(d1.view(torch.int16 if kind == 0 else torch.int32), d2.view(torch.int16 if kind == 0 else torch.int32))
+        assert am1.item() == am2.item() and (kind != 0 or am1.item() > 0)
+    with pytest.raises(qe.QEError) as e:  # a problem that needs the single-CTA variant cannot join
+        A = torch.zeros((384, 128), dtype=torch.uint8, device=DEV)
+        B = torch.zeros((256, 128), dtype=torch.uint8, device=DEV)
+        d = torch.zeros((384, 256), device=DEV)
+        qe.qe_gemm_fp8_group([probs_group[0], (A, 0, 0, B, 0, 0, one, one, d, 1, None)], status)
+    assert e.value.code == "UNSUPPORTED"
+    with pytest.raises(qe.QEError):
+        qe.qe_gemm_fp8_group(probs_group[:1], status)
