@@ -1,0 +1,96 @@
+"""The launch configuration bench.py times (config 2 at full size: graph mode, forward + input-gradient (+ deferred
+weight-gradient) units issued together in shared launches, the other weight gradients grouped on the second stream)
+against plain one-action-per-call eager execution, bit for bit, and against the oracle on one linear's state and
+sampled gradient rows."""
+import os
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+from harness import state_equal, state_equal_except_Y
+from oracle.layer import OracleLinear
+from paper_2609_23536_b200 import inputs
+from paper_2609_23536_b200.schedules import peak_live
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def qe():
+    from paper_2609_23536_b200 import build
+
+    build.build()
+    from paper_2609_23536_b200 import binding
+
+    return binding
+
+
+def test_bench_launch_configuration_equals_single_calls_and_oracle(qe):
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+
+    cfg = inputs.CONFIGS["C2"]
+    M, T, steps = cfg["M"], cfg["T"], 2
+    device = torch.device("cuda", 0)
+    with torch.cuda.stream(torch.cuda.Stream(device)):
+        stage = bench.Stage(qe, "C2", cfg, "graph", device, same_stream=True, overlap_dw=True)  # bench.py's defaults
+        for _ in range(steps):
+            stage.step()
+        torch.cuda.synchronize()
+        st = stage.ctx.stats()
+        assert st["paired_f_di"] > 0 and st["grouped_dw"] > 0  # the shared launches were really used
+        n = len(stage.layers)
+
+        # the same tensors through one call per action, eager, no second stream
+        ctx = qe.Context(qe.EAGER)
+        ref = [qe.Layer(ctx, T, L.K, L.N, cfg["H"], cfg["margin"], peak_live(stage.schedule), L.weight.clone(), unit=i)
+               for i, L in enumerate(stage.layers)]
+        grad = torch.zeros_like(stage.grad)
+        Y = [[torch.empty_like(t) for t in row] for row in stage.Y]
+        dX = [[torch.empty_like(t) for t in row] for row in stage.dX]
+        for step in range(steps):
+            tapes = {}
+            for a, m in stage.schedule:
+                for i in (range(n) if a == "F" else range(n - 1, -1, -1)):
+                    if a == "F":
+                        tapes[(m, i)] = ref[i].forward(m, step, stage.X[m][i], Y[m][i])
+                    elif a == "dI":
+                        ref[i].backward_dI(tapes[(m, i)], stage.dY[m][i], dX[m][i])
+                    else:
+                        ref[i].backward_dW(tapes[(m, i)], grad, stage.offsets[i])
+            for L in ref:
+                L.optimizer_boundary(M)
+        torch.cuda.synchronize()
+        for m in range(M):
+            for i in range(n):
+                assert torch.equal(stage.Y[m][i].view(torch.int16), Y[m][i].view(torch.int16)), ("Y", m, i)
+                assert torch.equal(stage.dX[m][i].view(torch.int16), dX[m][i].view(torch.int16)), ("dX", m, i)
+        assert torch.equal(stage.grad.view(torch.int32), grad.view(torch.int32))
+        for a, b in zip(stage.layers, ref):
+            sa, sb = a.state(), b.state()
+            assert state_equal({**sa, "slots": []}, {**sb, "slots": []}) and sa["device_token"] == sb["device_token"] and sa["device_status"] == 0
+
+        # the oracle on the attention output projection (linear 1): state after two steps, gradient rows of step 2
+        u = 1
+        L = stage.layers[u]
+        O = OracleLinear(T, L.K, L.N, cfg["H"], cfg["margin"], peak_live(stage.schedule), unit=u)
+        O.set_weight(inputs.bits(L.weight.cpu()))
+        rows = [0, 1, 777, L.N - 1]
+        obuf = np.zeros(L.N * L.K, np.float32)
+        for step in range(steps):
+            tapes = {}
+            for a, m in stage.schedule:
+                if a == "F":
+                    tapes[m], _ = O.forward(m, step, inputs.bits(stage.X[m][u].cpu()), rows=[0])
+                elif a == "dI":
+                    O.backward_dI(tapes[m], inputs.bits(stage.dY[m][u].cpu()), rows=[0])
+                else:
+                    O.backward_dW(tapes[m], obuf, 0, rows=rows)
+            O.optimizer_boundary(M)
+        assert state_equal_except_Y(L.state(), O.state())
+        got = stage.grad[stage.offsets[u]: stage.offsets[u] + L.N * L.K].view(L.N, L.K)[rows].cpu().numpy().astype(np.float64)
+        want = obuf.reshape(L.N, L.K)[rows].astype(np.float64)
+        assert np.linalg.norm(got - want) / np.linalg.norm(want) < 1e-5
