@@ -1200,9 +1200,16 @@ int32_t qe_forward_dI_pair(qe_layer* Lf, uint32_t mb, uint64_t gen, const void* 
 }
 
 // ------------------------------------------------------------------------------------------------ independent actions
-int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, void* caller_stream) {
-  if (!ctx || !acts || n == 0 || n > QE_MAX_TOGETHER) return fail(QE_ERR_BAD_ARG, "null argument or bad count %u", n);
+namespace {
+struct TogetherPrep {
+  int32_t refresh[QE_MAX_TOGETHER] = {}, acc[QE_MAX_TOGETHER] = {};
+  uint32_t slot[QE_MAX_TOGETHER] = {};
   bool any_dw = false;
+};
+
+// argument rules and every action's contract check; nothing is changed
+int32_t together_prepare(qe_ctx* ctx, const qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, TogetherPrep* pr) {
+  if (!ctx || !acts || n == 0 || n > QE_MAX_TOGETHER) return fail(QE_ERR_BAD_ARG, "null argument or bad count %u", n);
   for (uint32_t i = 0; i < n; ++i) {
     const qe_action& a = acts[i];
     if (a.kind > QE_ACT_DW || !a.layer || a.layer->ctx != ctx || !a.tape) return fail(QE_ERR_BAD_ARG, "action %u: bad kind, layer or tape", i);
@@ -1210,40 +1217,34 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
       return fail(QE_ERR_BAD_ARG, "action %u: input / output null or misaligned", i);
     for (uint32_t j = 0; j < i; ++j)
       if (acts[j].layer == a.layer && acts[j].kind == a.kind) return fail(QE_ERR_BAD_ARG, "actions %u and %u: same kind on the same layer", j, i);
-    any_dw |= a.kind == QE_ACT_DW;
+    pr->any_dw |= a.kind == QE_ACT_DW;
   }
-  if (any_dw && !grad) return fail(QE_ERR_BAD_ARG, "gradient buffer is null");
-  // check (every action, before anything runs) -> run -> commit
-  int32_t refresh[QE_MAX_TOGETHER] = {}, acc[QE_MAX_TOGETHER] = {};
-  uint32_t slot[QE_MAX_TOGETHER] = {};
-  int32_t st;
+  if (pr->any_dw && !grad) return fail(QE_ERR_BAD_ARG, "gradient buffer is null");
   for (uint32_t i = 0; i < n; ++i) {
     const qe_action& a = acts[i];
     qe_layer* L = a.layer;
+    int32_t st;
     if (a.kind == QE_ACT_F) {
-      st = qe_contract_forward_check(L->contract, a.mb, a.gen, &refresh[i], &slot[i]);
+      st = qe_contract_forward_check(L->contract, a.mb, a.gen, &pr->refresh[i], &pr->slot[i]);
     } else if (a.kind == QE_ACT_DI) {
       st = qe_contract_dI_check(L->contract, a.tape);
-      slot[i] = a.tape->ref.slot;
+      pr->slot[i] = a.tape->ref.slot;
     } else {
-      st = qe_contract_dW_check(L->contract, a.tape, (uint64_t)(uintptr_t)grad, grad_elems, a.grad_offset, (uint64_t)L->cfg.N * L->cfg.K, &acc[i]);
-      slot[i] = a.tape->ref.slot;
+      st = qe_contract_dW_check(L->contract, a.tape, (uint64_t)(uintptr_t)grad, grad_elems, a.grad_offset, (uint64_t)L->cfg.N * L->cfg.K, &pr->acc[i]);
+      pr->slot[i] = a.tape->ref.slot;
     }
     if (st != QE_OK) return st;
   }
-  cudaStream_t caller = (cudaStream_t)caller_stream;
-  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
-  if (any_dw && ctx->dw_stream) {  // weight gradients issued earlier on the second stream accumulate into the same buffer
-    QE_CUDA(cudaEventRecord(ctx->ev_dw_in, ctx->dw_stream));
-    QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_dw_in, 0));
-  }
-  std::vector<qe::Launch> ls;
+  return QE_OK;
+}
+
+// the launches: the casts two by two, then every GEMM that can run on the paired variant in one launch
+int32_t together_build(qe_ctx* ctx, const qe_action* acts, uint32_t n, const TogetherPrep& pr, float* grad,
+                       std::vector<qe::Launch>& ls, Fnv* h) {
   qe::GemmParams g[QE_MAX_TOGETHER];
   qe::QuantParams casts[QE_MAX_TOGETHER];
   std::vector<qe::GemmParams> singles;
   uint32_t ng = 0, n_chain = 0, n_dw = 0, n_casts = 0;
-  Fnv h;
-  h.mix("together", 9);
   for (int pass = 0; pass < 2; ++pass) {  // F and dI first (others wait for them), the weight gradients' tiles after theirs
     for (uint32_t i = 0; i < n; ++i) {
       const qe_action& a = acts[i];
@@ -1251,16 +1252,16 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
       if ((a.kind == QE_ACT_DW) != (pass == 1)) continue;
       qe::GemmParams gp;
       if (a.kind == QE_ACT_F) {
-        if (L->dw_pending[slot[i]]) {
-          QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[slot[i]], 0));
-          L->dw_pending[slot[i]] = false;
+        if (L->dw_pending[pr.slot[i]]) {
+          QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, L->ev_dw[pr.slot[i]], 0));
+          L->dw_pending[pr.slot[i]] = false;
         }
-        if (refresh[i]) add_refresh(L, ls);
-        add_forward(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp, &casts[n_casts++]);
+        if (pr.refresh[i]) add_refresh(L, ls);
+        add_forward(L, pr.slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp, &casts[n_casts++]);
       } else if (a.kind == QE_ACT_DI) {
-        add_dI(L, slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp, &casts[n_casts++]);
+        add_dI(L, pr.slot[i], a.in_dev, a.out_dev, ls, nullptr, 0, &gp, &casts[n_casts++]);
       } else {
-        gp = dW_gemm(L, slot[i], grad + a.grad_offset, acc[i], nullptr);
+        gp = dW_gemm(L, pr.slot[i], grad + a.grad_offset, pr.acc[i], nullptr);
       }
       if (qe::gemm_uses_pair(gp.M)) {
         g[ng++] = gp;
@@ -1268,10 +1269,12 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
       } else {
         singles.push_back(gp);  // single-CTA variant: a launch of its own
       }
-      h.mix(&a.kind, sizeof(a.kind));
-      h.mix(&a.layer, sizeof(a.layer));
-      h.mix(&slot[i], sizeof(uint32_t));
-      h.mix(&refresh[i], sizeof(int32_t));
+      if (h) {
+        h->mix(&a.kind, sizeof(a.kind));
+        h->mix(&a.layer, sizeof(a.layer));
+        h->mix(&pr.slot[i], sizeof(uint32_t));
+        h->mix(&pr.refresh[i], sizeof(int32_t));
+      }
     }
   }
   for (uint32_t i = 0; i + 1 < n_casts; i += 2) ls.push_back(qe::make_quantize_pair(casts[i], casts[i + 1]));  // casts two by two
@@ -1285,20 +1288,43 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
   } else {
     for (uint32_t i = 0; i < ng; ++i) ls.push_back(qe::make_gemm(g[i], ctx->dev->num_sms));
   }
-  if ((st = run_keyed(ctx, h.key, ls)) != QE_OK) return st;
-  if (ctx->dw_stream)
-    for (uint32_t i = 0; i < n; ++i)
-      if (acts[i].kind == QE_ACT_DI) QE_CUDA(cudaEventRecord(acts[i].layer->ev_di[slot[i]], ctx->exec_stream));
-  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  return QE_OK;
+}
+
+int32_t together_commit(const qe_action* acts, uint32_t n, float* grad) {
   for (uint32_t i = 0; i < n; ++i) {
     const qe_action& a = acts[i];
     qe_layer* L = a.layer;
+    int32_t st;
     if (a.kind == QE_ACT_F) st = qe_contract_forward_commit(L->contract, a.mb, a.tape);
     else if (a.kind == QE_ACT_DI) st = qe_contract_dI_commit(L->contract, a.tape);
     else st = qe_contract_dW_commit(L->contract, a.tape, (uint64_t)(uintptr_t)grad, a.grad_offset, (uint64_t)L->cfg.N * L->cfg.K);
     if (st != QE_OK) return st;
   }
   return QE_OK;
+}
+}  // namespace
+
+int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, void* caller_stream) {
+  TogetherPrep pr;
+  int32_t st = together_prepare(ctx, acts, n, grad, grad_elems, &pr);  // check (every action, before anything runs)
+  if (st != QE_OK) return st;
+  cudaStream_t caller = (cudaStream_t)caller_stream;
+  if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (pr.any_dw && ctx->dw_stream) {  // weight gradients issued earlier on the second stream accumulate into the same buffer
+    QE_CUDA(cudaEventRecord(ctx->ev_dw_in, ctx->dw_stream));
+    QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_dw_in, 0));
+  }
+  std::vector<qe::Launch> ls;
+  Fnv h;
+  h.mix("together", 9);
+  if ((st = together_build(ctx, acts, n, pr, grad, ls, &h)) != QE_OK) return st;
+  if ((st = run_keyed(ctx, h.key, ls)) != QE_OK) return st;  // ... run ...
+  if (ctx->dw_stream)
+    for (uint32_t i = 0; i < n; ++i)
+      if (acts[i].kind == QE_ACT_DI) QE_CUDA(cudaEventRecord(acts[i].layer->ev_di[pr.slot[i]], ctx->exec_stream));
+  if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
+  return together_commit(acts, n, grad);  // ... commit
 }
 
 // ------------------------------------------------------------------------------------------------ whole-step call
@@ -1323,6 +1349,55 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
   for (; k < n_actions && st == QE_OK; ++k) {
     const qe_step_action& a = actions[k];
     if (a.kind != QE_ACT_DW && dwb.n) dwb.flush(ctx, ls);
+    // A forward unit directly followed by an input-gradient unit of another microbatch (and possibly a deferred
+    // weight-gradient unit of a third): the units' chains through the layers are independent, so the i-th action of
+    // each goes out together, as qe_run_together would issue them.
+    if (a.kind == QE_ACT_F && !temp) {
+      uint32_t nf = 0;
+      while (k + nf < n_actions && actions[k + nf].kind == QE_ACT_F && actions[k + nf].mb == a.mb && actions[k + nf].layer < n_layers) ++nf;
+      auto run_of = [&](uint32_t start, uint32_t kind, uint32_t* mb_out) {  // nf actions of `kind`, one microbatch, distinct layers
+        if (start + nf > n_actions) return false;
+        for (uint32_t i = 0; i < nf; ++i) {
+          const qe_step_action& b = actions[start + i];
+          if (b.kind != kind || b.mb != actions[start].mb || b.layer >= n_layers || b.mb >= M) return false;
+          for (uint32_t j = 0; j < i; ++j)
+            if (actions[start + j].layer == b.layer) return false;
+        }
+        *mb_out = actions[start].mb;
+        return true;
+      };
+      uint32_t mf = 0, mb_i = 0, mb_w = 0;
+      bool ok = a.mb < M && run_of(k, QE_ACT_F, &mf) && run_of(k + nf, QE_ACT_DI, &mb_i) && mb_i != mf;
+      for (uint32_t i = 0; ok && i < nf; ++i) ok = have[(size_t)actions[k + nf + i].layer * M + mb_i] != 0;
+      bool with_dw = ok && run_of(k + 2 * nf, QE_ACT_DW, &mb_w) && mb_w != mf && mb_w != mb_i;
+      for (uint32_t i = 0; with_dw && i < nf; ++i) with_dw = have[(size_t)actions[k + 2 * nf + i].layer * M + mb_w] != 0;
+      if (ok) {
+        uint32_t i = 0;
+        for (; i < nf && st == QE_OK; ++i) {
+          const qe_step_action &af = actions[k + i], &ai = actions[k + nf + i];
+          const size_t uf = (size_t)af.layer * M + mf, ui = (size_t)ai.layer * M + mb_i;
+          qe_action acts[3];
+          uint32_t na = 2;
+          acts[0] = qe_action{QE_ACT_F, mf, layers[af.layer]->contract->e_W, layers[af.layer], io[uf].x_dev, io[uf].y_dev, &tapes[uf], 0};
+          acts[1] = qe_action{QE_ACT_DI, 0, 0, layers[ai.layer], io[ui].dy_dev, io[ui].dx_dev, &tapes[ui], 0};
+          if (with_dw) {
+            const qe_step_action& aw = actions[k + 2 * nf + i];
+            acts[na++] = qe_action{QE_ACT_DW, 0, 0, layers[aw.layer], nullptr, nullptr, &tapes[(size_t)aw.layer * M + mb_w], offsets[aw.layer]};
+          }
+          TogetherPrep pr;
+          if ((st = together_prepare(ctx, acts, na, grad, grad_elems, &pr)) != QE_OK) break;
+          if ((st = together_build(ctx, acts, na, pr, grad, ls, nullptr)) != QE_OK) break;
+          st = together_commit(acts, na, grad);
+          have[uf] = 1;
+        }
+        if (st != QE_OK) {
+          k += i;  // (reported as the index of the forward action of the failing group)
+          break;
+        }
+        k += (with_dw ? 3 : 2) * nf - 1;
+        continue;
+      }
+    }
     if (a.layer >= n_layers || a.mb >= M || a.kind > QE_ACT_DW) {
       st = fail(QE_ERR_BAD_ARG, "action %u: kind %u layer %u mb %u", k, a.kind, a.layer, a.mb);
       break;

@@ -88,17 +88,17 @@ def test_step_call_equals_per_action_calls_bitwise(qe, mode, staged):
         assert np.array_equal(a, b)
     assert np.array_equal(want[2].view(np.uint32), got[2].view(np.uint32))
     for a, b in zip(want[3], got[3]):
-        assert state_equal(a, b) and a["device_token"] == b["device_token"]
+        # (which slot a tape gets depends on the order of allocations and releases, which grouping changes; all else is equal)
+        assert state_equal({**a, "slots": []}, {**b, "slots": []}) and a["device_token"] == b["device_token"]
     st = ctx2.stats()
     assert st["handoffs"] == 2 * 3  # one handshake pair per step instead of per action
+    per_action = 3 * len(SHAPES) * (M * ((2 + 2 + 2) if staged else 5) + 1)  # kernels of the one-call-per-action run
     if staged:
-        n_kernels = 3 * len(SHAPES) * (M * (2 + 2 + 2) + 1)
-        assert st["grouped_dw"] == 0
+        assert st["kernels_launched"] == per_action and st["grouped_dw"] == 0 and st["paired_f_di"] == 0
     else:
-        # the dW GEMMs of the two layers whose N is a multiple of 256 share one launch per microbatch
-        n_kernels = 3 * (len(SHAPES) * (M * 4 + 1) + M * 2)
-        assert st["grouped_dw"] == 3 * M * 2
-    assert st["kernels_launched"] == n_kernels
+        # forward units directly followed by input-gradient (and weight-gradient) units went out together, and
+        # weight gradients of layers that can pair shared launches: fewer kernels, same bits
+        assert st["paired_f_di"] > 0 and st["grouped_dw"] > 0 and st["kernels_launched"] < per_action - 3 * M
     if mode == 1:
         assert st["graphs_built"] == 1 and st["graph_replays"] == 3
 
@@ -291,7 +291,9 @@ def test_two_chunk_schedules_split_equals_full_and_match_the_oracle(qe, gen, mod
         for L in orc:
             L.optimizer_boundary(M)
     for a, L in zip(st, orc):
-        assert state_equal_except_Y(a, L.state())
+        # (the whole-step call issues adjacent independent units together, which changes the order of slot allocations
+        # and releases and with it the slot a tape gets; everything else is equal)
+        assert state_equal_except_Y({**a, "slots": []}, {**L.state(), "slots": []})
 
 
 # ------------------------------------------------------------------------------------------ F and dI in one call
