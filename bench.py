@@ -216,6 +216,17 @@ class Stage:
                     if n % 2:  # the middle linear went out alone above: its weight gradient too
                         self.layers[n // 2].backward_dW(tapes[(mb_w, n // 2)], self.grad, self.offsets[n // 2])
                 continue
+            if (self.together and not host_io and a == "dI" and k + 1 < len(self.schedule) and self.schedule[k + 1][0] == "dW"
+                    and self.schedule[k + 1][1] != m):
+                # cool-down: an input-gradient unit and a deferred weight-gradient unit of an earlier microbatch: dI of
+                # linear n-1-i goes out with dW of linear i
+                mb_w = self.schedule[k + 1][1]
+                for i in range(n):
+                    j = n - 1 - i
+                    self.qe.run_together(self.ctx, [("dI", self.layers[j], tapes[(m, j)], self.dY[m][j], self.dX[m][j]),
+                                                    ("dW", self.layers[i], tapes[(mb_w, i)], self.offsets[i])], self.grad)
+                skip = 1
+                continue
             if self.chain and a != "dW" and not host_io:
                 # the linears as directly chained groups of up to 16 (FP8 hand-off: one cast per group and direction)
                 for g in (self.groups if a == "F" else reversed(self.groups)):

@@ -326,7 +326,8 @@ int32_t qe_next_slot(const qe_layer*, uint32_t* slot_out);
  * the one-by-one order): consecutive dW actions of different layers as in qe_backward_dW_multi; and, when n forward
  * actions of one microbatch over n different layers are directly followed by n input-gradient actions of another
  * microbatch (and those possibly by n weight-gradient actions of a third), the i-th action of each run is issued
- * together as qe_run_together would (not with temp_dev).
+ * together as qe_run_together would; likewise n input-gradient actions directly followed by n weight-gradient
+ * actions of another microbatch (none of this with temp_dev).
  * If a check fails at action k, the kernels of actions 0..k-1 are still issued (device and host state stay in step),
  * then every layer of the list is aborted as at a failure boundary (Sec. 4.5) and the failing check's status is
  * returned; qe_arena_rebuild restarts the epoch. */

@@ -1352,6 +1352,39 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
     // A forward unit directly followed by an input-gradient unit of another microbatch (and possibly a deferred
     // weight-gradient unit of a third): the units' chains through the layers are independent, so the i-th action of
     // each goes out together, as qe_run_together would issue them.
+    if (a.kind == QE_ACT_DI && !temp && a.mb < M) {
+      // cool-down: an input-gradient unit directly followed by a weight-gradient unit of an earlier microbatch
+      uint32_t nd = 0;
+      while (k + nd < n_actions && actions[k + nd].kind == QE_ACT_DI && actions[k + nd].mb == a.mb && actions[k + nd].layer < n_layers) ++nd;
+      bool ok = k + 2 * nd <= n_actions;
+      uint32_t mw = ok ? actions[k + nd].mb : 0;
+      for (uint32_t i = 0; ok && i < nd; ++i) {
+        const qe_step_action &ai = actions[k + i], &aw = actions[k + nd + i];
+        ok = aw.kind == QE_ACT_DW && aw.mb == mw && mw != a.mb && mw < M && aw.layer < n_layers &&
+             have[(size_t)ai.layer * M + a.mb] && have[(size_t)aw.layer * M + mw];
+        for (uint32_t j = 0; ok && j < i; ++j) ok = actions[k + j].layer != ai.layer && actions[k + nd + j].layer != aw.layer;
+      }
+      if (ok) {
+        uint32_t i = 0;
+        for (; i < nd && st == QE_OK; ++i) {
+          const qe_step_action &ai = actions[k + i], &aw = actions[k + nd + i];
+          const size_t ui = (size_t)ai.layer * M + a.mb;
+          qe_action acts[2];
+          acts[0] = qe_action{QE_ACT_DI, 0, 0, layers[ai.layer], io[ui].dy_dev, io[ui].dx_dev, &tapes[ui], 0};
+          acts[1] = qe_action{QE_ACT_DW, 0, 0, layers[aw.layer], nullptr, nullptr, &tapes[(size_t)aw.layer * M + mw], offsets[aw.layer]};
+          TogetherPrep pr;
+          if ((st = together_prepare(ctx, acts, 2, grad, grad_elems, &pr)) != QE_OK) break;
+          if ((st = together_build(ctx, acts, 2, pr, grad, ls, nullptr)) != QE_OK) break;
+          st = together_commit(acts, 2, grad);
+        }
+        if (st != QE_OK) {
+          k += i;
+          break;
+        }
+        k += 2 * nd - 1;
+        continue;
+      }
+    }
     if (a.kind == QE_ACT_F && !temp) {
       uint32_t nf = 0;
       while (k + nf < n_actions && actions[k + nf].kind == QE_ACT_F && actions[k + nf].mb == a.mb && actions[k + nf].layer < n_layers) ++nf;
