@@ -1291,15 +1291,25 @@ int32_t together_build(qe_ctx* ctx, const qe_action* acts, uint32_t n, const Tog
   return QE_OK;
 }
 
-int32_t together_commit(const qe_action* acts, uint32_t n, float* grad) {
-  for (uint32_t i = 0; i < n; ++i) {
-    const qe_action& a = acts[i];
-    qe_layer* L = a.layer;
-    int32_t st;
-    if (a.kind == QE_ACT_F) st = qe_contract_forward_commit(L->contract, a.mb, a.tape);
-    else if (a.kind == QE_ACT_DI) st = qe_contract_dI_commit(L->contract, a.tape);
-    else st = qe_contract_dW_commit(L->contract, a.tape, (uint64_t)(uintptr_t)grad, a.grad_offset, (uint64_t)L->cfg.N * L->cfg.K);
-    if (st != QE_OK) return st;
+// Forward commits first: a forward's tape slot was chosen by its check, on the state before the call, and the kernels
+// used it; a weight-gradient commit of the same layer releases a slot and must not come in between.
+int32_t together_commit(const qe_action* acts, uint32_t n, float* grad, const TogetherPrep& pr) {
+  for (uint32_t kind = QE_ACT_F; kind <= QE_ACT_DW; ++kind) {
+    for (uint32_t i = 0; i < n; ++i) {
+      const qe_action& a = acts[i];
+      if (a.kind != kind) continue;
+      qe_layer* L = a.layer;
+      int32_t st;
+      if (a.kind == QE_ACT_F) {
+        st = qe_contract_forward_commit(L->contract, a.mb, a.tape);
+        if (st == QE_OK && a.tape->ref.slot != pr.slot[i]) return fail(QE_ERR_ORDER, "forward committed to slot %u, ran in slot %u", a.tape->ref.slot, pr.slot[i]);
+      } else if (a.kind == QE_ACT_DI) {
+        st = qe_contract_dI_commit(L->contract, a.tape);
+      } else {
+        st = qe_contract_dW_commit(L->contract, a.tape, (uint64_t)(uintptr_t)grad, a.grad_offset, (uint64_t)L->cfg.N * L->cfg.K);
+      }
+      if (st != QE_OK) return st;
+    }
   }
   return QE_OK;
 }
@@ -1324,7 +1334,7 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
     for (uint32_t i = 0; i < n; ++i)
       if (acts[i].kind == QE_ACT_DI) QE_CUDA(cudaEventRecord(acts[i].layer->ev_di[pr.slot[i]], ctx->exec_stream));
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
-  return together_commit(acts, n, grad);  // ... commit
+  return together_commit(acts, n, grad, pr);  // ... commit
 }
 
 // ------------------------------------------------------------------------------------------------ whole-step call
@@ -1375,7 +1385,7 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
           TogetherPrep pr;
           if ((st = together_prepare(ctx, acts, 2, grad, grad_elems, &pr)) != QE_OK) break;
           if ((st = together_build(ctx, acts, 2, pr, grad, ls, nullptr)) != QE_OK) break;
-          st = together_commit(acts, 2, grad);
+          st = together_commit(acts, 2, grad, pr);
         }
         if (st != QE_OK) {
           k += i;
@@ -1420,7 +1430,7 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
           TogetherPrep pr;
           if ((st = together_prepare(ctx, acts, na, grad, grad_elems, &pr)) != QE_OK) break;
           if ((st = together_build(ctx, acts, na, pr, grad, ls, nullptr)) != QE_OK) break;
-          st = together_commit(acts, na, grad);
+          st = together_commit(acts, na, grad, pr);
           have[uf] = 1;
         }
         if (st != QE_OK) {

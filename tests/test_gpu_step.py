@@ -459,3 +459,74 @@ def test_run_together_is_all_or_nothing(qe):
     qe.run_together(ctx, [("dI", A, ta, ya, xa), ("dW", B, tb, 512 * 256)], grad)
     torch.cuda.synchronize()
     assert not torch.any(torch.isnan(grad[512 * 256:])).item() and torch.all(torch.isnan(grad[: 512 * 256])).item()
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_run_together_random_groupings_equal_sequential_bitwise(qe, seed):
+    """Random legal action orders over three linears and four microbatches, cut at random into groups of independent
+    neighbours (at most one action of a kind per layer, a dW never in the group of its own dI): every grouping must
+    give the bits of the plain one-by-one order."""
+    rng = np.random.default_rng(seed)
+    T, M = 256, 4
+    shapes = [(256, 512), (512, 256), (256, 256)]
+    n = len(shapes)
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in shapes])
+    # a random legal order: per (layer, mb) F < dI < dW; per layer F, dI and dW each in microbatch order
+    nxt = {(k, l): 0 for k in ("F", "dI", "dW") for l in range(n)}
+    order = []
+    while len(order) < 3 * n * M:
+        cand = []
+        for l in range(n):
+            if nxt[("F", l)] < M and nxt[("F", l)] - nxt[("dW", l)] < 3:  # at most three live tapes per layer
+                cand.append(("F", l, nxt[("F", l)]))
+            if nxt[("dI", l)] < nxt[("F", l)]:
+                cand.append(("dI", l, nxt[("dI", l)]))
+            if nxt[("dW", l)] < nxt[("dI", l)]:
+                cand.append(("dW", l, nxt[("dW", l)]))
+        k, l, m = cand[rng.integers(len(cand))]
+        order.append((k, l, m))
+        nxt[(k, l)] += 1
+    # random grouping of neighbours
+    groups, cur = [], []
+    for act in order:
+        k, l, m = act
+        clash = any((k2 == k and l2 == l) or (l2 == l and m2 == m) for k2, l2, m2 in cur)  # same kind+layer, or same unit
+        if cur and (clash or len(cur) == 4 or rng.random() < 0.3):
+            groups.append(cur)
+            cur = []
+        cur.append(act)
+    groups.append(cur)
+    assert any(len(g) >= 3 for g in groups)
+    results = []
+    for grouped in (False, True):
+        ctx = qe.Context(int(seed % 2))
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, 3, inputs.weights("RG", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(shapes)]
+        grad = torch.full((total,), float("nan"), device=DEV)
+        X = [[inputs.activations("RG", 0, 0, j, m, T, K).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+        dY = [[inputs.upstream_grads("RG", 0, 0, j, m, T, N).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+        Y = [[torch.zeros((T, N), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        dX = [[torch.zeros((T, K), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        tapes = {}
+        for g in (groups if grouped else [[a] for a in order]):
+            acts, fkeys = [], []
+            for k, l, m in g:
+                if k == "F":
+                    acts.append(("F", layers[l], m, 0, X[m][l], Y[m][l]))
+                    fkeys.append((l, m))
+                elif k == "dI":
+                    acts.append(("dI", layers[l], tapes[(l, m)], dY[m][l], dX[m][l]))
+                else:
+                    acts.append(("dW", layers[l], tapes[(l, m)], offs[l]))
+            for key, t in zip(fkeys, qe.run_together(ctx, acts, grad)):
+                tapes[key] = t
+        for L in layers:
+            L.optimizer_boundary(M)
+        torch.cuda.synchronize()
+        results.append(([inputs.bits(t.cpu()) for row in Y for t in row], [inputs.bits(t.cpu()) for row in dX for t in row],
+                        grad.cpu().numpy().copy(), [L.state() for L in layers]))
+    a, b = results
+    for u, v in zip(a[0] + a[1], b[0] + b[1]):
+        assert np.array_equal(u, v)
+    assert np.array_equal(a[2].view(np.uint32), b[2].view(np.uint32)) and not np.any(np.isnan(b[2]))
+    for u, v in zip(a[3], b[3]):
+        assert state_equal({**u, "slots": []}, {**v, "slots": []}) and u["device_token"] == v["device_token"]
