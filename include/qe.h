@@ -239,8 +239,10 @@ int32_t qe_forward_dI_pair(qe_layer* layer_f, uint32_t mb, uint64_t gen, const v
  * all GEMMs that can run on the paired-CTA variant share one kernel launch (forward and input-gradient tiles
  * first, weight-gradient tiles after them).  1 <= n <= QE_MAX_TOGETHER; at most one
  * action of a kind per layer; a dW action's tape must already have had its dI (ORDER otherwise, also when that dI
- * is part of the same call).  Every check is made before anything runs: on a contract error nothing ran and no
- * state changed.  Everything runs on the execution stream (weight gradients issued earlier on the context's second
+ * is part of the same call).  Every check is made before anything runs, against the state before the call: on a
+ * contract error nothing ran and no state changed; in particular a forward cannot take the slot that a dW of the same
+ * call is about to release (POOL_FULL if no other slot is free), and the slot a tape lands in may differ from the
+ * one-by-one order.  Everything runs on the execution stream (weight gradients issued earlier on the context's second
  * stream are waited for). */
 #define QE_MAX_TOGETHER 4
 typedef struct qe_action {

@@ -500,7 +500,9 @@ def test_run_together_random_groupings_equal_sequential_bitwise(qe, seed):
     results = []
     for grouped in (False, True):
         ctx = qe.Context(int(seed % 2))
-        layers = [qe.Layer(ctx, T, K, N, 4, 0, 3, inputs.weights("RG", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(shapes)]
+        # four slots for at most three live tapes: a forward is checked against the pool as it stands before the call, so a
+        # slot released by a dW of the same group is not yet available to it
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, 4, inputs.weights("RG", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(shapes)]
         grad = torch.full((total,), float("nan"), device=DEV)
         X = [[inputs.activations("RG", 0, 0, j, m, T, K).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
         dY = [[inputs.upstream_grads("RG", 0, 0, j, m, T, N).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
