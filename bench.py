@@ -216,6 +216,25 @@ class Stage:
                     if n % 2:  # the middle linear went out alone above: its weight gradient too
                         self.layers[n // 2].backward_dW(tapes[(mb_w, n // 2)], self.grad, self.offsets[n // 2])
                 continue
+            if self.together and not host_io and a == "F" and k + 1 < len(self.schedule) and self.schedule[k + 1][0] == "F":
+                # warm-up: several forward units in a row (the last of them goes out with what follows it).  Their chains
+                # through the linears are independent, so they advance as a wavefront: round r holds F of linear r-j of
+                # the j-th unit; each linear still sees the microbatches in order
+                ms, kk = [], k
+                while kk + 1 < len(self.schedule) and self.schedule[kk][0] == "F" and self.schedule[kk + 1][0] == "F" and len(ms) < 4:
+                    ms.append(self.schedule[kk][1])
+                    kk += 1
+                for r in range(n + len(ms) - 1):
+                    acts, keys = [], []
+                    for j, mm in enumerate(ms):
+                        i = r - j
+                        if 0 <= i < n:
+                            acts.append(("F", self.layers[i], mm, self.epoch, self.X[mm][i], self.Y[mm][i]))
+                            keys.append((mm, i))
+                    for key, t in zip(keys, self.qe.run_together(self.ctx, acts)):
+                        tapes[key] = t
+                skip = len(ms) - 1
+                continue
             if (self.together and not host_io and a == "dI" and k + 1 < len(self.schedule) and self.schedule[k + 1][0] == "dW"
                     and self.schedule[k + 1][1] != m):
                 # cool-down: an input-gradient unit and a deferred weight-gradient unit of an earlier microbatch: dI of
