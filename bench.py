@@ -102,7 +102,7 @@ class Stage:
     """All linears of the configuration on one device, with resident per-microbatch inputs and outputs."""
 
     def __init__(self, qe, cfg_name, cfg, mode, device, host_io=False, same_stream=True, overlap_dw=False, staged=False,
-                 group_dw=True, arena=False, chain=False, pair_f_di=True, together=True):
+                 group_dw=True, arena=False, chain=False, pair_f_di=True, together=True, plan_window=0):
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
@@ -110,12 +110,16 @@ class Stage:
         self.chain = chain
         self.pair_f_di = pair_f_di and not chain and not host_io
         self.together = together and self.pair_f_di and not staged and not arena
+        self.plan_window = plan_window
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
                               exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
                               overlap_dw=overlap_dw)
         self.schedule = sched(cfg["M"], *cfg["sched"])
         P = peak_live(self.schedule)
+        if plan_window:
+            from paper_2609_23536_b200.schedules import plan_rounds
+            self.rounds = plan_rounds(self.schedule, len(cfg["linears"]) * cfg["layers"], P, 4, plan_window)
         T, M = cfg["T"], cfg["M"]
         self.layers, self.offsets = [], []
         lin = cfg["linears"]
@@ -183,6 +187,25 @@ class Stage:
         tapes = {}
         n = len(self.layers)
         t_issue = time.perf_counter()
+        if self.plan_window and not host_io:
+            # the schedule cut into rounds of independent per-linear actions (schedules.plan_rounds), one call each
+            for group in self.rounds:
+                acts, keys = [], []
+                for a, i, m in group:
+                    if a == "F":
+                        acts.append(("F", self.layers[i], m, self.epoch, self.X[m][i], self.Y[m][i]))
+                        keys.append((m, i))
+                    elif a == "dI":
+                        acts.append(("dI", self.layers[i], tapes[(m, i)], self.dY[m][i], self.dX[m][i]))
+                    else:
+                        acts.append(("dW", self.layers[i], tapes[(m, i)], self.offsets[i]))
+                for key, t in zip(keys, self.qe.run_together(self.ctx, acts, self.grad)):
+                    tapes[key] = t
+            self.issue_s += time.perf_counter() - t_issue
+            for L in self.layers:
+                L.optimizer_boundary(self.cfg["M"])
+            self.epoch += 1
+            return
         skip = 0
         for k, (a, m) in enumerate(self.schedule):
             if skip:  # this dI (and dW) went out together with the forward before it
@@ -596,6 +619,10 @@ def main():
                     help="one qe_backward_dW call per linear instead of qe_backward_dW_multi per microbatch")
     ap.add_argument("--no-pair-f-di", dest="pair_f_di", action="store_false",
                     help="never issue a forward and the input gradient that follows it in the schedule as qe_forward_dI_pair calls")
+    ap.add_argument("--plan", type=int, default=-1, metavar="WINDOW",
+                    help="issue the step as rounds of independent per-linear actions planned by schedules.plan_rounds, looking WINDOW "
+                         "schedule units ahead (default: the schedule's warm-up depth + 1, the units a stage holds at once; 0: issue "
+                         "unit by unit, pairing only direct neighbours)")
     ap.add_argument("--no-together", dest="together", action="store_false",
                     help="keep the deferred dW out of the shared F + dI launches (it then goes to the second stream)")
     ap.add_argument("--chain", action="store_true",
@@ -635,7 +662,8 @@ def main():
 
     use_step = args.step_api
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
-                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain, pair_f_di=args.pair_f_di, together=args.together)
+                  overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain, pair_f_di=args.pair_f_di, together=args.together,
+                  plan_window=0 if (use_step or args.staged or args.arena or args.chain or not args.together or not args.pair_f_di) else (cfg["sched"][0] + 1 if args.plan < 0 else args.plan))
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:
@@ -651,7 +679,7 @@ def main():
         "config": {
             "workload": cfg_name, "tokens": cfg["T"], "linears": [[n, K, N] for n, K, N in cfg["linears"]],
             "layers": cfg["layers"], "microbatches": cfg["M"], "schedule": "sched(M,%d,%d) zero-bubble style, dW deferred" % cfg["sched"],
-            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else "one C-ABI call per action; a forward and the input gradient (and deferred dW) that follow it in the schedule go out linear by linear through qe_forward_dI_pair / qe_run_together" if args.pair_f_di else "one C-ABI call per action", "chained_fp8_handoff": bool(args.chain), "f_with_next_dI": "one shared GEMM launch per (F of linear i, dI of linear n-1-i)" if (args.pair_f_di and not args.chain and not args.step_api) else "separate", "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
+            "history_len": cfg["H"], "exec": args.mode, "overlap_dw": bool(args.overlap_dw and not args.step_api), "issue": "qe_step_run (one call per step)" if args.step_api else ("rounds of independent per-linear actions (schedules.plan_rounds, window %d), one qe_run_together call each" % stage.plan_window) if stage.plan_window else "one C-ABI call per action; a forward and the input gradient (and deferred dW) that follow it in the schedule go out linear by linear through qe_forward_dI_pair / qe_run_together" if args.pair_f_di else "one C-ABI call per action", "chained_fp8_handoff": bool(args.chain), "f_with_next_dI": "one shared GEMM launch per (F of linear i, dI of linear n-1-i)" if (args.pair_f_di and not args.chain and not args.step_api) else "separate", "gradient_path": "per-microbatch bf16 arena + reduction" if args.arena else "staged copy-add" if args.staged else "direct placement", "dw_launches": "shared by up to 4 linears" if (args.group_dw and not args.staged and not args.arena) else "one per linear", "exec_stream": "context-owned (event handoffs)" if args.own_stream else "caller's stream", "parallelism": "replicas x%d (path does not shard)" % world,
             "l2": "per-step inputs (%.0f MB) exceed L2; distinct tensors per microbatch" % (
                 sum(cfg["T"] * (K + N) * 2 for _, K, N in cfg["linears"]) * cfg["M"] * cfg["layers"] / 1e6),
             "flop_per_step": step_flops(cfg),

@@ -51,9 +51,10 @@ struct QuantParams {
 };
 
 
-struct QuantPairParams {
-  QuantParams q[2];            // neither carries a commit tail
-  uint32_t blocks0;            // blocks of the first cast
+struct QuantMultiParams {
+  QuantParams q[4];            // none carries a commit tail
+  uint32_t block_end[4];       // cumulative block counts
+  uint32_t n;
   uint32_t pad[3];
 };
 
@@ -133,7 +134,7 @@ struct Launch {
 };
 
 Launch make_quantize(const QuantParams& p);
-Launch make_quantize_pair(const QuantParams& a, const QuantParams& b);
+Launch make_quantize_multi(const QuantParams* casts, uint32_t n);  // 2..4 independent casts in one launch
 Launch make_commit(const CommitParams& p);
 Launch make_amax_pass1(const AmaxParams& p);
 Launch make_amax_pass2(const AmaxParams& p);

@@ -124,29 +124,34 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_co
   }
 }
 
-// Two independent casts in one launch (the X of a forward unit and the dY of an input-gradient unit that go out
-// together): blocks [0, blocks0) work on the first, the rest on the second.  No commit tails.
-__global__ void __launch_bounds__(kQuantThreads) quantize_pair_kernel(const __grid_constant__ QuantPairParams pp) {
+// Two to four independent casts in one launch (the X of forward units and the dY of input-gradient units that go out
+// together): the blocks are dealt to the casts one cast after the other.  No commit tails.
+__global__ void __launch_bounds__(kQuantThreads) quantize_multi_kernel(const __grid_constant__ QuantMultiParams mp) {
   __shared__ uint32_t wmax[kQuantThreads / 32];
   grid_dep_wait();
   grid_dep_launch();
-  const uint32_t which = blockIdx.x >= pp.blocks0 ? 1u : 0u;
-  const QuantParams& p = pp.q[which];
-  const uint32_t b = blockIdx.x - (which ? pp.blocks0 : 0u), bxn = p.cols / 64u;
+  uint32_t which = 0, base = 0;
+  while (which + 1 < mp.n && blockIdx.x >= mp.block_end[which]) base = mp.block_end[which++];
+  const QuantParams& p = mp.q[which];
+  const uint32_t b = blockIdx.x - base, bxn = p.cols / 64u;
   if (p.fmt == 0) quantize_block<0>(p, b % bxn, b / bxn, wmax);
   else quantize_block<1>(p, b % bxn, b / bxn, wmax);
 }
 
-Launch make_quantize_pair(const QuantParams& a, const QuantParams& b) {
-  QuantPairParams pp{};
-  pp.q[0] = a;
-  pp.q[1] = b;
-  pp.blocks0 = (a.cols / 64) * ((a.rows + 255) / 256);
+Launch make_quantize_multi(const QuantParams* casts, uint32_t n) {
+  QuantMultiParams mp{};
+  uint32_t blocks = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    mp.q[i] = casts[i];
+    blocks += (casts[i].cols / 64) * ((casts[i].rows + 255) / 256);
+    mp.block_end[i] = blocks;
+  }
+  mp.n = n;
   Launch l;
-  l.func = (const void*)quantize_pair_kernel;
-  l.grid = dim3(pp.blocks0 + (b.cols / 64) * ((b.rows + 255) / 256), 1, 1);
+  l.func = (const void*)quantize_multi_kernel;
+  l.grid = dim3(blocks, 1, 1);
   l.block = dim3(kQuantThreads, 1, 1);
-  l.set(pp);
+  l.set(mp);
   return l;
 }
 

@@ -1176,7 +1176,7 @@ int32_t qe_forward_dI_pair(qe_layer* Lf, uint32_t mb, uint64_t gen, const void* 
   qe::QuantParams c[2];
   add_forward(Lf, p, x, y, ls, nullptr, 0, &g[0], &c[0]);  // hands the casts and the GEMMs back
   add_dI(Lb, pb, dy, dx, ls, nullptr, 0, &g[1], &c[1]);
-  ls.push_back(qe::make_quantize_pair(c[0], c[1]));  // both casts in one launch
+  ls.push_back(qe::make_quantize_multi(c, 2));  // both casts in one launch
   qe::Launch shared;
   if (qe::make_gemm_group(g, 2, ctx->dev->num_sms, &shared)) {
     ls.push_back(shared);
@@ -1238,7 +1238,7 @@ int32_t together_prepare(qe_ctx* ctx, const qe_action* acts, uint32_t n, float* 
   return QE_OK;
 }
 
-// the launches: the casts two by two, then every GEMM that can run on the paired variant in one launch
+// the launches: the casts in one launch, then every GEMM that can run on the paired variant in one launch
 int32_t together_build(qe_ctx* ctx, const qe_action* acts, uint32_t n, const TogetherPrep& pr, float* grad,
                        std::vector<qe::Launch>& ls, Fnv* h) {
   qe::GemmParams g[QE_MAX_TOGETHER];
@@ -1277,8 +1277,8 @@ int32_t together_build(qe_ctx* ctx, const qe_action* acts, uint32_t n, const Tog
       }
     }
   }
-  for (uint32_t i = 0; i + 1 < n_casts; i += 2) ls.push_back(qe::make_quantize_pair(casts[i], casts[i + 1]));  // casts two by two
-  if (n_casts & 1u) ls.push_back(qe::make_quantize(casts[n_casts - 1]));
+  if (n_casts >= 2) ls.push_back(qe::make_quantize_multi(casts, n_casts));  // all casts of the call in one launch
+  else if (n_casts == 1) ls.push_back(qe::make_quantize(casts[0]));
   for (const qe::GemmParams& gp : singles) ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
   qe::Launch shared;
   if (ng >= 2 && qe::make_gemm_group(g, ng, ctx->dev->num_sms, &shared)) {

@@ -197,3 +197,68 @@ def full_backward_chunks(schedule: List[ChunkAction]) -> List[ChunkAction]:
         if a == "dI":
             out.append(("dW", m, c))
     return out
+
+
+# ------------------------------------------------------------------------------------------------ issue plan
+# A unit of the schedule ("F" | "dI" | "dW", microbatch) stands for one action per linear of the stage.  Units whose
+# inputs are at hand at the same time are independent of each other, so their per-linear actions may share launches.
+LayerAction = Tuple[str, int, int]  # (kind, linear, microbatch)
+
+
+def plan_rounds(schedule: List[Action], n_linears: int, slots: int, max_group: int = 4, window: int = 3) -> List[List[LayerAction]]:
+    """Cuts a schedule into rounds of at most `max_group` per-linear actions that may be issued together.
+
+    Looking at most `window` units ahead of the earliest unfinished one, a round takes every action whose
+    predecessors were issued in EARLIER rounds: the previous linear of its own unit (F walks the linears up, dI
+    down; dW has no order among linears), the same linear of the previous unit of its kind (each linear sees the
+    microbatches in schedule order), F before dI before dW of a (linear, microbatch), and a free tape slot for a
+    forward (slots are released by rounds before this one).  At most one action of a kind per linear in a round,
+    and never two actions of the same (linear, microbatch).  The one-action-per-round plan is the schedule itself.
+    """
+    units = list(schedule)
+    prev_of_kind = {}
+    last = {}
+    for idx, (a, m) in enumerate(units):
+        prev_of_kind[idx] = last.get(a)
+        last[a] = idx
+    todo = []  # per unit: linears still to issue, in chain order
+    for a, _ in units:
+        todo.append(list(range(n_linears)) if a == "F" else list(range(n_linears - 1, -1, -1)))
+    issued = set()
+    live = [0] * n_linears
+    rounds: List[List[LayerAction]] = []
+    first = 0
+    while first < len(units):
+        group: List[LayerAction] = []
+        for idx in range(first, min(first + window, len(units))):
+            a, m = units[idx]
+            cands = todo[idx][:1] if a != "dW" else list(todo[idx])
+            for l in cands:
+                if len(group) == max_group:
+                    break
+                if any((a2 == a and l2 == l) or (l2 == l and m2 == m) for a2, l2, m2 in group):
+                    continue
+                p = prev_of_kind[idx]
+                if p is not None and (a, l, units[p][1]) not in issued:
+                    continue
+                if a == "F" and live[l] >= slots:
+                    continue
+                if a == "dI" and ("F", l, m) not in issued:
+                    continue
+                if a == "dW" and ("dI", l, m) not in issued:
+                    continue
+                group.append((a, l, m))
+        if not group:
+            raise RuntimeError("no action is ready: the schedule is not legal for this pool size")
+        for a, l, m in group:
+            issued.add((a, l, m))
+            idx = next(i for i in range(first, len(units)) if units[i] == (a, m))
+            todo[idx].remove(l)
+            if a == "F":
+                live[l] += 1
+            elif a == "dW":
+                live[l] -= 1
+        rounds.append(group)
+        while first < len(units) and not todo[first]:
+            first += 1
+    return rounds

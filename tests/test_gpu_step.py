@@ -532,3 +532,55 @@ def test_run_together_random_groupings_equal_sequential_bitwise(qe, seed):
     assert np.array_equal(a[2].view(np.uint32), b[2].view(np.uint32)) and not np.any(np.isnan(b[2]))
     for u, v in zip(a[3], b[3]):
         assert state_equal({**u, "slots": []}, {**v, "slots": []}) and u["device_token"] == v["device_token"]
+
+
+@pytest.mark.parametrize("M,w,d,window", [(4, 1, 0, 2), (6, 3, 3, 4), (5, 2, 1, 3), (6, 3, 3, 6)])
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_planned_rounds_equal_the_schedule_issued_action_by_action_bitwise(qe, mode, M, w, d, window):
+    """schedules.plan_rounds regroups the schedule into rounds of independent per-linear actions; issuing a round per
+    qe_run_together call must give the bits of issuing the schedule one action at a time."""
+    from paper_2609_23536_b200.schedules import plan_rounds
+
+    T = 256
+    shapes = [(256, 512), (512, 256), (256, 256), (256, 768)]
+    n = len(shapes)
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in shapes])
+    s = sched(M, w, d)
+    P = peak_live(s)
+    rounds = plan_rounds(s, n, P, 4, window)
+    plain = [[(a, l, m)] for a, m in s for l in (range(n) if a == "F" else range(n - 1, -1, -1))]
+    results = []
+    for plan in (plain, rounds):
+        ctx = qe.Context(mode)
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, P, inputs.weights("PL", 0, j, N, K).to(DEV), unit=j) for j, (K, N) in enumerate(shapes)]
+        grad = torch.full((total,), float("nan"), device=DEV)
+        Y = [[torch.zeros((T, N), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        dX = [[torch.zeros((T, K), dtype=torch.bfloat16, device=DEV) for K, N in shapes] for m in range(M)]
+        for step in range(2):
+            X = [[inputs.activations("PL", step, 0, j, m, T, K).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+            dY = [[inputs.upstream_grads("PL", step, 0, j, m, T, N).to(DEV) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+            tapes = {}
+            for g in plan:
+                acts, keys = [], []
+                for a, l, m in g:
+                    if a == "F":
+                        acts.append(("F", layers[l], m, step, X[m][l], Y[m][l]))
+                        keys.append((l, m))
+                    elif a == "dI":
+                        acts.append(("dI", layers[l], tapes[(l, m)], dY[m][l], dX[m][l]))
+                    else:
+                        acts.append(("dW", layers[l], tapes[(l, m)], offs[l]))
+                for key, t in zip(keys, qe.run_together(ctx, acts, grad)):
+                    tapes[key] = t
+            for L in layers:
+                L.optimizer_boundary(M)
+        torch.cuda.synchronize()
+        results.append(([inputs.bits(t.cpu()) for row in Y for t in row], [inputs.bits(t.cpu()) for row in dX for t in row],
+                        grad.cpu().numpy().copy(), [L.state() for L in layers]))
+    a, b = results
+    for u, v in zip(a[0] + a[1], b[0] + b[1]):
+        assert np.array_equal(u, v)
+    assert np.array_equal(a[2].view(np.uint32), b[2].view(np.uint32)) and not np.any(np.isnan(b[2]))
+    for u, v in zip(a[3], b[3]):
+        assert state_equal({**u, "slots": []}, {**v, "slots": []}) and u["device_token"] == v["device_token"]
+    assert len(rounds) < len(plain)
