@@ -119,7 +119,7 @@ class Stage:
         P = peak_live(self.schedule)
         if plan_window:
             from paper_2609_23536_b200.schedules import plan_rounds
-            self.rounds = plan_rounds(self.schedule, len(cfg["linears"]) * cfg["layers"], P, 4, plan_window)
+            self.rounds = plan_rounds(self.schedule, len(cfg["linears"]) * cfg["layers"], P, 8, plan_window)
         T, M = cfg["T"], cfg["M"]
         self.layers, self.offsets = [], []
         lin = cfg["linears"]
@@ -621,8 +621,8 @@ def main():
                     help="never issue a forward and the input gradient that follows it in the schedule as qe_forward_dI_pair calls")
     ap.add_argument("--plan", type=int, default=-1, metavar="WINDOW",
                     help="issue the step as rounds of independent per-linear actions planned by schedules.plan_rounds, looking WINDOW "
-                         "schedule units ahead (default: the schedule's warm-up depth + 1, the units a stage holds at once; 0: issue "
-                         "unit by unit, pairing only direct neighbours)")
+                         "schedule units ahead (default: warm-up depth + deferral of the schedule, the units a stage holds at once; 0: "
+                         "issue unit by unit, pairing only direct neighbours)")
     ap.add_argument("--no-together", dest="together", action="store_false",
                     help="keep the deferred dW out of the shared F + dI launches (it then goes to the second stream)")
     ap.add_argument("--chain", action="store_true",
@@ -663,7 +663,7 @@ def main():
     use_step = args.step_api
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
                   overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain, pair_f_di=args.pair_f_di, together=args.together,
-                  plan_window=0 if (use_step or args.staged or args.arena or args.chain or not args.together or not args.pair_f_di) else (cfg["sched"][0] + 1 if args.plan < 0 else args.plan))
+                  plan_window=0 if (use_step or args.staged or args.arena or args.chain or not args.together or not args.pair_f_di) else (max(2, cfg["sched"][0] + cfg["sched"][1]) if args.plan < 0 else args.plan))
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:

@@ -244,7 +244,7 @@ int32_t qe_forward_dI_pair(qe_layer* layer_f, uint32_t mb, uint64_t gen, const v
  * call is about to release (POOL_FULL if no other slot is free), and the slot a tape lands in may differ from the
  * one-by-one order.  Everything runs on the execution stream (weight gradients issued earlier on the context's second
  * stream are waited for). */
-#define QE_MAX_TOGETHER 4
+#define QE_MAX_TOGETHER 8
 typedef struct qe_action {
   uint32_t kind;          /* QE_ACT_F, QE_ACT_DI or QE_ACT_DW                                                */
   uint32_t mb;            /* F: microbatch                                                                   */
@@ -293,7 +293,7 @@ int32_t qe_arena_finalize(qe_layer*, const void* arena_dev, uint64_t arena_elems
 int32_t qe_arena_reduce(const void* views_dev, uint64_t view_elems, uint32_t M, float* dst_dev, void* stream);
 /* The W action of Sec. 4.2 for several layers of the stage at once (typically one microbatch's deferred weight
  * gradients): the same checks, results (bit for bit) and state transitions as qe_backward_dW(layers[i], &tapes[i],
- * grad_buf_dev, grad_buf_elems, offsets[i], stream) for i = 0..n-1, but the GEMMs of up to four layers share one
+ * grad_buf_dev, grad_buf_elems, offsets[i], stream) for i = 0..n-1, but the GEMMs of up to four layers at a time share one
  * kernel launch where each of them can run on the paired-CTA variant (N_i a multiple of 256); the others are
  * launched one by one inside the same call.  layers[] (host array) distinct and of one context, 1 <= n <=
  * QE_MAX_MULTI_DW; tapes[] and offsets[] host arrays of n entries.  All n checks are made before anything runs: on
@@ -415,7 +415,7 @@ int32_t qe_gemm_fp8_ex(const void* a_dev, uint32_t a_format, uint32_t a_mn, cons
                        const float* alpha_b_dev, void* d_dev, uint32_t out_kind, float* amax_dev, uint32_t* status_dev,
                        void* stream);
 
-/* Two to four independent FP8 GEMMs in ONE kernel launch (the launch shape the layer uses for F + dI pairs and for
+/* Two to eight independent FP8 GEMMs in ONE kernel launch (the launch shape the layer uses for F + dI pairs and for
  * the weight gradients of a microbatch): the persistent CTAs work through the problems' tiles one problem after the
  * other, so the launch cost is paid once and partial waves are shared.  Each problem as in qe_gemm_fp8_ex; every M
  * must be a multiple of 256 (QE_ERR_UNSUPPORTED otherwise); outputs must not overlap.  descs: host array. */

@@ -14,7 +14,7 @@
 //               accumulation straight into the destination (direct gradient placement): the addition is done in
 //               L2, one per element and launch, and the destination tile is prefetched into L2 while the tile's
 //               main loop runs.  The reduction is a plain round-to-nearest FP32 addition (subnormal values kept).
-//   The launch may also carry up to four independent problems (grouped launch): tiles are numbered problem after
+//   The launch may also carry up to eight independent problems (grouped launch): tiles are numbered problem after
 //   problem and each role looks its tile's problem up, so that one set of persistent CTAs packs them all.
 // When asked to, the last CTA to finish folds the pending amax values into their histories and updates the scales
 // (the commit that ends F and dI), so that no extra launch is needed for it.
@@ -614,7 +614,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
   gemm_body<true>(OneProblem{p});
 }
 
-// Up to four independent GEMMs (each eligible for the paired variant) in one launch.
+// Up to eight independent GEMMs (each eligible for the paired variant) in one launch.
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
     gemm_fp8_pair_group_kernel(const __grid_constant__ GemmGroupParams g) {
   gemm_body<true>(ProblemGroup{g});
@@ -645,7 +645,7 @@ cudaError_t gemm_prepare() {
 }
 
 bool make_gemm_group(const GemmParams* probs, uint32_t n, int num_sms, Launch* out) {
-  if (n < 2 || n > 4) return false;
+  if (n < 2 || n > 8) return false;
   GemmGroupParams g{};
   uint32_t tiles = 0;
   for (uint32_t i = 0; i < n; ++i) {

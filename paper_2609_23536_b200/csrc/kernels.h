@@ -52,8 +52,8 @@ struct QuantParams {
 
 
 struct QuantMultiParams {
-  QuantParams q[4];            // none carries a commit tail
-  uint32_t block_end[4];       // cumulative block counts
+  QuantParams q[8];            // none carries a commit tail
+  uint32_t block_end[8];       // cumulative block counts
   uint32_t n;
   uint32_t pad[3];
 };
@@ -110,12 +110,12 @@ struct GemmParams {
   CommitParams commit;         // performed by the last CTA to finish (commit.st != null)
 };
 
-// Up to four independent GEMMs computed by one launch: tiles are numbered problem after problem.
+// Up to eight independent GEMMs computed by one launch: tiles are numbered problem after problem.
 struct GemmGroupParams {
   uint32_t n;
-  uint32_t tile_end[4];        // cumulative tile counts (256 x 256 tiles)
-  uint32_t pad[11];
-  GemmParams prob[4];
+  uint32_t tile_end[8];        // cumulative tile counts (256 x 256 tiles)
+  uint32_t pad[7];
+  GemmParams prob[8];
 };
 
 // One launch, self-contained.
@@ -124,7 +124,7 @@ struct Launch {
   dim3 grid{1, 1, 1}, block{1, 1, 1};
   uint32_t smem = 0;
   uint32_t nbytes = 0;
-  alignas(64) unsigned char params[2560];
+  alignas(64) unsigned char params[4864];
   template <class P>
   void set(const P& p) {
     static_assert(sizeof(P) <= sizeof(params), "parameter block too large");
@@ -134,14 +134,14 @@ struct Launch {
 };
 
 Launch make_quantize(const QuantParams& p);
-Launch make_quantize_multi(const QuantParams* casts, uint32_t n);  // 2..4 independent casts in one launch
+Launch make_quantize_multi(const QuantParams* casts, uint32_t n);  // 2..8 independent casts in one launch
 Launch make_commit(const CommitParams& p);
 Launch make_amax_pass1(const AmaxParams& p);
 Launch make_amax_pass2(const AmaxParams& p);
 Launch make_accumulate(const AccumParams& p);
 Launch make_arena_reduce(const ArenaReduceParams& p);
 Launch make_gemm(const GemmParams& p, int num_sms);
-// One launch for n = 2..4 GEMMs (each may carry its own commit tail); false if the group cannot be formed (a problem
+// One launch for n = 2..8 GEMMs (each may carry its own commit tail); false if the group cannot be formed (a problem
 // needs the single-CTA variant), in which case the caller launches them one by one.
 bool make_gemm_group(const GemmParams* probs, uint32_t n, int num_sms, Launch* out);
 cudaError_t gemm_prepare();  // opt in to the dynamic shared memory the GEMM needs (once per device)

@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const __grid_co
   }
 }
 
-// Two to four independent casts in one launch (the X of forward units and the dY of input-gradient units that go out
+// Two to eight independent casts in one launch (the X of forward units and the dY of input-gradient units that go out
 // together): the blocks are dealt to the casts one cast after the other.  No commit tails.
 __global__ void __launch_bounds__(kQuantThreads) quantize_multi_kernel(const __grid_constant__ QuantMultiParams mp) {
   __shared__ uint32_t wmax[kQuantThreads / 32];

@@ -1824,11 +1824,11 @@ int32_t qe_gemm_fp8_ex(const void* a, uint32_t a_fmt, uint32_t a_mn, const void*
 
 int32_t qe_gemm_fp8_group(const qe_gemm_desc* descs, uint32_t n, uint32_t* status_dev, void* stream) {
   if (!descs || !status_dev) return fail(QE_ERR_BAD_ARG, "null argument");
-  if (n < 2 || n > 4) return fail(QE_ERR_BAD_ARG, "a group holds 2 to 4 problems, got %u", n);
+  if (n < 2 || n > 8) return fail(QE_ERR_BAD_ARG, "a group holds 2 to 8 problems, got %u", n);
   DeviceInfo* dev = nullptr;
   int32_t st = current_device_info(&dev);
   if (st != QE_OK) return st;
-  qe::GemmParams gp[4];
+  qe::GemmParams gp[8];
   for (uint32_t i = 0; i < n; ++i) {
     const qe_gemm_desc& q = descs[i];
     if (!qe::gemm_uses_pair(q.M)) return fail(QE_ERR_UNSUPPORTED, "problem %u: M=%u is not a multiple of 256", i, q.M);

@@ -37,7 +37,7 @@ def test_bench_launch_configuration_equals_single_calls_and_oracle(qe):
     device = torch.device("cuda", 0)
     with torch.cuda.stream(torch.cuda.Stream(device)):
         stage = bench.Stage(qe, "C2", cfg, "graph", device, same_stream=True, overlap_dw=True,
-                            plan_window=cfg["sched"][0] + 1)  # bench.py's defaults
+                            plan_window=cfg["sched"][0] + cfg["sched"][1])  # bench.py's defaults
         for _ in range(steps):
             stage.step()
         torch.cuda.synchronize()

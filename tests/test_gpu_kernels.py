@@ -288,3 +288,29 @@ def test_gemm_group_equals_single_launches_bitwise(qe):
     assert e.value.code == "UNSUPPORTED"
     with pytest.raises(qe.QEError):
         qe.qe_gemm_fp8_group(probs_group[:1], status)
+
+
+def test_gemm_group_of_eight(qe):
+    """The largest group: eight small problems in one launch against eight single launches."""
+    rng = np.random.default_rng(8)
+    one = torch.ones(1, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    probs, outs = [], []
+    for i in range(8):
+        M, N, Kc = 256 * (1 + i % 3), 256 + 128 * (i % 4), 128 * (1 + i % 5)
+        kind = i % 3
+        A = torch.from_numpy(rng.integers(0, 120, (M, Kc), dtype=np.uint8)).to(DEV)
+        B = torch.from_numpy(rng.integers(0, 120, (N, Kc), dtype=np.uint8)).to(DEV)
+        init = torch.randn((M, N), device=DEV)
+        d1 = init.to(torch.bfloat16) if kind == 0 else init.clone()
+        d2 = d1.clone()
+        qe.qe_gemm_fp8_ex(A, 0, False, B, i % 2, False, one, one, d1, kind, None, status)
+        probs.append((A, 0, 0, B, i % 2, 0, one, one, d2, kind, None))
+        outs.append((d1, d2, kind))
+    qe.qe_gemm_fp8_group(probs, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for d1, d2, kind in outs:
+        assert torch.equal(d1.view(torch.int16 if kind == 0 else torch.int32), d2.view(torch.int16 if kind == 0 else torch.int32))
+    with pytest.raises(qe.QEError):
+        qe.qe_gemm_fp8_group(probs + probs[:1], status)

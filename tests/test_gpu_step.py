@@ -534,9 +534,9 @@ def test_run_together_random_groupings_equal_sequential_bitwise(qe, seed):
         assert state_equal({**u, "slots": []}, {**v, "slots": []}) and u["device_token"] == v["device_token"]
 
 
-@pytest.mark.parametrize("M,w,d,window", [(4, 1, 0, 2), (6, 3, 3, 4), (5, 2, 1, 3), (6, 3, 3, 6)])
+@pytest.mark.parametrize("M,w,d,window,group", [(4, 1, 0, 2, 4), (6, 3, 3, 4, 4), (5, 2, 1, 3, 8), (6, 3, 3, 6, 8)])
 @pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
-def test_planned_rounds_equal_the_schedule_issued_action_by_action_bitwise(qe, mode, M, w, d, window):
+def test_planned_rounds_equal_the_schedule_issued_action_by_action_bitwise(qe, mode, M, w, d, window, group):
     """schedules.plan_rounds regroups the schedule into rounds of independent per-linear actions; issuing a round per
     qe_run_together call must give the bits of issuing the schedule one action at a time."""
     from paper_2609_23536_b200.schedules import plan_rounds
@@ -547,7 +547,8 @@ def test_planned_rounds_equal_the_schedule_issued_action_by_action_bitwise(qe, m
     offs, total = inputs.grad_offsets([("l", K, N) for K, N in shapes])
     s = sched(M, w, d)
     P = peak_live(s)
-    rounds = plan_rounds(s, n, P, 4, window)
+    rounds = plan_rounds(s, n, P, group, window)
+    assert group == 4 or any(len(g) > 4 for g in rounds)
     plain = [[(a, l, m)] for a, m in s for l in (range(n) if a == "F" else range(n - 1, -1, -1))]
     results = []
     for plan in (plain, rounds):

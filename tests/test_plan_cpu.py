@@ -36,12 +36,12 @@ def _check(schedule, n, slots, rounds, max_group):
 
 @pytest.mark.parametrize("M,w,d", [(4, 1, 0), (8, 3, 3), (8, 1, 2), (6, 2, 1), (32, 3, 3), (5, 5, 5)])
 @pytest.mark.parametrize("n", [1, 3, 4])
-@pytest.mark.parametrize("window", [1, 2, 4, 6])
-def test_plans_are_legal(M, w, d, n, window):
+@pytest.mark.parametrize("window,group", [(1, 4), (2, 4), (4, 8), (6, 8)])
+def test_plans_are_legal(M, w, d, n, window, group):
     s = sched(M, w, d)
     slots = peak_live(s)
-    rounds = plan_rounds(s, n, slots, 4, window)
-    _check(s, n, slots, rounds, 4)
+    rounds = plan_rounds(s, n, slots, group, window)
+    _check(s, n, slots, rounds, group)
     if window == 1 and n == 1:
         assert [g[0] for g in rounds] == [(a, 0, m) for a, m in s]  # nothing to regroup: the schedule itself
     assert len(rounds) <= 3 * n * M
