@@ -361,10 +361,15 @@ def time_steps(stage, steps, warmup, host_io, dist):
     return ms, stage.ctx.stats()["kernels_launched"] - k0
 
 
+# 19 launches: 3528.2 MB read + 1820.6 MB written (profiles/gemm_fp8_pair_dram_traffic_config2_microbatch.md)
+QE_TRAFFIC_C2, QE_TRAFFIC_C2_LAUNCHES = 281.5e6, 19
+
+
 def gemm_roofline(qe, cfg, peaks, device):
-    """Times the dominant kernel (the tcgen05 FP8 GEMM) alone, live: every GEMM shape of one microbatch, launched
-    back to back through the C-ABI on the current stream over rotating operand sets larger than L2, CUDA events
-    around the loop.  achieved = algorithmic flops / average launch duration."""
+    """Times the dominant kernel (the tcgen05 FP8 GEMM) alone, live, through the C-ABI on the current stream with CUDA
+    events around the loop: first every GEMM shape of one microbatch in a launch of its own over rotating operand sets
+    larger than L2 (per-action rates), then the GEMM launches of one whole step as the issue plan groups them (the
+    roofline figure: achieved = algorithmic flops of the step / time of its GEMM launches)."""
     import torch
 
     T = cfg["T"]
@@ -403,52 +408,23 @@ def gemm_roofline(qe, cfg, peaks, device):
         per[name][1] += ms
         del A, B, D
     assert status.item() == 0
-    # ... and the same twelve GEMMs in the launches the layer path issues in its steady state: F of linear i with dI
-    # of linear n-1-i in one launch each, the weight gradients of all linears in one launch
-    lin = cfg["linears"]
-    nl = len(lin)
-    groups = []
-    for i in range(nl):
-        j = nl - 1 - i
-        (_, Ki, Ni), (_, Kj, Nj) = lin[i], lin[j]
-        groups.append([("F", T, Ni, Ki, 0, 0, 0, 0), ("dI", T, Kj, Nj, 1, 0, 1, 0)] if i != j else [("F", T, Ni, Ki, 0, 0, 0, 0)])
-        if i == j:
-            groups.append([("dI", T, Kj, Nj, 1, 0, 1, 0)])
-    for lo in range(0, nl, 4):
-        groups.append([("dW", N, K, T, 1, 1, 1, 2) for _, K, N in lin[lo:lo + 4]])
-    g_flops = g_ms = 0.0
-    g_launches = 0
-    for grp in groups:
-        if any(M_ % 256 for _, M_, *_ in grp) or len(grp) < 2:  # shapes that cannot share a launch: one by one (timed above)
-            for name, M_, N_, Kc, *_ in grp:
-                g_flops += 2.0 * M_ * N_ * Kc
-            g_ms += sum(per_shape_ms[(name, M_, N_, Kc)] for name, M_, N_, Kc, *_ in grp)
-            g_launches += len(grp)
-            continue
-        nbytes = sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if kind == 0 else 8) for _, M_, N_, Kc, _, _, _, kind in grp)
-        nset = min(max(2, int(160e6 // nbytes) + 1), 12)
-        sets = []
-        for _ in range(nset):
-            ps = []
-            for name, M_, N_, Kc, af, amn, bmn, kind in grp:
-                ps.append((torch.randint(0, 120, (Kc, M_) if amn else (M_, Kc), dtype=torch.uint8, device=device), af, amn,
-                           torch.randint(0, 120, (Kc, N_) if bmn else (N_, Kc), dtype=torch.uint8, device=device), 0, bmn, one, one,
-                           torch.zeros((M_, N_), dtype=torch.bfloat16 if kind == 0 else torch.float32, device=device), kind, None))
-            sets.append(ps)
-        for ps in sets:
-            qe.qe_gemm_fp8_group(ps, status)
-        torch.cuda.synchronize()
-        reps = 3 * nset
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for r in range(reps):
-            qe.qe_gemm_fp8_group(sets[r % nset], status)
-        e1.record()
-        torch.cuda.synchronize()
-        g_ms += e0.elapsed_time(e1) / reps
-        g_flops += sum(2.0 * M_ * N_ * Kc for _, M_, N_, Kc, *_ in grp)
-        g_launches += 1
-        del sets
+    # ... and the GEMM launches of one whole step as the default issue plan makes them (schedules.plan_rounds: up to
+    # eight independent per-linear GEMMs per launch), every (linear, microbatch) with operands and outputs of its own
+    from paper_2609_23536_b200 import step_gemms
+
+    launches, g_flops, g_bytes = step_gemms.build(cfg, device)
+    step_gemms.run(qe, launches, status)
+    torch.cuda.synchronize()
+    reps = 3
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        step_gemms.run(qe, launches, status)
+    e1.record()
+    torch.cuda.synchronize()
+    g_ms = e0.elapsed_time(e1) / reps
+    g_launches = len(launches)
+    del launches
     assert status.item() == 0
     lib = None
     try:  # context only: the vendor library's FP8 GEMM (cuBLASLt through torch._scaled_mm) on the forward shapes
@@ -473,21 +449,20 @@ def gemm_roofline(qe, cfg, peaks, device):
         lib = "unavailable: " + str(e)[:80]
     single = tot_flops / (tot_ms * 1e-3) / 1e12
     achieved = g_flops / (g_ms * 1e-3) / 1e12
-    # dram__bytes_read + dram__bytes_write per launch, averaged over the five launches of a microbatch, from one ncu
-    # capture of `python -m paper_2609_23536_b200.profile_case gemm_microbatch_grouped --small` (config-2 shapes only)
-    # (five launches: 445.0 MB read + 159.6 MB written)
-    traffic = 120.9e6 if (T, tuple(cfg["linears"])) == (2048, tuple(inputs.CONFIGS["C2"]["linears"])) and g_launches == 5 else None
+    # dram__bytes_read + dram__bytes_write per launch, averaged over the GEMM launches of one step, from one ncu
+    # capture of `python -m paper_2609_23536_b200.profile_case gemm_step --small` (config-2 shapes only)
+    traffic = QE_TRAFFIC_C2 if (T, tuple(cfg["linears"]), cfg["layers"], g_launches) == (2048, tuple(inputs.CONFIGS["C2"]["linears"]), 1, QE_TRAFFIC_C2_LAUNCHES) else None
     peak = 2.0 * peaks["bf16_burst"]  # FP8 dense = 2 x the bf16 peak (nominal ratio), kernels timed alone -> burst figure
     return {
-        "bound": "tensor", "kernel": "gemm_fp8_pair_group_kernel (F + dI pairs, grouped dW: the launches of the steady state)",
+        "bound": "tensor", "kernel": "gemm_fp8_pair_group_kernel (the GEMM launches of one step as the issue plan groups them)",
         "achieved": round(achieved, 1), "peak": round(peak, 1),
         "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": traffic,
-        "algorithmic_bytes_per_launch": round(sum(M_ * Kc + N_ * Kc + M_ * N_ * (2 if k == 0 else 8) for _, M_, N_, Kc, _, _, _, k in shapes) / g_launches),
+        "algorithmic_bytes_per_launch": round(g_bytes / g_launches),
         "flop_per_launch": round(g_flops / g_launches), "launches_timed": g_launches, "peak_source": peaks["source"] + " bf16 burst x2",
         "frac_of_nominal_4500": round(achieved / 4500.0, 4),
         "one_problem_per_launch_tflops": round(single, 1),
         "per_action_tflops": {k: round(v[0] / (v[1] * 1e-3) / 1e12, 1) for k, v in per.items()},
-        "gemm_ms_per_microbatch": round(g_ms, 4),
+        "gemm_ms_per_step": round(g_ms, 4),
         "vendor_library_fp8_forward_tflops_same_shapes": lib,
     }
 
@@ -707,7 +682,7 @@ def main():
         torch.cuda.empty_cache()
         if rank == 0:
             line["roofline"] = gemm_roofline(qe, cfg, peaks, device)
-            line["roofline"]["gemm_share_of_step"] = round(line["roofline"]["gemm_ms_per_microbatch"] * cfg["M"] * cfg["layers"] / (ms / args.steps), 3)
+            line["roofline"]["gemm_share_of_step"] = round(line["roofline"]["gemm_ms_per_step"] / (ms / args.steps), 3)
             line["hbm_kernels"] = hbm_kernels(qe, cfg, peaks, device)
             if world == 1:
                 s, f = oracle_sample(cfg_name, cfg)

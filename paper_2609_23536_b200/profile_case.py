@@ -1,6 +1,6 @@
 """Small single-kernel cases for profiling (ncu) and quick timing.
 
-    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|gemm_microbatch|gemm_microbatch_grouped|quantize|quantize_t|amax|accumulate [--reps N]
+    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|gemm_microbatch|gemm_microbatch_grouped|gemm_step|quantize|quantize_t|amax|accumulate [--reps N]
 
 Each case holds well under 2 GB on the device, uses operands larger than the 126 MB L2 where DRAM traffic is
 the question, does 2 warm-up launches and then `reps` launches, and prints the CUDA-event time per launch.
@@ -29,7 +29,14 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     T, H, F = (2048, 2048, 11264) if a.small else (4096, 4096, 28672)
     work = None
-    if a.case == "gemm_microbatch_grouped":
+    if a.case == "gemm_step":
+        # the GEMM launches of one optimizer step as the default issue plan groups them (config 2 with --small)
+        from . import inputs, step_gemms
+
+        launches, flops, nbytes = step_gemms.build(inputs.CONFIGS["C2" if a.small else "C3"], dev)
+        fn = lambda: step_gemms.run(qe, launches, status)
+        work = {"flop": flops, "bytes": nbytes, "launches": len(launches)}
+    elif a.case == "gemm_microbatch_grouped":
         # the same twelve GEMMs in the five launches of the layer's steady state: F of linear i with dI of linear
         # 3-i (four launches), then the four weight gradients in one launch
         lin = ((H, 6144), (H, H), (H, F), (F // 2, H))
@@ -112,6 +119,8 @@ def main():
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / a.reps
     out = {"case": a.case, "ms": round(ms, 4), "status": int(status.item())}
+    if "launches" in work:
+        out["launches"] = work["launches"]
     if "flop" in work:
         out["TFLOP/s"] = round(work["flop"] / ms / 1e9, 1)
     out["GB/s_algorithmic"] = round(work["bytes"] / ms / 1e6, 1)
