@@ -1,5 +1,6 @@
 // Host side of the layer API: workspace carve-up, tensor maps, the three checked actions and the execution layer
 // (eager launches or one CUDA graph per (action, slot), both bracketed by the two-way stream handshake).
+#include <algorithm>
 #include <chrono>
 #include <cmath>
 #include <cstdio>
@@ -1277,6 +1278,10 @@ int32_t together_build(qe_ctx* ctx, const qe_action* acts, uint32_t n, const Tog
       }
     }
   }
+  // longest tiles first (their contraction length decides a tile's duration): the launch's last, partial wave is then
+  // made of short tiles.  The weight gradients (contraction over T only) stay behind the others.
+  std::stable_sort(g, g + n_chain, [](const qe::GemmParams& x, const qe::GemmParams& y) { return x.Kc > y.Kc; });
+  std::stable_sort(g + n_chain, g + ng, [](const qe::GemmParams& x, const qe::GemmParams& y) { return x.Kc > y.Kc; });
   if (n_casts >= 2) ls.push_back(qe::make_quantize_multi(casts, n_casts));  // all casts of the call in one launch
   else if (n_casts == 1) ls.push_back(qe::make_quantize(casts[0]));
   for (const qe::GemmParams& gp : singles) ls.push_back(qe::make_gemm(gp, ctx->dev->num_sms));
