@@ -241,6 +241,13 @@ __device__ __forceinline__ void tile_coords(uint32_t tile, uint32_t tiles_m, uin
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory"); }
 
+// Which tile cluster `first` of `step` clusters takes in wave w: the clusters walk the tile list back and forth, so
+// that with tiles sorted by decreasing duration the cluster that got the longest tile of one wave gets the shortest
+// of the next (a static approximation of longest-processing-time-first).
+__device__ __forceinline__ uint32_t snake_tile(uint32_t w, uint32_t first, uint32_t step) {
+  return w * step + ((w & 1u) ? step - 1u - first : first);
+}
+
 // ------------------------------------------------------------------------------------------------ problem lookup
 // A launch computes one GEMM, or (grouped launch) up to four independent ones whose tiles are numbered one after the
 // other, so that one set of persistent CTAs packs them into common waves and the launch overhead is paid once.
@@ -368,7 +375,7 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
+      for (uint32_t wave = 0, tile = first_tile; ok && tile < num_tiles; ++wave, tile = snake_tile(wave, first_tile, tile_step)) {
         QE_TILE_PROBLEM();
         uint32_t m0, n0;
         tile_coords(local_tile, tiles_m, tiles_n, m_fastest, C::TILE_M, m0, n0);
@@ -406,7 +413,7 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
       int s = 0;
       uint32_t ph = 0, acc = 0, acc_ph = 0;
       bool ok = true;
-      for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
+      for (uint32_t wave = 0, tile = first_tile; ok && tile < num_tiles; ++wave, tile = snake_tile(wave, first_tile, tile_step)) {
         QE_TILE_PROBLEM();
         (void)tiles_m; (void)tiles_n; (void)m_fastest;
         if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, status, ERR_MMA))) break;
@@ -445,7 +452,7 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
     bool ok = true;
     const uint32_t tempty_leader0 = TWO ? map_to_cta(tempty_bar(0), 0) : tempty_bar(0);
     const uint32_t tempty_leader1 = TWO ? map_to_cta(tempty_bar(1), 0) : tempty_bar(1);
-    for (uint32_t tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
+    for (uint32_t wave = 0, tile = first_tile; ok && tile < num_tiles; ++wave, tile = snake_tile(wave, first_tile, tile_step)) {
       QE_TILE_PROBLEM();
       (void)num_kb;
       const float alpha = __fmul_rn(*p.alpha_a, *p.alpha_b);
