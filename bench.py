@@ -361,8 +361,8 @@ def time_steps(stage, steps, warmup, host_io, dist):
     return ms, stage.ctx.stats()["kernels_launched"] - k0
 
 
-# 19 launches: 3528.2 MB read + 1820.6 MB written (profiles/gemm_fp8_pair_dram_traffic_config2_microbatch.md)
-QE_TRAFFIC_C2, QE_TRAFFIC_C2_LAUNCHES = 281.5e6, 19
+# 19 launches: 3599.4 MB read + 1864.3 MB written (profiles/gemm_fp8_pair_dram_traffic_config2_microbatch.md)
+QE_TRAFFIC_C2, QE_TRAFFIC_C2_LAUNCHES = 287.6e6, 19
 
 
 def gemm_roofline(qe, cfg, peaks, device):
