@@ -114,7 +114,7 @@ class Stage:
         # the context executes on the stream the benchmark issues from: no cross-stream event hops between actions
         self.ctx = qe.Context(qe.GRAPH if mode == "graph" else qe.EAGER, device.index or 0,
                               exec_stream=(torch.cuda.current_stream().cuda_stream or None) if same_stream else None,
-                              overlap_dw=overlap_dw)
+                              overlap_dw=overlap_dw, step_window=max(2, cfg["sched"][0] + cfg["sched"][1]))
         self.schedule = sched(cfg["M"], *cfg["sched"])
         P = peak_live(self.schedule)
         if plan_window:

@@ -154,7 +154,9 @@ typedef struct qe_ctx_config {
                          on; an action called with that same stream as caller_stream needs no event handoff, stream
                          order gives both directions of the completion guarantee.                                     */
   uint32_t flags;     /* QE_CTX_* bits                                                                                 */
-  uint32_t reserved[3];
+  uint32_t step_window; /* qe_step_run: how many units of the list it looks ahead when it cuts the list into rounds of
+                         independent actions (0: default 4; 1: action by action, only consecutive dW grouped)         */
+  uint32_t reserved[2];
 } qe_ctx_config;
 /* Run the deferred weight-gradient actions on a second, lower-priority stream of the context so that their
  * thread blocks fill SMs the forward / input-gradient kernels leave idle (dW never touches scaling state, which is
@@ -324,13 +326,15 @@ int32_t qe_next_slot(const qe_layer*, uint32_t* slot_out);
  * wait and ONE execution->caller event: in eager mode as plain launches, in graph mode as one captured graph that is
  * cached per (layers, actions) and replayed, with kernel-node parameters patched where pointers or the accumulate flag
  * differ from the previous replay.  dW runs on the execution stream here (QE_CTX_OVERLAP_DW does not apply).
- * Independent neighbours share launches, with bit-identical results (only the slot a tape lands in may differ from
- * the one-by-one order): consecutive dW actions of different layers as in qe_backward_dW_multi; and, when n forward
- * actions of one microbatch over n different layers are directly followed by n input-gradient actions of another
- * microbatch (and those possibly by n weight-gradient actions of a third), the i-th action of each run is issued
- * together as qe_run_together would; likewise n input-gradient actions directly followed by n weight-gradient
- * actions of another microbatch (none of this with temp_dev).
- * If a check fails at action k, the kernels of actions 0..k-1 are still issued (device and host state stay in step),
+ * Independent actions share launches, with bit-identical results (only the slot a tape lands in may differ from the
+ * one-by-one order).  The list is read as units -- runs of actions of one kind and microbatch over distinct layers: a
+ * forward, input-gradient or weight-gradient unit of the stage -- and cut into rounds of up to QE_MAX_TOGETHER actions
+ * whose predecessors were issued in earlier rounds (the previous layer of the own unit for F and dI, the same layer of
+ * the previous unit of the kind, F before dI before dW of a (layer, microbatch), a free tape slot), looking
+ * qe_ctx_config.step_window units ahead of the earliest unfinished one; a round is issued as qe_run_together would.
+ * With temp_dev, with step_window 1, or when the list admits no such plan, actions go one by one and only
+ * consecutive dW actions of different layers share launches (as in qe_backward_dW_multi).
+ * If a check fails at action k (the first action of the failing round), the kernels issued so far still run (device and host state stay in step),
  * then every layer of the list is aborted as at a failure boundary (Sec. 4.5) and the failing check's status is
  * returned; qe_arena_rebuild restarts the epoch. */
 typedef struct qe_step_action { uint32_t kind; uint32_t layer; uint32_t mb; uint32_t reserved; } qe_step_action;

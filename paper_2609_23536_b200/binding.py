@@ -63,7 +63,7 @@ class qe_contract_view(C.Structure):
 
 
 class qe_ctx_config(C.Structure):
-    _fields_ = [("exec_mode", C.c_uint32), ("device", C.c_int32), ("exec_stream", C.c_void_p), ("flags", C.c_uint32), ("reserved", C.c_uint32 * 3)]
+    _fields_ = [("exec_mode", C.c_uint32), ("device", C.c_int32), ("exec_stream", C.c_void_p), ("flags", C.c_uint32), ("step_window", C.c_uint32), ("reserved", C.c_uint32 * 2)]
 
 
 class qe_layer_config(C.Structure):
@@ -309,10 +309,10 @@ def contract_view_to_dict(v: qe_contract_view) -> dict:
 
 # ---------------------------------------------------------------------------------------- layer API
 class Context:
-    def __init__(self, exec_mode=EAGER, device=0, exec_stream=None, overlap_dw=False, unsafe_one_way=False):
+    def __init__(self, exec_mode=EAGER, device=0, exec_stream=None, overlap_dw=False, unsafe_one_way=False, step_window=0):
         """exec_stream: a cudaStream_t (int) the context should execute on, or None for a context-owned stream.
         overlap_dw: QE_CTX_OVERLAP_DW (dW actions on a second stream, joined at the optimizer boundary)."""
-        cfg = qe_ctx_config(exec_mode=exec_mode, device=device, exec_stream=exec_stream, flags=(OVERLAP_DW if overlap_dw else 0) | (UNSAFE_ONE_WAY_HANDOFF if unsafe_one_way else 0))
+        cfg = qe_ctx_config(exec_mode=exec_mode, device=device, exec_stream=exec_stream, flags=(OVERLAP_DW if overlap_dw else 0) | (UNSAFE_ONE_WAY_HANDOFF if unsafe_one_way else 0), step_window=step_window)
         self.h = _P()
         _check(lib.qe_ctx_create(C.byref(cfg), C.byref(self.h)))
         self.exec_mode = exec_mode

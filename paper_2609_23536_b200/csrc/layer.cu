@@ -122,6 +122,7 @@ struct qe_ctx {
   cudaStream_t exec_stream = nullptr;
   bool owns_stream = true;
   bool one_way = false;              // QE_CTX_UNSAFE_ONE_WAY_HANDOFF
+  uint32_t step_window = 4;          // qe_step_run: units looked ahead when planning rounds (1: action by action)
   cudaStream_t dw_stream = nullptr;  // only with QE_CTX_OVERLAP_DW
   cudaEvent_t ev_dw_in = nullptr;
   cudaEvent_t ev_in = nullptr, ev_out = nullptr;
@@ -655,6 +656,7 @@ int32_t qe_ctx_create(const qe_ctx_config* cfg, qe_ctx** out) {
   c->dev = d;
   c->exec_mode = cfg->exec_mode;
   c->one_way = (cfg->flags & QE_CTX_UNSAFE_ONE_WAY_HANDOFF) != 0;
+  if (cfg->step_window) c->step_window = cfg->step_window > 64 ? 64 : cfg->step_window;
   e = cudaSuccess;
   if (cfg->exec_stream) {
     c->exec_stream = (cudaStream_t)cfg->exec_stream;
@@ -1353,99 +1355,116 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
     if (!layers[l] || layers[l]->ctx != ctx) return fail(QE_ERR_BAD_ARG, "layer %u is null or belongs to another context", l);
   cudaStream_t caller = (cudaStream_t)caller_stream;
 
-  // ---- host pass: check -> collect launches -> commit, action by action (Algorithm 1)
   std::vector<qe_tape> tapes((size_t)n_layers * M);
   std::vector<uint8_t> have((size_t)n_layers * M, 0);
   std::vector<qe::Launch> ls;
   ls.reserve(2 * (size_t)n_actions + n_layers);
   int32_t st = QE_OK;
   uint32_t k = 0;
+
+  // ---- issue plan.  The list is read as units (runs of actions of one kind and microbatch over distinct layers: a
+  // forward, input-gradient or weight-gradient unit of the stage).  Units a stage holds at the same time are
+  // independent, so the list is cut into rounds of actions whose predecessors were issued in earlier rounds -- the
+  // previous layer of the own unit (F and dI walk their layers in list order), the same layer of the previous unit of
+  // the kind, F before dI before dW of a (layer, microbatch), a free tape slot -- looking `window` units ahead, and a
+  // round goes out as qe_run_together would issue it.  If no such plan exists (an illegal list) the action-by-action
+  // pass below runs instead and reports the failing action.
+  std::vector<std::vector<uint32_t>> rounds;  // indices into actions[]
+  if (!temp && ctx->step_window > 1) {
+    struct Unit { uint32_t kind, mb, begin, end, done; int prev; };
+    std::vector<Unit> units;
+    std::vector<uint8_t> taken(n_actions, 0);
+    bool ok = true;
+    int last_of_kind[3] = {-1, -1, -1};
+    for (uint32_t i = 0; i < n_actions && ok; ++i) {
+      const qe_step_action& a = actions[i];
+      ok = a.kind <= QE_ACT_DW && a.layer < n_layers && a.mb < M;
+      if (!ok) break;
+      bool fresh = units.empty() || units.back().kind != a.kind || units.back().mb != a.mb;
+      for (uint32_t j = fresh ? i : units.back().begin; !fresh && j < i; ++j) fresh = actions[j].layer == a.layer;
+      if (fresh) {
+        units.push_back(Unit{a.kind, a.mb, i, i, 0, last_of_kind[a.kind]});
+        last_of_kind[a.kind] = (int)units.size() - 1;
+      }
+      units.back().end = i + 1;
+    }
+    std::vector<uint8_t> issued((size_t)3 * n_layers * M, 0);  // [kind][layer][mb]
+    auto was = [&](uint32_t kind, uint32_t layer, uint32_t mb) -> uint8_t& { return issued[((size_t)kind * n_layers + layer) * M + mb]; };
+    std::vector<uint32_t> live(n_layers);
+    for (uint32_t l = 0; l < n_layers; ++l) live[l] = layers[l]->contract->live_tapes();
+    size_t first = 0;
+    while (ok && first < units.size()) {
+      std::vector<uint32_t> group;
+      for (size_t ui = first; ui < units.size() && ui < first + ctx->step_window && group.size() < QE_MAX_TOGETHER; ++ui) {
+        const Unit& u = units[ui];
+        for (uint32_t i = u.begin; i < u.end && group.size() < QE_MAX_TOGETHER; ++i) {
+          if (taken[i]) continue;
+          const qe_step_action& a = actions[i];
+          bool ready = true;
+          for (uint32_t gi : group)  // one action of a kind per layer, never two of one (layer, microbatch)
+            ready = ready && !((actions[gi].kind == a.kind && actions[gi].layer == a.layer) || (actions[gi].layer == a.layer && actions[gi].mb == a.mb));
+          if (u.prev >= 0) {  // each layer sees the units of a kind in list order
+            const Unit& p = units[u.prev];
+            for (uint32_t j = p.begin; j < p.end; ++j)
+              if (actions[j].layer == a.layer) ready = ready && taken[j] == 2;
+          }
+          if (a.kind == QE_ACT_F) ready = ready && live[a.layer] < layers[a.layer]->cfg.slots;
+          if (a.kind == QE_ACT_DI) ready = ready && was(QE_ACT_F, a.layer, a.mb) == 2;
+          if (a.kind == QE_ACT_DW) ready = ready && was(QE_ACT_DI, a.layer, a.mb) == 2;
+          if (ready) {
+            group.push_back(i);
+            taken[i] = 1;
+          }
+          if (a.kind != QE_ACT_DW) break;  // F and dI: only the unit's next layer can be ready
+        }
+      }
+      if (group.empty()) {
+        ok = false;
+        break;
+      }
+      for (uint32_t gi : group) {  // visible to later rounds only
+        const qe_step_action& a = actions[gi];
+        taken[gi] = 2;
+        was(a.kind, a.layer, a.mb) = 2;
+        if (a.kind == QE_ACT_F) live[a.layer] += 1;
+        if (a.kind == QE_ACT_DW) live[a.layer] -= 1;
+      }
+      // F and dI actions must be taken in the unit's order: mark "next" by skipping taken ones above; advance `first`
+      rounds.push_back(group);
+      while (first < units.size()) {
+        bool all = true;
+        for (uint32_t i = units[first].begin; i < units[first].end; ++i) all = all && taken[i] == 2;
+        if (!all) break;
+        ++first;
+      }
+    }
+    if (!ok) rounds.clear();
+  }
+  for (size_t r = 0; r < rounds.size() && st == QE_OK; ++r) {
+    qe_action acts[QE_MAX_TOGETHER];
+    uint32_t na = 0;
+    for (uint32_t gi : rounds[r]) {
+      const qe_step_action& a = actions[gi];
+      const size_t u = (size_t)a.layer * M + a.mb;
+      qe_layer* L = layers[a.layer];
+      if (a.kind == QE_ACT_F) acts[na++] = qe_action{QE_ACT_F, a.mb, L->contract->e_W, L, io[u].x_dev, io[u].y_dev, &tapes[u], 0};
+      else if (a.kind == QE_ACT_DI) acts[na++] = qe_action{QE_ACT_DI, 0, 0, L, io[u].dy_dev, io[u].dx_dev, &tapes[u], 0};
+      else acts[na++] = qe_action{QE_ACT_DW, 0, 0, L, nullptr, nullptr, &tapes[u], offsets[a.layer]};
+    }
+    TogetherPrep pr;
+    if ((st = together_prepare(ctx, acts, na, grad, grad_elems, &pr)) != QE_OK || (st = together_build(ctx, acts, na, pr, grad, ls, nullptr)) != QE_OK) {
+      k = rounds[r][0];  // (reported as the index of the first action of the failing round)
+      break;
+    }
+    st = together_commit(acts, na, grad, pr);
+  }
+  if (!rounds.empty()) k = st == QE_OK ? n_actions : k;
+
+  // ---- host pass: check -> collect launches -> commit, action by action (Algorithm 1)
   DWBatch dwb;
-  for (; k < n_actions && st == QE_OK; ++k) {
+  for (; rounds.empty() && k < n_actions && st == QE_OK; ++k) {
     const qe_step_action& a = actions[k];
     if (a.kind != QE_ACT_DW && dwb.n) dwb.flush(ctx, ls);
-    // A forward unit directly followed by an input-gradient unit of another microbatch (and possibly a deferred
-    // weight-gradient unit of a third): the units' chains through the layers are independent, so the i-th action of
-    // each goes out together, as qe_run_together would issue them.
-    if (a.kind == QE_ACT_DI && !temp && a.mb < M) {
-      // cool-down: an input-gradient unit directly followed by a weight-gradient unit of an earlier microbatch
-      uint32_t nd = 0;
-      while (k + nd < n_actions && actions[k + nd].kind == QE_ACT_DI && actions[k + nd].mb == a.mb && actions[k + nd].layer < n_layers) ++nd;
-      bool ok = k + 2 * nd <= n_actions;
-      uint32_t mw = ok ? actions[k + nd].mb : 0;
-      for (uint32_t i = 0; ok && i < nd; ++i) {
-        const qe_step_action &ai = actions[k + i], &aw = actions[k + nd + i];
-        ok = aw.kind == QE_ACT_DW && aw.mb == mw && mw != a.mb && mw < M && aw.layer < n_layers &&
-             have[(size_t)ai.layer * M + a.mb] && have[(size_t)aw.layer * M + mw];
-        for (uint32_t j = 0; ok && j < i; ++j) ok = actions[k + j].layer != ai.layer && actions[k + nd + j].layer != aw.layer;
-      }
-      if (ok) {
-        uint32_t i = 0;
-        for (; i < nd && st == QE_OK; ++i) {
-          const qe_step_action &ai = actions[k + i], &aw = actions[k + nd + i];
-          const size_t ui = (size_t)ai.layer * M + a.mb;
-          qe_action acts[2];
-          acts[0] = qe_action{QE_ACT_DI, 0, 0, layers[ai.layer], io[ui].dy_dev, io[ui].dx_dev, &tapes[ui], 0};
-          acts[1] = qe_action{QE_ACT_DW, 0, 0, layers[aw.layer], nullptr, nullptr, &tapes[(size_t)aw.layer * M + mw], offsets[aw.layer]};
-          TogetherPrep pr;
-          if ((st = together_prepare(ctx, acts, 2, grad, grad_elems, &pr)) != QE_OK) break;
-          if ((st = together_build(ctx, acts, 2, pr, grad, ls, nullptr)) != QE_OK) break;
-          st = together_commit(acts, 2, grad, pr);
-        }
-        if (st != QE_OK) {
-          k += i;
-          break;
-        }
-        k += 2 * nd - 1;
-        continue;
-      }
-    }
-    if (a.kind == QE_ACT_F && !temp) {
-      uint32_t nf = 0;
-      while (k + nf < n_actions && actions[k + nf].kind == QE_ACT_F && actions[k + nf].mb == a.mb && actions[k + nf].layer < n_layers) ++nf;
-      auto run_of = [&](uint32_t start, uint32_t kind, uint32_t* mb_out) {  // nf actions of `kind`, one microbatch, distinct layers
-        if (start + nf > n_actions) return false;
-        for (uint32_t i = 0; i < nf; ++i) {
-          const qe_step_action& b = actions[start + i];
-          if (b.kind != kind || b.mb != actions[start].mb || b.layer >= n_layers || b.mb >= M) return false;
-          for (uint32_t j = 0; j < i; ++j)
-            if (actions[start + j].layer == b.layer) return false;
-        }
-        *mb_out = actions[start].mb;
-        return true;
-      };
-      uint32_t mf = 0, mb_i = 0, mb_w = 0;
-      bool ok = a.mb < M && run_of(k, QE_ACT_F, &mf) && run_of(k + nf, QE_ACT_DI, &mb_i) && mb_i != mf;
-      for (uint32_t i = 0; ok && i < nf; ++i) ok = have[(size_t)actions[k + nf + i].layer * M + mb_i] != 0;
-      bool with_dw = ok && run_of(k + 2 * nf, QE_ACT_DW, &mb_w) && mb_w != mf && mb_w != mb_i;
-      for (uint32_t i = 0; with_dw && i < nf; ++i) with_dw = have[(size_t)actions[k + 2 * nf + i].layer * M + mb_w] != 0;
-      if (ok) {
-        uint32_t i = 0;
-        for (; i < nf && st == QE_OK; ++i) {
-          const qe_step_action &af = actions[k + i], &ai = actions[k + nf + i];
-          const size_t uf = (size_t)af.layer * M + mf, ui = (size_t)ai.layer * M + mb_i;
-          qe_action acts[3];
-          uint32_t na = 2;
-          acts[0] = qe_action{QE_ACT_F, mf, layers[af.layer]->contract->e_W, layers[af.layer], io[uf].x_dev, io[uf].y_dev, &tapes[uf], 0};
-          acts[1] = qe_action{QE_ACT_DI, 0, 0, layers[ai.layer], io[ui].dy_dev, io[ui].dx_dev, &tapes[ui], 0};
-          if (with_dw) {
-            const qe_step_action& aw = actions[k + 2 * nf + i];
-            acts[na++] = qe_action{QE_ACT_DW, 0, 0, layers[aw.layer], nullptr, nullptr, &tapes[(size_t)aw.layer * M + mb_w], offsets[aw.layer]};
-          }
-          TogetherPrep pr;
-          if ((st = together_prepare(ctx, acts, na, grad, grad_elems, &pr)) != QE_OK) break;
-          if ((st = together_build(ctx, acts, na, pr, grad, ls, nullptr)) != QE_OK) break;
-          st = together_commit(acts, na, grad, pr);
-          have[uf] = 1;
-        }
-        if (st != QE_OK) {
-          k += i;  // (reported as the index of the forward action of the failing group)
-          break;
-        }
-        k += (with_dw ? 3 : 2) * nf - 1;
-        continue;
-      }
-    }
     if (a.layer >= n_layers || a.mb >= M || a.kind > QE_ACT_DW) {
       st = fail(QE_ERR_BAD_ARG, "action %u: kind %u layer %u mb %u", k, a.kind, a.layer, a.mb);
       break;
