@@ -15,7 +15,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OUT = os.path.join(HERE, "libqe.so")
-SOURCES = ["error.cpp", "contract.cpp", "kernels_hbm.cu", "gemm_sm100.cu", "layer.cu", "noalloc.cu"]
+SOURCES = ["error.cpp", "contract.cpp", "kernels_hbm.cu", "gemm_sm100.cu", "layer_core.cu", "layer.cu", "layer_group.cu",
+           "standalone.cu", "noalloc.cu"]
 
 
 def _nvcc() -> str:
