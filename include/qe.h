@@ -343,6 +343,15 @@ typedef struct qe_step_io { const void* x_dev; void* y_dev; const void* dy_dev; 
 int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, const qe_step_action* actions,
                     uint32_t n_actions, uint32_t microbatches, const qe_step_io* io, float* grad_buf_dev,
                     uint64_t grad_buf_elems, const uint64_t* offsets, float* temp_dev, void* caller_stream);
+/* The issue plan qe_step_run makes, as host logic of its own (no device needed): cuts actions[0..n) into rounds as
+ * described above.  slots[l]: tape slots of layer l; live_now[l]: tapes of layer l alive before the list (NULL: none);
+ * window >= 1 units of look-ahead; max_group actions per round.  round_of_action[i] receives the round of action i
+ * (rounds are numbered from 0 in issue order), *n_rounds_out their number.  ORDER if the list admits no plan (an
+ * action whose predecessors never become ready, or a pool too small), BAD_ARG for a malformed action. */
+int32_t qe_plan_rounds(const qe_step_action* actions, uint32_t n_actions, uint32_t n_layers, uint32_t microbatches,
+                       const uint32_t* slots, const uint32_t* live_now, uint32_t window, uint32_t max_group,
+                       uint32_t* round_of_action, uint32_t* n_rounds_out);
+
 
 typedef struct qe_class_state {
   float scale, scale_inv;

@@ -154,6 +154,8 @@ _SIGNATURES = {
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
     "qe_forward_dI_pair": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, C.POINTER(qe_tape), _P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_gemm_fp8_group": (C.c_int32, [C.POINTER(qe_gemm_desc), C.c_uint32, _P, _P]),
+    "qe_plan_rounds": (C.c_int32, [C.POINTER(qe_step_action), C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32),
+                                   C.POINTER(C.c_uint32), C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]),
     "qe_run_together": (C.c_int32, [_P, C.POINTER(qe_action), C.c_uint32, _P, C.c_uint64, _P]),
     "qe_forward_chain": (C.c_int32, [C.POINTER(_P), C.c_uint32, C.c_uint32, C.c_uint64, _P, _P, _P, C.POINTER(qe_tape)]),
     "qe_backward_dI_chain": (C.c_int32, [C.POINTER(_P), C.POINTER(qe_tape), C.c_uint32, _P, _P, _P]),
@@ -519,6 +521,21 @@ def qe_gemm_fp8_group(problems, status, stream=None):
         Kc = a.shape[0] if amn else a.shape[1]
         arr[i] = qe_gemm_desc(_ptr(a), _ptr(b), _ptr(d), _ptr(sa), _ptr(sb), _ptr(amax), af, int(amn), bf, int(bmn), M, Nn, Kc, kind)
     _check(lib.qe_gemm_fp8_group(arr, n, _ptr(status), _stream(stream)))
+
+
+def plan_rounds(actions, n_layers, microbatches, slots, window, max_group=8, live_now=None):
+    """qe_plan_rounds (host only).  actions: (kind name, layer, mb) triples; returns the rounds as lists of triples."""
+    n = len(actions)
+    arr = (qe_step_action * n)(*[qe_step_action(ACT[k], l, m, 0) for k, l, m in actions])
+    sl = (C.c_uint32 * n_layers)(*([slots] * n_layers if isinstance(slots, int) else slots))
+    lv = (C.c_uint32 * n_layers)(*live_now) if live_now is not None else None
+    rnd = (C.c_uint32 * n)()
+    nr = C.c_uint32()
+    _check(lib.qe_plan_rounds(arr, n, n_layers, microbatches, sl, lv, window, max_group, rnd, C.byref(nr)))
+    out = [[] for _ in range(nr.value)]
+    for i, a in enumerate(actions):
+        out[rnd[i]].append(tuple(a))
+    return out
 
 
 def run_together(ctx, actions, grad_buf=None, stream=None):

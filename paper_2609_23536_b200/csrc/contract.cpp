@@ -4,6 +4,7 @@
 
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "error.h"
 
@@ -278,6 +279,82 @@ int32_t qe_contract_get(const qe_contract* c, qe_contract_view* v) {
     v->slot[p].bits = c->slot[p].bits;
     v->slot[p].key = c->slot[p].key;
   }
+  return QE_OK;
+}
+
+// ---- issue plan of a whole-step action list (host logic only; used by qe_step_run)
+int32_t qe_plan_rounds(const qe_step_action* actions, uint32_t n_actions, uint32_t n_layers, uint32_t microbatches,
+                       const uint32_t* slots, const uint32_t* live_now, uint32_t window, uint32_t max_group,
+                       uint32_t* round_of_action, uint32_t* n_rounds_out) {
+  if (!actions || !slots || !round_of_action || !n_rounds_out) return fail(QE_ERR_BAD_ARG, "null argument");
+  if (n_actions == 0 || n_layers == 0 || microbatches == 0 || window == 0 || max_group == 0) return fail(QE_ERR_BAD_ARG, "empty list or zero limit");
+  const uint32_t M = microbatches;
+  struct Unit { uint32_t kind, mb, begin, end; int prev; };
+  std::vector<Unit> units;
+  std::vector<uint8_t> taken(n_actions, 0);
+  int last_of_kind[3] = {-1, -1, -1};
+  for (uint32_t i = 0; i < n_actions; ++i) {
+    const qe_step_action& a = actions[i];
+    if (a.kind > QE_ACT_DW || a.layer >= n_layers || a.mb >= M) return fail(QE_ERR_BAD_ARG, "action %u: kind %u layer %u mb %u", i, a.kind, a.layer, a.mb);
+    // a unit: a run of actions of one kind and microbatch over distinct layers
+    bool fresh = units.empty() || units.back().kind != a.kind || units.back().mb != a.mb;
+    for (uint32_t j = fresh ? i : units.back().begin; !fresh && j < i; ++j) fresh = actions[j].layer == a.layer;
+    if (fresh) {
+      units.push_back(Unit{a.kind, a.mb, i, i, last_of_kind[a.kind]});
+      last_of_kind[a.kind] = (int)units.size() - 1;
+    }
+    units.back().end = i + 1;
+  }
+  std::vector<uint8_t> issued((size_t)3 * n_layers * M, 0);  // [kind][layer][mb]
+  auto was = [&](uint32_t kind, uint32_t layer, uint32_t mb) -> uint8_t& { return issued[((size_t)kind * n_layers + layer) * M + mb]; };
+  std::vector<uint32_t> live(n_layers, 0);
+  for (uint32_t l = 0; live_now && l < n_layers; ++l) live[l] = live_now[l];
+  size_t first = 0;
+  uint32_t round = 0;
+  std::vector<uint32_t> group;
+  while (first < units.size()) {
+    group.clear();
+    for (size_t ui = first; ui < units.size() && ui < first + window && group.size() < max_group; ++ui) {
+      const Unit& u = units[ui];
+      for (uint32_t i = u.begin; i < u.end && group.size() < max_group; ++i) {
+        if (taken[i]) continue;
+        const qe_step_action& a = actions[i];
+        bool ready = true;
+        for (uint32_t gi : group)  // one action of a kind per layer, never two of one (layer, microbatch)
+          ready = ready && !((actions[gi].kind == a.kind && actions[gi].layer == a.layer) || (actions[gi].layer == a.layer && actions[gi].mb == a.mb));
+        if (u.prev >= 0) {  // each layer sees the units of a kind in list order
+          const Unit& p = units[u.prev];
+          for (uint32_t j = p.begin; j < p.end; ++j)
+            if (actions[j].layer == a.layer) ready = ready && taken[j] == 2;
+        }
+        if (a.kind == QE_ACT_F) ready = ready && live[a.layer] < slots[a.layer];
+        if (a.kind == QE_ACT_DI) ready = ready && was(QE_ACT_F, a.layer, a.mb) == 2;
+        if (a.kind == QE_ACT_DW) ready = ready && was(QE_ACT_DI, a.layer, a.mb) == 2;
+        if (ready) {
+          group.push_back(i);
+          taken[i] = 1;
+        }
+        if (a.kind != QE_ACT_DW) break;  // F and dI walk their layers in list order: only the next one can be ready
+      }
+    }
+    if (group.empty()) return fail(QE_ERR_ORDER, "no action of units %zu.. is ready: the list is not a legal schedule for these pools", first);
+    for (uint32_t gi : group) {  // visible to later rounds only
+      const qe_step_action& a = actions[gi];
+      taken[gi] = 2;
+      was(a.kind, a.layer, a.mb) = 2;
+      if (a.kind == QE_ACT_F) live[a.layer] += 1;
+      if (a.kind == QE_ACT_DW && live[a.layer]) live[a.layer] -= 1;
+      round_of_action[gi] = round;
+    }
+    ++round;
+    while (first < units.size()) {
+      bool all = true;
+      for (uint32_t i = units[first].begin; i < units[first].end; ++i) all = all && taken[i] == 2;
+      if (!all) break;
+      ++first;
+    }
+  }
+  *n_rounds_out = round;
   return QE_OK;
 }
 

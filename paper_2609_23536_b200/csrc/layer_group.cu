@@ -376,74 +376,17 @@ int32_t qe_step_run(qe_ctx* ctx, qe_layer* const* layers, uint32_t n_layers, con
   // pass below runs instead and reports the failing action.
   std::vector<std::vector<uint32_t>> rounds;  // indices into actions[]
   if (!temp && ctx->step_window > 1) {
-    struct Unit { uint32_t kind, mb, begin, end, done; int prev; };
-    std::vector<Unit> units;
-    std::vector<uint8_t> taken(n_actions, 0);
-    bool ok = true;
-    int last_of_kind[3] = {-1, -1, -1};
-    for (uint32_t i = 0; i < n_actions && ok; ++i) {
-      const qe_step_action& a = actions[i];
-      ok = a.kind <= QE_ACT_DW && a.layer < n_layers && a.mb < M;
-      if (!ok) break;
-      bool fresh = units.empty() || units.back().kind != a.kind || units.back().mb != a.mb;
-      for (uint32_t j = fresh ? i : units.back().begin; !fresh && j < i; ++j) fresh = actions[j].layer == a.layer;
-      if (fresh) {
-        units.push_back(Unit{a.kind, a.mb, i, i, 0, last_of_kind[a.kind]});
-        last_of_kind[a.kind] = (int)units.size() - 1;
-      }
-      units.back().end = i + 1;
+    std::vector<uint32_t> slots(n_layers), live(n_layers), round_of(n_actions);
+    for (uint32_t l = 0; l < n_layers; ++l) {
+      slots[l] = layers[l]->cfg.slots;
+      live[l] = layers[l]->contract->live_tapes();
     }
-    std::vector<uint8_t> issued((size_t)3 * n_layers * M, 0);  // [kind][layer][mb]
-    auto was = [&](uint32_t kind, uint32_t layer, uint32_t mb) -> uint8_t& { return issued[((size_t)kind * n_layers + layer) * M + mb]; };
-    std::vector<uint32_t> live(n_layers);
-    for (uint32_t l = 0; l < n_layers; ++l) live[l] = layers[l]->contract->live_tapes();
-    size_t first = 0;
-    while (ok && first < units.size()) {
-      std::vector<uint32_t> group;
-      for (size_t ui = first; ui < units.size() && ui < first + ctx->step_window && group.size() < QE_MAX_TOGETHER; ++ui) {
-        const Unit& u = units[ui];
-        for (uint32_t i = u.begin; i < u.end && group.size() < QE_MAX_TOGETHER; ++i) {
-          if (taken[i]) continue;
-          const qe_step_action& a = actions[i];
-          bool ready = true;
-          for (uint32_t gi : group)  // one action of a kind per layer, never two of one (layer, microbatch)
-            ready = ready && !((actions[gi].kind == a.kind && actions[gi].layer == a.layer) || (actions[gi].layer == a.layer && actions[gi].mb == a.mb));
-          if (u.prev >= 0) {  // each layer sees the units of a kind in list order
-            const Unit& p = units[u.prev];
-            for (uint32_t j = p.begin; j < p.end; ++j)
-              if (actions[j].layer == a.layer) ready = ready && taken[j] == 2;
-          }
-          if (a.kind == QE_ACT_F) ready = ready && live[a.layer] < layers[a.layer]->cfg.slots;
-          if (a.kind == QE_ACT_DI) ready = ready && was(QE_ACT_F, a.layer, a.mb) == 2;
-          if (a.kind == QE_ACT_DW) ready = ready && was(QE_ACT_DI, a.layer, a.mb) == 2;
-          if (ready) {
-            group.push_back(i);
-            taken[i] = 1;
-          }
-          if (a.kind != QE_ACT_DW) break;  // F and dI: only the unit's next layer can be ready
-        }
-      }
-      if (group.empty()) {
-        ok = false;
-        break;
-      }
-      for (uint32_t gi : group) {  // visible to later rounds only
-        const qe_step_action& a = actions[gi];
-        taken[gi] = 2;
-        was(a.kind, a.layer, a.mb) = 2;
-        if (a.kind == QE_ACT_F) live[a.layer] += 1;
-        if (a.kind == QE_ACT_DW) live[a.layer] -= 1;
-      }
-      // F and dI actions must be taken in the unit's order: mark "next" by skipping taken ones above; advance `first`
-      rounds.push_back(group);
-      while (first < units.size()) {
-        bool all = true;
-        for (uint32_t i = units[first].begin; i < units[first].end; ++i) all = all && taken[i] == 2;
-        if (!all) break;
-        ++first;
-      }
+    uint32_t n_rounds = 0;
+    if (qe_plan_rounds(actions, n_actions, n_layers, M, slots.data(), live.data(), ctx->step_window, QE_MAX_TOGETHER,
+                       round_of.data(), &n_rounds) == QE_OK) {
+      rounds.resize(n_rounds);
+      for (uint32_t i = 0; i < n_actions; ++i) rounds[round_of[i]].push_back(i);
     }
-    if (!ok) rounds.clear();
   }
   for (size_t r = 0; r < rounds.size() && st == QE_OK; ++r) {
     qe_action acts[QE_MAX_TOGETHER];

@@ -54,3 +54,49 @@ def test_plan_for_the_benchmark_schedule_groups_most_actions():
     assert rounds[0] == [("F", 0, 0)] and rounds[1] == [("F", 1, 0), ("F", 0, 1)]  # warm-up wavefront
     with pytest.raises(RuntimeError):
         plan_rounds(s, 4, 2, 4, 4)  # two slots cannot hold this schedule
+
+
+# ------------------------------------------------------------------------------------------ the library's own planner
+@pytest.fixture(scope="module")
+def qe():
+    from paper_2609_23536_b200 import build
+
+    build.build()
+    from paper_2609_23536_b200 import binding
+
+    return binding
+
+
+def _actions(schedule, n):
+    return [(a, l, m) for a, m in schedule for l in (range(n) if a == "F" else range(n - 1, -1, -1))]
+
+
+@pytest.mark.parametrize("M,w,d", [(4, 1, 0), (8, 3, 3), (8, 1, 2), (6, 2, 1), (32, 3, 3)])
+@pytest.mark.parametrize("n", [1, 3, 4])
+@pytest.mark.parametrize("window,group", [(1, 4), (2, 4), (4, 8), (6, 8)])
+def test_native_planner_makes_the_same_legal_plan(qe, M, w, d, n, window, group):
+    """qe_plan_rounds (what qe_step_run uses; host logic, no device) against schedules.plan_rounds (what bench.py uses)."""
+    s = sched(M, w, d)
+    slots = peak_live(s)
+    native = qe.plan_rounds(_actions(s, n), n, M, slots, window, group)
+    _check(s, n, slots, native, group)
+    assert native == plan_rounds(s, n, slots, group, window)
+
+
+def test_native_planner_refuses_lists_without_a_plan(qe):
+    s = sched(8, 3, 3)
+    with pytest.raises(qe.QEError) as e:
+        qe.plan_rounds(_actions(s, 4), 4, 8, 2, 4, 8)  # two slots cannot hold seven live tapes
+    assert e.value.code == "ORDER"
+    with pytest.raises(qe.QEError) as e:
+        qe.plan_rounds([("dI", 0, 0), ("F", 0, 0), ("dW", 0, 0)], 1, 1, 1, 1, 8)  # dI before its forward, no look-ahead
+    assert e.value.code == "ORDER"
+    with pytest.raises(qe.QEError) as e:
+        qe.plan_rounds([("F", 3, 0)], 1, 1, 1, 4, 8)
+    assert e.value.code == "BAD_ARG"
+    # (with look-ahead the forward is simply taken first)
+    assert qe.plan_rounds([("dI", 0, 0), ("F", 0, 0), ("dW", 0, 0)], 1, 1, 1, 4, 8) == [[("F", 0, 0)], [("dI", 0, 0)], [("dW", 0, 0)]]
+    # tapes alive before the list count against the pool
+    assert len(qe.plan_rounds([("F", 0, 0), ("dI", 0, 0), ("dW", 0, 0)], 1, 1, 2, 4, 8, live_now=[1])) == 3
+    with pytest.raises(qe.QEError):
+        qe.plan_rounds([("F", 0, 0), ("dI", 0, 0), ("dW", 0, 0)], 1, 1, 2, 4, 8, live_now=[2])
