@@ -334,6 +334,8 @@ int32_t qe_next_slot(const qe_layer*, uint32_t* slot_out);
  * qe_ctx_config.step_window units ahead of the earliest unfinished one; a round is issued as qe_run_together would.
  * With temp_dev, with step_window 1, or when the list admits no such plan, actions go one by one and only
  * consecutive dW actions of different layers share launches (as in qe_backward_dW_multi).
+ * (The plan honours dependencies, not positions: an action listed before a predecessor that lies within the look-ahead
+ * simply runs after it.)
  * If a check fails at action k (the first action of the failing round), the kernels issued so far still run (device and host state stay in step),
  * then every layer of the list is aborted as at a failure boundary (Sec. 4.5) and the failing check's status is
  * returned; qe_arena_rebuild restarts the epoch. */
