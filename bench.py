@@ -187,23 +187,34 @@ class Stage:
         tapes = {}
         n = len(self.layers)
         t_issue = time.perf_counter()
-        if self.plan_window and not host_io:
-            # the schedule cut into rounds of independent per-linear actions (schedules.plan_rounds), one call each
+        if self.plan_window:
+            # the schedule cut into rounds of independent per-linear actions (schedules.plan_rounds), one call each;
+            # host_io: host pointers straight into the C-ABI (qe_run_together_host stages, runs and reads back)
+            X, Y, dY, dX = (self.Xh, self.Yh, self.dYh, self.dXh) if host_io else (self.X, self.Y, self.dY, self.dX)
             for group in self.rounds:
                 acts, keys = [], []
                 for a, i, m in group:
                     if a == "F":
-                        acts.append(("F", self.layers[i], m, self.epoch, self.X[m][i], self.Y[m][i]))
+                        acts.append(("F", self.layers[i], m, self.epoch, X[m][i], Y[m][i]))
                         keys.append((m, i))
+                        if host_io:
+                            self.h2d += X[m][i].numel() * 2
+                            self.d2h += Y[m][i].numel() * 2
                     elif a == "dI":
-                        acts.append(("dI", self.layers[i], tapes[(m, i)], self.dY[m][i], self.dX[m][i]))
+                        acts.append(("dI", self.layers[i], tapes[(m, i)], dY[m][i], dX[m][i]))
+                        if host_io:
+                            self.h2d += dY[m][i].numel() * 2
+                            self.d2h += dX[m][i].numel() * 2
                     else:
                         acts.append(("dW", self.layers[i], tapes[(m, i)], self.offsets[i]))
-                for key, t in zip(keys, self.qe.run_together(self.ctx, acts, self.grad)):
+                for key, t in zip(keys, self.qe.run_together(self.ctx, acts, self.grad, host=host_io)):
                     tapes[key] = t
             self.issue_s += time.perf_counter() - t_issue
             for L in self.layers:
                 L.optimizer_boundary(self.cfg["M"])
+            if host_io:  # the step's result: the accumulated gradients, complete after the boundary
+                self.grad_host.copy_(self.grad, non_blocking=True)
+                self.d2h += self.grad.numel() * 4
             self.epoch += 1
             return
         skip = 0
@@ -637,9 +648,11 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     use_step = args.step_api
+    plan_window = 0 if (use_step or args.staged or args.arena or args.chain or not args.together or not args.pair_f_di) else (
+        max(2, cfg["sched"][0] + cfg["sched"][1]) if args.plan < 0 else args.plan)
     stage = Stage(qe, cfg_name, cfg, args.mode, device, same_stream=not args.own_stream,
                   overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena, chain=args.chain, pair_f_di=args.pair_f_di, together=args.together,
-                  plan_window=0 if (use_step or args.staged or args.arena or args.chain or not args.together or not args.pair_f_di) else (max(2, cfg["sched"][0] + cfg["sched"][1]) if args.plan < 0 else args.plan))
+                  plan_window=plan_window)
     if use_step:
         stage.make_plan()
     with ClockSampler(local) as clk:
@@ -672,6 +685,7 @@ def main():
     torch.cuda.empty_cache()
 
     if not args.no_extras:
+        # (one host call per action: finer-grained than qe_run_together_host per round, so more of the transfers overlap)
         stage = Stage(qe, cfg_name, cfg, args.mode, device, host_io=True, same_stream=not args.own_stream, overlap_dw=args.overlap_dw)
         n2 = min(20, max(2, args.steps // 2))
         ms2, _ = time_steps(stage, n2, 3, True, dist)

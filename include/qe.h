@@ -259,6 +259,12 @@ typedef struct qe_action {
 } qe_action;
 int32_t qe_run_together(qe_ctx*, qe_action* actions, uint32_t n, float* grad_buf_dev, uint64_t grad_buf_elems,
                         void* caller_stream);
+/* The same with HOST buffers for the F and dI actions (layers created with host_io = 1): in_dev / out_dev then hold
+ * host pointers (out may be NULL to skip the read-back); every input is uploaded into its layer's staging buffer
+ * first, the kernels run on the staging buffers, the outputs are read back afterwards -- copies on the context's
+ * two copy streams as in qe_forward_host, so the uploads of a call overlap the read-backs of the call before it. */
+int32_t qe_run_together_host(qe_ctx*, qe_action* actions, uint32_t n, float* grad_buf_dev, uint64_t grad_buf_elems,
+                             void* caller_stream);
 /* FP8 hand-off between directly chained linears (layers[i+1] consumes layers[i]'s output: same T,
  * K_{i+1} = N_i; host array of n <= QE_MAX_CHAIN distinct layers of one context).  qe_forward_chain runs F of every
  * layer for microbatch mb: x_dev bf16 [T, K_0] in, y_dev bf16 [T, N_{n-1}] out, tapes_out[n].  The output of

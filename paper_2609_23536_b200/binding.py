@@ -154,6 +154,7 @@ _SIGNATURES = {
     "qe_backward_dW_staged": (C.c_int32, [_P, C.POINTER(qe_tape), _P, C.c_uint64, C.c_uint64, _P, _P]),
     "qe_forward_dI_pair": (C.c_int32, [_P, C.c_uint32, C.c_uint64, _P, _P, C.POINTER(qe_tape), _P, C.POINTER(qe_tape), _P, _P, _P]),
     "qe_gemm_fp8_group": (C.c_int32, [C.POINTER(qe_gemm_desc), C.c_uint32, _P, _P]),
+    "qe_run_together_host": (C.c_int32, [_P, C.POINTER(qe_action), C.c_uint32, _P, C.c_uint64, _P]),
     "qe_plan_rounds": (C.c_int32, [C.POINTER(qe_step_action), C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32),
                                    C.POINTER(C.c_uint32), C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]),
     "qe_run_together": (C.c_int32, [_P, C.POINTER(qe_action), C.c_uint32, _P, C.c_uint64, _P]),
@@ -538,8 +539,8 @@ def plan_rounds(actions, n_layers, microbatches, slots, window, max_group=8, liv
     return out
 
 
-def run_together(ctx, actions, grad_buf=None, stream=None):
-    """qe_run_together.  actions: ("F", layer, mb, gen, x, y) | ("dI", layer, tape, dy, dx) | ("dW", layer, tape, offset).
+def run_together(ctx, actions, grad_buf=None, stream=None, host=False):
+    """qe_run_together (host=True: qe_run_together_host, x / y / dy / dx are pinned host tensors, y / dx may be None).  actions: ("F", layer, mb, gen, x, y) | ("dI", layer, tape, dy, dx) | ("dW", layer, tape, offset).
     Returns the tapes of the F actions, in order."""
     n = len(actions)
     arr = (qe_action * n)()
@@ -556,7 +557,8 @@ def run_together(ctx, actions, grad_buf=None, stream=None):
         else:
             _, L, tape, off = a
             arr[i] = qe_action(ACT["dW"], 0, 0, L.h, None, None, C.pointer(tape), off)
-    _check(lib.qe_run_together(ctx.h, arr, n, _ptr(grad_buf), grad_buf.numel() if grad_buf is not None else 0, _stream(stream)))
+    fn = lib.qe_run_together_host if host else lib.qe_run_together
+    _check(fn(ctx.h, arr, n, _ptr(grad_buf), grad_buf.numel() if grad_buf is not None else 0, _stream(stream)))
     return new_tapes
 
 

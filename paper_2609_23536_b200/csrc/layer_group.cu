@@ -327,12 +327,33 @@ int32_t together_commit(const qe_action* acts, uint32_t n, float* grad, const To
 }
 }  // namespace
 
-int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, void* caller_stream) {
+// host != 0: the in / out pointers of the F and dI actions are HOST buffers, staged through the layers' fixed device
+// buffers like qe_forward_host / qe_backward_dI_host do (uploads of all actions first, read-backs after the kernels).
+static int32_t run_together_impl(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, void* caller_stream,
+                                 int host) {
+  if (!ctx || !acts || n == 0 || n > QE_MAX_TOGETHER) return fail(QE_ERR_BAD_ARG, "null argument or bad count %u", n);
+  qe_action dev[QE_MAX_TOGETHER];
+  for (uint32_t i = 0; i < n; ++i) {
+    dev[i] = acts[i];
+    if (!host || acts[i].kind > QE_ACT_DI || !acts[i].layer) continue;
+    qe_layer* L = acts[i].layer;
+    if (!L->x_stage) return fail(QE_ERR_BAD_ARG, "action %u: layer was created without host_io", i);
+    if (!acts[i].in_dev) return fail(QE_ERR_BAD_ARG, "action %u: host input is null", i);
+    dev[i].in_dev = acts[i].kind == QE_ACT_F ? L->x_stage : L->dy_stage;
+    dev[i].out_dev = acts[i].kind == QE_ACT_F ? L->y_stage : L->dx_stage;
+  }
   TogetherPrep pr;
-  int32_t st = together_prepare(ctx, acts, n, grad, grad_elems, &pr);  // check (every action, before anything runs)
+  int32_t st = together_prepare(ctx, dev, n, grad, grad_elems, &pr);  // check (every action, before anything runs)
   if (st != QE_OK) return st;
   cudaStream_t caller = (cudaStream_t)caller_stream;
   if ((st = handoff_in(ctx, caller)) != QE_OK) return st;
+  if (host)
+    for (uint32_t i = 0; i < n; ++i) {
+      if (acts[i].kind > QE_ACT_DI) continue;
+      const qe_layer_config& c = acts[i].layer->cfg;
+      const size_t bytes = 2ull * c.T * (acts[i].kind == QE_ACT_F ? c.K : c.N);
+      if ((st = host_upload(ctx, const_cast<void*>(dev[i].in_dev), acts[i].in_dev, bytes, caller)) != QE_OK) return st;
+    }
   if (pr.any_dw && ctx->dw_stream) {  // weight gradients issued earlier on the second stream accumulate into the same buffer
     QE_CUDA(cudaEventRecord(ctx->ev_dw_in, ctx->dw_stream));
     QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_dw_in, 0));
@@ -340,13 +361,28 @@ int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, u
   std::vector<qe::Launch> ls;
   Fnv h;
   h.mix("together", 9);
-  if ((st = together_build(ctx, acts, n, pr, grad, ls, &h)) != QE_OK) return st;
+  if ((st = together_build(ctx, dev, n, pr, grad, ls, &h)) != QE_OK) return st;
   if ((st = run_keyed(ctx, h.key, ls)) != QE_OK) return st;  // ... run ...
+  if (host)
+    for (uint32_t i = 0; i < n; ++i) {
+      if (acts[i].kind > QE_ACT_DI) continue;
+      const qe_layer_config& c = acts[i].layer->cfg;
+      const size_t bytes = 2ull * c.T * (acts[i].kind == QE_ACT_F ? c.N : c.K);
+      if ((st = host_download(ctx, acts[i].out_dev, dev[i].out_dev, bytes)) != QE_OK) return st;
+    }
   if (ctx->dw_stream)
     for (uint32_t i = 0; i < n; ++i)
       if (acts[i].kind == QE_ACT_DI) QE_CUDA(cudaEventRecord(acts[i].layer->ev_di[pr.slot[i]], ctx->exec_stream));
   if ((st = handoff_out(ctx, caller)) != QE_OK) return st;
-  return together_commit(acts, n, grad, pr);  // ... commit
+  return together_commit(dev, n, grad, pr);  // ... commit (the tapes are written through the callers' pointers)
+}
+
+int32_t qe_run_together(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, void* caller_stream) {
+  return run_together_impl(ctx, acts, n, grad, grad_elems, caller_stream, 0);
+}
+
+int32_t qe_run_together_host(qe_ctx* ctx, qe_action* acts, uint32_t n, float* grad, uint64_t grad_elems, void* caller_stream) {
+  return run_together_impl(ctx, acts, n, grad, grad_elems, caller_stream, 1);
 }
 
 // ------------------------------------------------------------------------------------------------ whole-step call

@@ -585,3 +585,55 @@ def test_planned_rounds_equal_the_schedule_issued_action_by_action_bitwise(qe, m
     for u, v in zip(a[3], b[3]):
         assert state_equal({**u, "slots": []}, {**v, "slots": []}) and u["device_token"] == v["device_token"]
     assert len(rounds) < len(plain)
+
+
+def test_run_together_host_equals_device_buffers_bitwise(qe):
+    """Rounds with pinned HOST tensors (qe_run_together_host) against the same rounds with device tensors."""
+    from paper_2609_23536_b200.schedules import plan_rounds
+
+    T, M = 256, 4
+    shapes = [(256, 512), (512, 256), (256, 256)]
+    n = len(shapes)
+    offs, total = inputs.grad_offsets([("l", K, N) for K, N in shapes])
+    s = sched(M, 2, 1)
+    P = peak_live(s)
+    rounds = plan_rounds(s, n, P, 8, 4)
+    results = []
+    for host in (False, True):
+        ctx = qe.Context(1)
+        layers = [qe.Layer(ctx, T, K, N, 4, 0, P, inputs.weights("HR", 0, j, N, K).to(DEV), unit=j, host_io=host) for j, (K, N) in enumerate(shapes)]
+        grad = torch.full((total,), float("nan"), device=DEV)
+        place = (lambda t: t.pin_memory()) if host else (lambda t: t.to(DEV))
+        X = [[place(inputs.activations("HR", 0, 0, j, m, T, K)) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+        dY = [[place(inputs.upstream_grads("HR", 0, 0, j, m, T, N)) for j, (K, N) in enumerate(shapes)] for m in range(M)]
+        Y = [[place(torch.zeros((T, N), dtype=torch.bfloat16)) for K, N in shapes] for m in range(M)]
+        dX = [[place(torch.zeros((T, K), dtype=torch.bfloat16)) for K, N in shapes] for m in range(M)]
+        tapes = {}
+        for g in rounds:
+            acts, keys = [], []
+            for a, l, m in g:
+                if a == "F":
+                    acts.append(("F", layers[l], m, 0, X[m][l], Y[m][l]))
+                    keys.append((l, m))
+                elif a == "dI":
+                    acts.append(("dI", layers[l], tapes[(l, m)], dY[m][l], dX[m][l]))
+                else:
+                    acts.append(("dW", layers[l], tapes[(l, m)], offs[l]))
+            for key, t in zip(keys, qe.run_together(ctx, acts, grad, host=host)):
+                tapes[key] = t
+        for L in layers:
+            L.optimizer_boundary(M)
+        torch.cuda.synchronize()
+        results.append(([inputs.bits(t.cpu()) for row in Y for t in row], [inputs.bits(t.cpu()) for row in dX for t in row],
+                        grad.cpu().numpy().copy(), [L.state() for L in layers]))
+    a, b = results
+    for u, v in zip(a[0] + a[1], b[0] + b[1]):
+        assert np.array_equal(u, v)
+    assert np.array_equal(a[2].view(np.uint32), b[2].view(np.uint32)) and not np.any(np.isnan(b[2]))
+    for u, v in zip(a[3], b[3]):
+        assert state_equal(u, v) and u["device_token"] == v["device_token"]
+    ctx = qe.Context(0)
+    L = qe.Layer(ctx, T, 256, 256, 4, 0, 2, inputs.weights("HR", 0, 0, 256, 256).to(DEV))  # no staging buffers
+    with pytest.raises(qe.QEError) as e:
+        qe.run_together(ctx, [("F", L, 0, 0, torch.zeros((T, 256), dtype=torch.bfloat16).pin_memory(), None)], host=True)
+    assert e.value.code == "BAD_ARG"
