@@ -10,7 +10,6 @@ Modules
   bf16     bfloat16 bit helpers (decode, single-rounding encode from float64)
   scaling  amax history + delayed scale rule (scale = fp8_max / max(hist) / 2^margin)
   layer    the F / dI / dW state machine with tape pool, versions and arena mask
-  run      drives a list of layers through a schedule and records a trace
 
 Pins (tests/test_oracle_*.py): hand-computed FP8 bytes, exhaustive decode/encode
 round trip and midpoint ties, ml_dtypes agreement inside the finite range, the

@@ -39,4 +39,5 @@ def ulp(v: np.ndarray) -> np.ndarray:
     """Spacing of bfloat16 values at magnitude |v| (float64)."""
     v = np.abs(np.asarray(v, dtype=np.float64))
     _, e = np.frexp(v)
-    return np.ldexp(1.0, np.maximum(e.astype(np.int64) - 8, -133))
+    e = np.where(v == 0, -(1 << 20), e.astype(np.int64))  # frexp(0) reports exponent 0; zero sits among the subnormals
+    return np.ldexp(1.0, np.maximum(e - 8, -133))
