@@ -74,8 +74,30 @@ def decode(codes: np.ndarray, fmt: FP8Format) -> np.ndarray:
     return _FULL[fmt.name][codes]
 
 
+_BLOCK = 1 << 18  # elements handled at a time by encode()
+
+
 def encode(values: np.ndarray, fmt: FP8Format) -> np.ndarray:
-    """float32 values -> uint8 codes: round to nearest even, saturate to finite.
+    """float32 values -> uint8 codes, element by element (see _encode_block).
+
+    The map is elementwise, so the tensor is walked in blocks of 2^18 elements
+    only to keep the float64 / int64 temporaries of a block small; the result
+    does not depend on the block size (full-size test tensors have 10^8
+    elements, and whole-tensor temporaries of a gigabyte each made the cast
+    six times slower without changing a bit of it).
+    """
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    if v.size <= _BLOCK:
+        return _encode_block(v, fmt)
+    flat = v.reshape(-1)
+    out = np.empty(flat.size, dtype=np.uint8)
+    for lo in range(0, flat.size, _BLOCK):
+        out[lo : lo + _BLOCK] = _encode_block(flat[lo : lo + _BLOCK], fmt)
+    return out.reshape(v.shape)
+
+
+def _encode_block(values: np.ndarray, fmt: FP8Format) -> np.ndarray:
+    """Round to nearest even, saturate to finite.
 
     For a magnitude a: find neighbouring codes lo <= a <= hi among the positive
     finite values; pick lo if a is below their midpoint, hi if above, and the
@@ -111,6 +133,12 @@ def quantize(x_f32: np.ndarray, scale: np.float32, fmt: FP8Format) -> np.ndarray
     rounding once from a wider type.
     """
     x = np.asarray(x_f32, dtype=np.float32)
+    if x.size > _BLOCK:  # elementwise, so block by block (see encode); same bits as the whole tensor at once
+        flat = np.ascontiguousarray(x).reshape(-1)
+        out = np.empty(flat.size, dtype=np.uint8)
+        for lo in range(0, flat.size, _BLOCK):
+            out[lo : lo + _BLOCK] = quantize(flat[lo : lo + _BLOCK], scale, fmt)
+        return out.reshape(x.shape)
     with np.errstate(over="ignore", invalid="ignore"):
         prod = x * np.float32(scale)  # numpy keeps float32 * float32 in float32 (IEEE RN)
     assert prod.dtype == np.float32

@@ -30,8 +30,17 @@ def _gen(*parts) -> torch.Generator:
     return g
 
 
-def normal_bf16(shape, std: float, *seed_parts) -> torch.Tensor:
-    x = torch.randn(shape, generator=_gen(*seed_parts), dtype=torch.float32)
+def normal_bf16(shape, std: float, *seed_parts, device=None) -> torch.Tensor:
+    """device=None: drawn by the CPU generator.  With a CUDA device the same seed feeds that device's generator
+    instead (other numbers, equally reproducible): the full-size configurations draw gigabytes per step, which the
+    CPU generator would take minutes over; whoever needs the tensor on the host copies it back, so both sides of a
+    comparison still see identical bits."""
+    if device is None or torch.device(device).type == "cpu":
+        x = torch.randn(shape, generator=_gen(*seed_parts), dtype=torch.float32)
+    else:
+        g = torch.Generator(device=device)
+        g.manual_seed(seed_for(*seed_parts))
+        x = torch.randn(shape, generator=g, dtype=torch.float32, device=device)
     return (x * std).to(torch.bfloat16)
 
 
@@ -47,22 +56,27 @@ def spike_mask(shape, fraction: float, *seed_parts) -> torch.Tensor:
     return torch.rand(shape, generator=_gen(*seed_parts)) < fraction
 
 
-def activations(cfg: str, step: int, layer: int, linear: int, mb: int, T: int, K: int) -> torch.Tensor:
-    return normal_bf16((T, K), 1.0, cfg, step, layer, linear, mb, "X")
+def activations(cfg: str, step: int, layer: int, linear: int, mb: int, T: int, K: int, device=None) -> torch.Tensor:
+    return normal_bf16((T, K), 1.0, cfg, step, layer, linear, mb, "X", device=device)
 
 
-def upstream_grads(cfg: str, step: int, layer: int, linear: int, mb: int, T: int, N: int) -> torch.Tensor:
-    return normal_bf16((T, N), 1e-3, cfg, step, layer, linear, mb, "dY")
+def upstream_grads(cfg: str, step: int, layer: int, linear: int, mb: int, T: int, N: int, device=None) -> torch.Tensor:
+    return normal_bf16((T, N), 1e-3, cfg, step, layer, linear, mb, "dY", device=device)
 
 
-def weights(cfg: str, layer: int, linear: int, N: int, K: int) -> torch.Tensor:
-    return normal_bf16((N, K), 0.02, cfg, 0, layer, linear, "W")
+def weights(cfg: str, layer: int, linear: int, N: int, K: int, device=None) -> torch.Tensor:
+    return normal_bf16((N, K), 0.02, cfg, 0, layer, linear, "W", device=device)
 
 
 def optimizer_perturbation(w: torch.Tensor, cfg: str, step: int, layer: int, linear: int) -> torch.Tensor:
     """Stand-in for the optimizer: W <- bf16(W + delta), delta ~ N(0, (2e-5)^2), independent
-    of every GEMM output so state trajectories stay comparable bit for bit."""
-    d = torch.randn(w.shape, generator=_gen(cfg, step, layer, linear, "dW_opt"), dtype=torch.float32) * 2e-5
+    of every GEMM output so state trajectories stay comparable bit for bit.  Drawn on w's device."""
+    if w.device.type == "cpu":
+        d = torch.randn(w.shape, generator=_gen(cfg, step, layer, linear, "dW_opt"), dtype=torch.float32) * 2e-5
+    else:
+        g = torch.Generator(device=w.device)
+        g.manual_seed(seed_for(cfg, step, layer, linear, "dW_opt"))
+        d = torch.randn(w.shape, generator=g, dtype=torch.float32, device=w.device) * 2e-5
     return (w.float() + d).to(torch.bfloat16)
 
 

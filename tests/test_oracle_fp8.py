@@ -139,3 +139,22 @@ def test_bf16_round_matches_torch_on_float32_inputs():
     lib = torch.from_numpy(v).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(ours, lib)
     assert np.array_equal(bf16.decode(ours), torch.from_numpy(v).to(torch.bfloat16).float().numpy())
+
+
+@pytest.mark.parametrize("fmt", [fp8.E4M3, fp8.E5M2], ids=lambda f: f.name)
+def test_walking_a_large_tensor_in_blocks_changes_no_byte(fmt):
+    # encode() and quantize() walk tensors above 2^18 elements block by block; the map is elementwise, so the bytes
+    # must equal those of the one-pass rule applied with any other split (here: element by element ranges of a prime size)
+    n = (1 << 19) + 12345  # two full blocks and a ragged tail
+    rng = np.random.default_rng(7)
+    v = (rng.standard_normal(n) * np.exp(rng.uniform(-12, 12, n))).astype(np.float32)
+    v[::1001] = 0.0
+    v[5::5003] = np.inf
+    s = np.float32(3.7)
+    got = fp8.quantize(v.reshape(-1, 1), s, fmt)
+    assert got.shape == (n, 1) and got.dtype == np.uint8
+    with np.errstate(over="ignore"):
+        prod = (v * s).astype(np.float32)
+    want = np.concatenate([fp8._encode_block(prod[i:i + 99991], fmt) for i in range(0, n, 99991)])
+    assert np.array_equal(got.reshape(-1), want)
+    assert np.array_equal(fp8.encode(prod, fmt), want)
