@@ -1,6 +1,6 @@
 """Small single-kernel cases for profiling (ncu) and quick timing.
 
-    python -m paper_2609_23536_b200.profile_case gemm_f|gemm_di|gemm_dw|gemm_microbatch|gemm_microbatch_grouped|gemm_step|quantize|quantize_t|amax|accumulate [--reps N]
+    python profile_case.py gemm_f|gemm_di|gemm_dw|gemm_microbatch|gemm_microbatch_grouped|gemm_step|quantize|quantize_t|amax|accumulate [--reps N]
 
 Each case holds well under 2 GB on the device, uses operands larger than the 126 MB L2 where DRAM traffic is
 the question, does 2 warm-up launches and then `reps` launches, and prints the CUDA-event time per launch.
@@ -12,10 +12,15 @@ import json
 
 import torch
 
-from . import build
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+
+from paper_2609_23536_b200 import build  # noqa: E402
 
 build.build()
-from . import binding as qe  # noqa: E402
+from paper_2609_23536_b200 import binding as qe  # noqa: E402
 
 
 def main():
@@ -31,7 +36,7 @@ def main():
     work = None
     if a.case == "gemm_step":
         # the GEMM launches of one optimizer step as the default issue plan groups them (config 2 with --small)
-        from . import inputs, step_gemms
+        from paper_2609_23536_b200 import inputs, step_gemms
 
         launches, flops, nbytes = step_gemms.build(inputs.CONFIGS["C2" if a.small else "C3"], dev)
         fn = lambda: step_gemms.run(qe, launches, status)
