@@ -196,8 +196,7 @@ class Stage:
             t_issue = time.perf_counter()
             self.plan.run()
             self.issue_s += time.perf_counter() - t_issue
-            for L in self.layers:
-                L.optimizer_boundary(self.cfg["M"])
+            self.qe.optimizer_boundary_all(self.layers, self.cfg["M"])
             self.epoch += 1
             return
         tapes = {}
@@ -226,8 +225,7 @@ class Stage:
                 for key, t in zip(keys, self.qe.run_together(self.ctx, acts, self.grad, host=host_io)):
                     tapes[key] = t
             self.issue_s += time.perf_counter() - t_issue
-            for L in self.layers:
-                L.optimizer_boundary(self.cfg["M"])
+            self.qe.optimizer_boundary_all(self.layers, self.cfg["M"])
             if host_io:  # the step's result: the accumulated gradients, complete after the boundary
                 self.grad_host.copy_(self.grad, non_blocking=True)
                 self.d2h += self.grad.numel() * 4
@@ -339,8 +337,7 @@ class Stage:
             for i, L in enumerate(self.layers):
                 L.arena_finalize(self.arena, self.cfg["M"] * self.offsets[i], self.cfg["M"], self.grad, self.offsets[i])
         self.issue_s += time.perf_counter() - t_issue  # host time to enqueue the step (before the boundary's sync)
-        for L in self.layers:
-            L.optimizer_boundary(self.cfg["M"])
+        self.qe.optimizer_boundary_all(self.layers, self.cfg["M"])  # one drain and one status read for the whole stage
         if host_io:  # the step's result: the accumulated gradients, complete after the boundary
             self.grad_host.copy_(self.grad, non_blocking=True)
             self.d2h += self.grad.numel() * 4

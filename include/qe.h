@@ -119,6 +119,9 @@ int32_t qe_contract_dW_commit(qe_contract*, const qe_tape*, uint64_t dest_addr, 
 /* Optimizer commit (Algorithm 1, after the loop): no live tape (else PENDING), every microbatch in [0, expected) wrote exactly
  * once (else INCOMPLETE); then e_W += 1, mask cleared, next forward refreshes the cache. */
 int32_t qe_contract_boundary(qe_contract*, uint32_t microbatches_expected);
+/* The checks of qe_contract_boundary alone (nothing changes): lets a caller that commits several layers together
+ * make every layer's check before the first commit. */
+int32_t qe_contract_boundary_check(const qe_contract*, uint32_t microbatches_expected);
 /* Failure boundary (Sec. 4.5): purge this epoch's tapes (generations kept), mark the arena unusable. */
 int32_t qe_contract_abort(qe_contract*);
 /* Make the arena usable again after an abort; the epoch restarts with nothing written (PENDING if a tape lives). */
@@ -189,7 +192,9 @@ int32_t qe_ctx_create(const qe_ctx_config*, qe_ctx** out);
 int32_t qe_ctx_destroy(qe_ctx*);
 int32_t qe_layer_workspace_bytes(const qe_layer_config*, uint64_t* bytes_out);
 /* workspace_dev: 256-byte aligned device memory of at least qe_layer_workspace_bytes; owned by the caller, must
- * outlive the layer.  The call zero-initialises the state in it (histories 0, scales 1) on the execution stream. */
+ * outlive the layer.  The call zero-initialises the state in it (histories 0, scales 1) on the execution stream, so
+ * the memory must have no work pending on any other stream when the call is made (memory fresh from a stream-ordered
+ * allocator may still be written by kernels that used it before it was freed: synchronise that stream first). */
 int32_t qe_layer_create(qe_ctx*, const qe_layer_config*, void* workspace_dev, uint64_t workspace_bytes,
                         qe_layer** out);
 int32_t qe_layer_destroy(qe_layer*);
@@ -306,13 +311,21 @@ int32_t qe_arena_reduce(const void* views_dev, uint64_t view_elems, uint32_t M, 
  * launched one by one inside the same call.  layers[] (host array) distinct and of one context, 1 <= n <=
  * QE_MAX_MULTI_DW; tapes[] and offsets[] host arrays of n entries.  All n checks are made before anything runs: on
  * a contract error nothing ran and no layer's state changed.  A bounded wait that expires inside a shared launch
- * is recorded in the status word of the first layer of that launch. */
+ * is recorded in the status word of every layer that has a GEMM in that launch. */
 #define QE_MAX_MULTI_DW 16
 int32_t qe_backward_dW_multi(qe_layer* const* layers, const qe_tape* tapes, uint32_t n, float* grad_buf_dev,
                              uint64_t grad_buf_elems, const uint64_t* offsets, void* caller_stream);
 /* Optimizer boundary: waits for the execution stream, reads the device status word, then applies
  * qe_contract_boundary (bumping the weight version so that the next forward refreshes the cache). */
 int32_t qe_optimizer_boundary(qe_layer*, uint32_t microbatches_expected);
+/* The optimizer boundary of n layers of ONE context in one call (Algorithm 1's commit after the loop, for a whole
+ * stage): the context's streams are drained once, one small kernel ORs the layers' device status words together and
+ * one 4-byte copy brings the result to the host -- where n separate qe_optimizer_boundary calls pay n drains and n
+ * blocking copies.  Then every layer's contract check is made (no live tape, every microbatch wrote exactly once)
+ * and, only if all n pass, every layer's weight version is bumped.  On any error (QE_ERR_TIMEOUT from a status word,
+ * a contract error of some layer) no layer's state has changed.  layers[]: host array of 1 <= n <= 4096 distinct
+ * layers. */
+int32_t qe_optimizer_boundary_all(qe_layer* const* layers, uint32_t n, uint32_t microbatches_expected);
 /* The scale update as a standalone call: push *amax_dev (one FP32 on the device) into the class's history ring and
  * recompute scale = fp8_max / max(history) / 2^margin and its inverse (unchanged if the maximum is 0 or not
  * finite; +Inf clamps to FLT_MAX).  Same kernel F and dI use.  Does not advance the effect token. */
@@ -461,8 +474,12 @@ int32_t qe_gemm_fp8_group(const qe_gemm_desc* descs, uint32_t n, uint32_t* statu
  * must not allocate, or in a process whose device memory was handed out completely at start-up.  The caller still
  * passes every input and the output; this call and everything under it call no cudaMalloc/cudaFree and no allocating
  * library routine.  A, B, shapes, formats, alphas and status_dev are as in qe_gemm_fp8; dst_dev is FP32 [M,Nn],
- * 16-byte aligned.  M*Nn above 2^20 is rejected with QE_ERR_UNSUPPORTED.  The first call on each device looks up
- * the staging area's device address (with that device current); make that first call outside any stream capture.
+ * 16-byte aligned.  M*Nn above 2^20 is rejected with QE_ERR_UNSUPPORTED.  The staging area used is the CURRENT
+ * device's: the current device must be the one `stream` and every pointer belong to (the call does not check it).
+ * The first call on each device is a warm-up: it looks up the staging area's device address and sets kernel
+ * attributes, and with lazy module loading the driver places this library's code and the 4 MiB array in device
+ * memory at that point -- so make that first call where the driver may still do so (not under an allocator lock, not
+ * in a fully partitioned process) and outside any stream capture.  Later calls on that device touch no allocator.
  * All calls share the one staging area and it keeps the previous call's contents: every call overwrites the part
  * it uses before reading it, so nothing needs clearing, but two calls whose work overlaps on the GPU (different
  * streams without an ordering between them) race on it -- keep them on one stream or order them with events. */

@@ -168,6 +168,8 @@ _SIGNATURES = {
     "qe_step_run": (C.c_int32, [_P, C.POINTER(_P), C.c_uint32, C.POINTER(qe_step_action), C.c_uint32, C.c_uint32,
                                 C.POINTER(qe_step_io), _P, C.c_uint64, C.POINTER(C.c_uint64), _P, _P]),
     "qe_optimizer_boundary": (C.c_int32, [_P, C.c_uint32]),
+    "qe_optimizer_boundary_all": (C.c_int32, [C.POINTER(_P), C.c_uint32, C.c_uint32]),
+    "qe_contract_boundary_check": (C.c_int32, [_P, C.c_uint32]),
     "qe_scale_commit": (C.c_int32, [_P, C.c_uint32, _P, _P]),
     "qe_abort_step": (C.c_int32, [_P]),
     "qe_arena_rebuild": (C.c_int32, [_P]),
@@ -267,6 +269,9 @@ class Contract:
     def boundary(self, expected):
         _check(lib.qe_contract_boundary(self.h, expected))
 
+    def boundary_check(self, expected):
+        _check(lib.qe_contract_boundary_check(self.h, expected))
+
     def abort(self):
         _check(lib.qe_contract_abort(self.h))
 
@@ -350,6 +355,9 @@ class Layer:
         self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=weight.device)
         base = (self.workspace.data_ptr() + 255) // 256 * 256
         self.h = _P()
+        # torch's allocator is stream-ordered: the block may still be written by earlier work of the current stream,
+        # while the library initialises it on the context's execution stream
+        torch.cuda.current_stream(weight.device).synchronize()
         _check(lib.qe_layer_create(ctx.h, C.byref(self.cfg), base, nbytes.value, C.byref(self.h)))
 
     # the five calls of the path
@@ -560,6 +568,13 @@ def run_together(ctx, actions, grad_buf=None, stream=None, host=False):
     fn = lib.qe_run_together_host if host else lib.qe_run_together
     _check(fn(ctx.h, arr, n, _ptr(grad_buf), grad_buf.numel() if grad_buf is not None else 0, _stream(stream)))
     return new_tapes
+
+
+def optimizer_boundary_all(layers, expected):
+    """qe_optimizer_boundary_all: the boundary of every layer of a stage (one context) with one drain and one read."""
+    n = len(layers)
+    hs = (_P * n)(*[L.h for L in layers])
+    _check(lib.qe_optimizer_boundary_all(hs, n, expected))
 
 
 def forward_chain(layers, mb, gen, x, y, stream=None):

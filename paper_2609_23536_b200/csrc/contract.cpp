@@ -192,7 +192,7 @@ int32_t qe_contract_dW_commit(qe_contract* c, const qe_tape* t, uint64_t dest_ad
 }
 
 // Algorithm 1, after the action loop.
-int32_t qe_contract_boundary(qe_contract* c, uint32_t expected) {
+int32_t qe_contract_boundary_check(const qe_contract* c, uint32_t expected) {
   if (!c) return fail(QE_ERR_BAD_ARG, "contract is null");
   if (c->aborted) return fail(QE_ERR_ABORTED, "step aborted");
   if (expected < 1 || expected > QE_MAX_MICROBATCHES) return fail(QE_ERR_BAD_ARG, "microbatches_expected %u", expected);
@@ -200,6 +200,12 @@ int32_t qe_contract_boundary(qe_contract* c, uint32_t expected) {
   const uint64_t want = expected == 64 ? ~0ull : ((1ull << expected) - 1);
   if (c->write_mask != want)
     return fail(QE_ERR_INCOMPLETE, "gradient write mask %#llx, expected %#llx", (unsigned long long)c->write_mask, (unsigned long long)want);
+  return QE_OK;
+}
+
+int32_t qe_contract_boundary(qe_contract* c, uint32_t expected) {
+  const int32_t st = qe_contract_boundary_check(c, expected);
+  if (st != QE_OK) return st;
   c->e_W += 1;
   c->write_mask = 0;
   c->fwd_in_epoch = 0;

@@ -261,6 +261,7 @@ struct OneProblem {
   __device__ __forceinline__ const GemmParams& first() const { return p; }
   __device__ __forceinline__ uint32_t count() const { return 1; }
   __device__ __forceinline__ const CommitParams& commit(uint32_t) const { return p.commit; }
+  __device__ __forceinline__ uint32_t* status_of(uint32_t) const { return p.status; }
 };
 struct ProblemGroup {
   const GemmGroupParams& g;
@@ -274,6 +275,7 @@ struct ProblemGroup {
   __device__ __forceinline__ const GemmParams& first() const { return g.prob[0]; }
   __device__ __forceinline__ uint32_t count() const { return g.n; }
   __device__ __forceinline__ const CommitParams& commit(uint32_t i) const { return g.prob[i].commit; }
+  __device__ __forceinline__ uint32_t* status_of(uint32_t i) const { return g.prob[i].status; }
 };
 
 // ------------------------------------------------------------------------------------------------ kernel
@@ -600,6 +602,13 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
 
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) {
+    // a wait gave up in this CTA: the error bits went to the first problem's status word; every other problem of a
+    // shared launch gets them too, since any of their tiles may be missing
+    const uint32_t bits = atomicOr(status, 0u);
+    for (uint32_t i = 1; i < ps.count(); ++i)
+      if (ps.status_of(i) && ps.status_of(i) != status) atomicOr(ps.status_of(i), bits);
+  }
   if (TWO) cluster_sync_all();  // no arrival may still be on its way to a CTA that has left
   if (warp == 1) {
     tc_fence_after();

@@ -23,7 +23,8 @@ struct DevState {
   float slot_sinv_G[64];
   uint32_t ticket;             // "last CTA" counter of the kernel whose tail performs the commit; self-resetting
   uint32_t wmax[4];            // bit pattern of max(history ring) per class, kept by the commit (derived state)
-  uint32_t pad[39];            // header is 768 bytes; history rings [4][H] follow
+  uint32_t status_all;         // scratch of the multi-layer boundary: OR of several layers' status words
+  uint32_t pad[38];            // header is 768 bytes; history rings [4][H] follow
 };
 static_assert(sizeof(DevState) == 768, "DevState layout");
 
@@ -118,6 +119,14 @@ struct GemmGroupParams {
   GemmParams prob[8];
 };
 
+// ORs the status words of up to 64 layers into *out (first chunk: out = OR; later chunks: out |= OR).
+struct StatusGatherParams {
+  const uint32_t* src[64];
+  uint32_t* out;
+  uint32_t n;
+  uint32_t accumulate;
+};
+
 // One launch, self-contained.
 struct Launch {
   const void* func = nullptr;
@@ -136,6 +145,7 @@ struct Launch {
 Launch make_quantize(const QuantParams& p);
 Launch make_quantize_multi(const QuantParams* casts, uint32_t n);  // 2..8 independent casts in one launch
 Launch make_commit(const CommitParams& p);
+Launch make_status_gather(const StatusGatherParams& p);
 Launch make_amax_pass1(const AmaxParams& p);
 Launch make_amax_pass2(const AmaxParams& p);
 Launch make_accumulate(const AccumParams& p);

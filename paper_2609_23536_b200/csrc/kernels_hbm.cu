@@ -173,6 +173,26 @@ __global__ void __launch_bounds__(256) commit_kernel(const __grid_constant__ Com
   commit_classes(p, threadIdx.x, red, [] { __syncthreads(); });
 }
 
+__global__ void __launch_bounds__(64) status_gather_kernel(const __grid_constant__ StatusGatherParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
+  uint32_t v = threadIdx.x < p.n ? __ldcg(p.src[threadIdx.x]) : 0u;
+  v = __reduce_or_sync(0xffffffffu, v);
+  __shared__ uint32_t w[2];
+  if ((threadIdx.x & 31) == 0) w[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x == 0) *p.out = (p.accumulate ? *p.out : 0u) | w[0] | w[1];
+}
+
+Launch make_status_gather(const StatusGatherParams& p) {
+  Launch l;
+  l.func = (const void*)status_gather_kernel;
+  l.grid = dim3(1, 1, 1);
+  l.block = dim3(64, 1, 1);
+  l.set(p);
+  return l;
+}
+
 Launch make_commit(const CommitParams& p) {
   Launch l;
   l.func = (const void*)commit_kernel;

@@ -343,6 +343,39 @@ int32_t qe_optimizer_boundary(qe_layer* L, uint32_t expected) {
   return qe_contract_boundary(L->contract, expected);
 }
 
+int32_t qe_optimizer_boundary_all(qe_layer* const* layers, uint32_t n, uint32_t expected) {
+  if (!layers || n < 1 || n > 4096) return fail(QE_ERR_BAD_ARG, "layers null or n = %u out of range", n);
+  for (uint32_t i = 0; i < n; ++i) {
+    if (!layers[i]) return fail(QE_ERR_BAD_ARG, "layers[%u] is null", i);
+    if (layers[i]->ctx != layers[0]->ctx) return fail(QE_ERR_BAD_ARG, "layers[%u] belongs to another context", i);
+  }
+  qe_ctx* ctx = layers[0]->ctx;
+  if (ctx->dw_stream) {  // deferred weight gradients run there: the gather below must come after them
+    QE_CUDA(cudaEventRecord(ctx->ev_dw_in, ctx->dw_stream));
+    QE_CUDA(cudaStreamWaitEvent(ctx->exec_stream, ctx->ev_dw_in, 0));
+  }
+  uint32_t* out = &layers[0]->st->status_all;
+  for (uint32_t lo = 0; lo < n; lo += 64) {
+    qe::StatusGatherParams gp{};
+    gp.n = std::min(64u, n - lo);
+    for (uint32_t i = 0; i < gp.n; ++i) gp.src[i] = &layers[lo + i]->st->status;
+    gp.out = out;
+    gp.accumulate = lo ? 1u : 0u;
+    QE_CUDA(launch_pdl(qe::make_status_gather(gp), ctx->exec_stream));
+    ctx->stats.kernels_launched += 1;
+  }
+  uint32_t status = 0;
+  QE_CUDA(cudaMemcpyAsync(&status, out, sizeof(status), cudaMemcpyDeviceToHost, ctx->exec_stream));
+  QE_CUDA(cudaStreamSynchronize(ctx->exec_stream));  // the one drain: everything issued before the boundary is done
+  if (status) return fail(QE_ERR_TIMEOUT, "device status word %#x: a bounded wait expired in a GEMM", status);
+  for (uint32_t i = 0; i < n; ++i) {
+    const int32_t st = qe_contract_boundary_check(layers[i]->contract, expected);
+    if (st != QE_OK) return st;
+  }
+  for (uint32_t i = 0; i < n; ++i) qe_contract_boundary(layers[i]->contract, expected);
+  return QE_OK;
+}
+
 int32_t qe_scale_commit(qe_layer* L, uint32_t cls, const float* amax_dev, void* caller_stream) {
   if (!L) return fail(QE_ERR_BAD_ARG, "layer is null");
   if (cls > QE_CLASS_Y) return fail(QE_ERR_BAD_ARG, "tensor_class %u", cls);

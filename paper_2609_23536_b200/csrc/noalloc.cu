@@ -3,6 +3,7 @@
 // plugin running inside another framework's memory-pool lock, a callback on a thread that must not touch the
 // allocator, an embedded runtime whose memory is fully partitioned at start-up -- so here the scratch is a fixed
 // array that is part of the library image on every GPU that loads it.
+#include <atomic>
 #include <cstdint>
 
 #include "error.h"
@@ -20,7 +21,9 @@ constexpr uint64_t kStagingElems = 1ull << 20;  // FP32 elements: 4 MiB, e.g. on
 static __device__ __align__(256) float g_staging[kStagingElems];
 
 constexpr int kMaxDevices = 16;
-float* g_staging_addr[kMaxDevices] = {nullptr};
+// One cached address per device.  Atomic, so that host threads making their first calls at the same time do not race
+// on it (each would look up and store the same value).
+std::atomic<float*> g_staging_addr[kMaxDevices];
 
 // First use on a device (that device current): resolve the device address of g_staging.
 int32_t staging_address(float** out) {
@@ -28,13 +31,13 @@ int32_t staging_address(float** out) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return fail(QE_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
   if (dev < 0 || dev >= kMaxDevices) return fail(QE_ERR_UNSUPPORTED, "device ordinal %d beyond %d", dev, kMaxDevices);
-  if (!g_staging_addr[dev]) {
-    float* p = nullptr;
+  float* p = g_staging_addr[dev].load(std::memory_order_acquire);
+  if (!p) {
     e = cudaGetSymbolAddress((void**)&p, g_staging);
     if (e != cudaSuccess || !p) return fail(QE_ERR_CUDA, "cudaGetSymbolAddress(staging): %s", cudaGetErrorString(e));
-    g_staging_addr[dev] = p;
+    g_staging_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_staging_addr[dev];
+  *out = p;
   return QE_OK;
 }
 

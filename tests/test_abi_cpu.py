@@ -119,6 +119,30 @@ def test_fault_table(qe):
     _expect(qe, "PENDING", c5.checkpoint_check)
 
 
+def test_boundary_check_is_the_boundary_without_its_effects(qe):
+    # the check half of the optimizer commit (Algorithm 1: a check precedes its action and changes nothing): the same
+    # verdicts as the boundary itself, state untouched, so that several layers can be checked before any is committed
+    c = qe.Contract(2)
+    t = c.forward_commit(0)
+    for code in ("PENDING",):
+        before = c.get()
+        _expect(qe, code, c.boundary_check, 1)
+        assert c.get() == before
+    c.dI_commit(t)
+    c.dW_check(t, BUF, ELEMS, 0, SLICE)
+    c.dW_commit(t, BUF, 0, SLICE)
+    before = c.get()
+    _expect(qe, "INCOMPLETE", c.boundary_check, 2)
+    _expect(qe, "BAD_ARG", c.boundary_check, 0)
+    c.boundary_check(1)
+    c.boundary_check(1)  # as often as one likes
+    assert c.get() == before and before["e_W"] == 0
+    c.boundary(1)
+    assert c.get()["e_W"] == 1 and c.get()["write_mask"] == 0
+    c.abort()
+    _expect(qe, "ABORTED", c.boundary_check, 1)
+
+
 def test_destination_rules(qe):
     reg = qe.Registry()
     a, b = qe.Contract(1, unit=0, registry=reg), qe.Contract(1, unit=1, registry=reg)

@@ -9,7 +9,8 @@ import numpy as np
 import pytest
 import torch
 
-from harness import assert_gemm_close, state_equal_except_Y, transposed_or_none
+from harness import (assert_gemm_close, assert_grad_close, dW_abs_products, state_equal, state_equal_except_Y,
+                     transposed_or_none)
 from oracle import bf16
 from oracle.layer import ArenaRegistry, OracleLinear
 from paper_2609_23536_b200 import inputs
@@ -54,6 +55,7 @@ class Stage:
             self.O = [OracleLinear(self.T, K, N, cfg["H"], cfg["margin"], self.P, unit=u, registry=reg)
                       for u, (l, j, K, N) in enumerate(self.units)]
             self.ograd = np.zeros(per_layer * L, np.float32)  # lazily committed: only sampled rows are touched
+            self.oabs = {}  # unit -> sum over the heavy microbatches of sum_t |g x| alpha on the sampled gradient rows
         self.epoch = 0
 
     def x(self, step, u, mb):
@@ -118,6 +120,11 @@ class Stage:
                     else:
                         G.backward_dW(gt[(u, m)], self.grad, self.offsets[u])
                     if self.O:
+                        slot = self.O[u].slots[ot[(u, m)].ref.slot]
+                        if r and slot.Xq is not None and slot.Gq is not None:
+                            if m == 0:
+                                self.oabs.pop(u, None)
+                            self.oabs[u] = self.oabs.get(u, 0.0) + dW_abs_products(slot, r[1])
                         self.O[u].backward_dW(ot[(u, m)], self.ograd, self.offsets[u], rows=r[1] if r else [0])
                 if self.O and check_state:
                     g = G.state()
@@ -127,12 +134,12 @@ class Stage:
         return outs
 
     def grads_match(self, u, rows_n, what):
-        """main_grad rows of unit u against the oracle's accumulation (all microbatches heavy for u)."""
+        """main_grad rows of unit u against the oracle's accumulation (all microbatches heavy for u): Frobenius norm
+        and every element within the FP32 accumulation bound."""
         l, j, K, N = self.units[u]
-        got = self.grad[self.offsets[u]: self.offsets[u] + N * K].view(N, K)[rows_n].cpu().numpy().astype(np.float64)
-        want = self.ograd[self.offsets[u]: self.offsets[u] + N * K].reshape(N, K)[rows_n].astype(np.float64)
-        rel = np.linalg.norm(got - want) / np.linalg.norm(want)
-        assert rel < 1e-5, (what, u, rel)
+        got = self.grad[self.offsets[u]: self.offsets[u] + N * K].view(N, K)[rows_n].cpu().numpy()
+        want = self.ograd[self.offsets[u]: self.offsets[u] + N * K].reshape(N, K)[rows_n]
+        assert_grad_close(got, want, (what, u), abs_products=self.oabs[u], rel_tol=1e-5)
 
     def boundary(self):
         for G in self.G:
@@ -152,12 +159,11 @@ def _rows(T, N, nr, seed):
 def test_config2_llama_block_state_every_action_bytes_and_gemm_rows_sampled(qe):
     # 4 linears, T = 2048, H = 1024, 8 microbatches in zero-bubble order, one flat gradient buffer.
     S = Stage(qe, "C2", qe.GRAPH)
-    rows = lambda u: _rows(S.T, S.units[u][3], 14, u)
-    # every microbatch heavy for the two smaller linears (so their gradient slices can be checked), microbatches
-    # 0 and 5 for the two large ones
-    heavy = lambda u, m: u in (1, 3) or m in (0, 5)
-    S.run_step(0, heavy, rows)
-    for u in (1, 3):
+    # 16 sampled token rows of Y / dX and gradient rows of every linear (fewer rows of the two large slices, whose
+    # casts dominate the oracle's time); every microbatch heavy, so that all four gradient slices can be checked
+    rows = lambda u: _rows(S.T, S.units[u][3], 14 if u in (1, 3) else 6, u)
+    S.run_step(0, lambda u, m: True, rows)
+    for u in range(4):
         S.grads_match(u, rows(u)[1], "C2")
     S.boundary()
     st = S.ctx.stats()
@@ -234,34 +240,250 @@ def test_config5_direct_placement_against_staged_and_oracle(qe):
     S.boundary()
 
 
-def test_config3_llama3_8b_layers_sampled(qe):
-    # 4 layers x 4 linears, T = 4096, 16 microbatches, graph replay over several steps.  Inputs are drawn once per
-    # (layer, linear, microbatch parity) and reused across steps (static buffers replayed); the oracle gets
-    # the same tensors.  State after every action of the sampled units; bytes and GEMM rows on sampled units.
+# ------------------------------------------------------------------------------------------ config 3 at its stated size
+class _OracleFollower:
+    """One sampled linear of config 3 followed by the oracle on a thread of its own (the linears are independent, and
+    numpy releases the interpreter lock inside its loops, so several followers run side by side while the GPU goes on).
+    The driver puts one item per action of that linear, in order; every item carries what the GPU produced (state after
+    the action, and for heavy actions FP8 bytes and output rows), which is compared here."""
+
+    def __init__(self, name, T, K, N, H, P, unit, rows_T, rows_N):
+        import queue
+        import threading
+
+        self.name, self.rows_T, self.rows_N = name, rows_T, rows_N
+        self.O = OracleLinear(T, K, N, H, 0, P, unit=unit)
+        self.buf = np.zeros(N * K, np.float32)  # untouched pages stay uncommitted: only sampled rows are written
+        self.absp = 0.0
+        self.tapes = {}
+        self.q = queue.Queue(maxsize=4)
+        self.error = None
+        self.checked = {"state": 0, "bytes": 0, "gemm_rows": 0, "grad_rows": 0}
+        self.t = threading.Thread(target=self._loop, daemon=True)
+        self.t.start()
+
+    def put(self, *item):
+        self.q.put(item)
+
+    def finish(self):
+        self.q.put(None)
+        self.t.join()
+        if self.error:
+            raise AssertionError(f"oracle follower {self.name}: {self.error}")
+
+    def _loop(self):
+        import traceback
+
+        while True:
+            item = self.q.get()
+            if item is None:
+                return
+            if self.error:
+                continue  # keep draining so that the driver never blocks
+            try:
+                self._do(*item)
+            except Exception:  # noqa: BLE001
+                self.error = traceback.format_exc()
+
+    def _state(self, g, what):
+        assert g["device_status"] == 0 and g["device_token"] == g["token"], what
+        assert state_equal_except_Y(g, self.O.state()), what
+        self.checked["state"] += 1
+
+    def _do(self, kind, step, m, *a):
+        O, what = self.O, (self.name, kind, step, m)
+        if kind == "W":
+            O.set_weight(a[0])
+        elif kind == "F":
+            x_bits, tape, g, heavy = a
+            self.tapes[m], oy = O.forward(m, O.e_W, x_bits, rows=self.rows_T, light=heavy is None)
+            assert tape == (tuple(self.tapes[m].key), tuple(self.tapes[m].ref)), what
+            self._state(g, what)
+            if heavy is not None:
+                slot = O.slots[self.tapes[m].ref.slot]
+                assert np.array_equal(heavy["Xq"], slot.Xq), ("Xq",) + what
+                assert np.array_equal(heavy["Wq"], O.Wq), ("Wq",) + what
+                assert g["slot_sinv_X"][self.tapes[m].ref.slot].view(np.uint32) == np.float32(slot.sinv_X).view(np.uint32)
+                assert_gemm_close(heavy["rows"], oy, ("Y",) + what)
+                self.checked["bytes"] += 2
+                self.checked["gemm_rows"] += len(self.rows_T)
+        elif kind == "dI":
+            dy_bits, g, heavy = a
+            odx = O.backward_dI(self.tapes[m], dy_bits, rows=self.rows_T, light=heavy is None)
+            self._state(g, what)
+            if heavy is not None:
+                slot = O.slots[self.tapes[m].ref.slot]
+                assert np.array_equal(heavy["Gq"], slot.Gq), ("Gq",) + what
+                assert g["slot_sinv_G"][self.tapes[m].ref.slot].view(np.uint32) == np.float32(slot.sinv_G).view(np.uint32)
+                assert_gemm_close(heavy["rows"], odx, ("dX",) + what)
+                self.checked["bytes"] += 1
+                self.checked["gemm_rows"] += len(self.rows_T)
+        elif kind == "dW":
+            g, grad_rows = a
+            slot = O.slots[self.tapes[m].ref.slot]
+            if slot.Xq is not None and slot.Gq is not None:
+                if m == 0:
+                    self.absp = 0.0
+                self.absp = self.absp + dW_abs_products(slot, self.rows_N)
+            O.backward_dW(self.tapes.pop(m), self.buf, 0, rows=self.rows_N)
+            self._state(g, what)
+            if grad_rows is not None:  # every microbatch up to this one was heavy: the slice's rows so far
+                want = self.buf.reshape(O.N, O.K)[self.rows_N]
+                assert_grad_close(grad_rows, want, ("main_grad",) + what, abs_products=self.absp, rel_tol=1e-5)
+                self.checked["grad_rows"] += len(self.rows_N)
+        elif kind == "boundary":
+            O.optimizer_boundary(a[0])
+            self._state(a[1], what)
+
+
+def _one_row_per_tile(n, mul):
+    """One row in every 128-row tile (so every 256-row tile pair, every wave and both CTAs of a pair are visited)."""
+    return [128 * i + (mul * i + 7) % 128 for i in range(n // 128)]
+
+
+def test_config3_four_layers_sixteen_microbatches_ten_steps_replayed(qe):
+    """Config 3 as stated: Llama-3-8B shapes (T = 4096; qkv 4096->6144, o 4096->4096, gate/up 4096->28672, down
+    14336->4096), 4 layers, 16 microbatches in zero-bubble order, every F / dI / dW captured once per slot and replayed
+    over static buffers for 10 steps with optimizer boundaries between them (Sec. 4.3-4.4), all weight gradients into
+    one 3.49 GB flat buffer at the layers' affine offsets.  Inputs are distinct per (step, layer, linear, microbatch),
+    drawn by the device generator from the usual seeds; the sampled linears' tensors are copied back for the oracle.
+
+    Checked: (1) step 0 in eager mode against the replayed step 0, bit for bit, every output of every unit at full
+    width; (2) the oracle's state after EVERY action of seven sampled linears (all four shapes, all four layers) --
+    over all ten steps for six of them; (3) FP8 bytes and GEMM rows (one row per 128-row tile) on heavy units of every
+    shape, including a whole step of the attention output projection of every layer, whose complete gradient slice is
+    then compared element by element; first-write and first-accumulate gradient rows of the two wide shapes."""
     name = "C3"
     cfg = inputs.CONFIGS[name]
-    T, M = cfg["T"], cfg["M"]
-    S = Stage(qe, name, qe.GRAPH, n_layers=1)  # one of the four (identical) layers keeps the host-side generation short
-    cache = {}
+    T, M, steps, nl = cfg["T"], cfg["M"], cfg["steps"], len(cfg["linears"])
+    schedule = sched(M, *cfg["sched"])
+    P = peak_live(schedule)
+    units = [(l, j, K, N) for l in range(cfg["layers"]) for j, (_, K, N) in enumerate(cfg["linears"])]
+    offs, per_layer = inputs.grad_offsets(cfg["linears"])
+    offsets = [l * per_layer + offs[j] for l, j, _, _ in units]
+    assert per_layer == 218103808 and offsets[4:8] == [218103808 + o for o in (0, 25165824, 41943040, 159383552)]
+    n = len(units)
 
-    def x(step, u, mb, _f=S.x):
-        k = ("x", u, mb % 2)
-        if k not in cache:
-            cache[k] = _f(0, u, mb % 2)
-        return cache[k]
+    def make(mode):
+        ctx = qe.Context(mode)
+        W = [inputs.weights(name, l, j, N, K, device=DEV) for l, j, K, N in units]
+        G = [qe.Layer(ctx, T, K, N, cfg["H"], cfg["margin"], P, W[u], unit=u) for u, (l, j, K, N) in enumerate(units)]
+        grad = torch.full((per_layer * cfg["layers"],), 3.0, device=DEV)  # stale contents: microbatch 0 must overwrite
+        return ctx, W, G, grad
 
-    def dy(step, u, mb, _f=S.dy):
-        k = ("dy", u, mb % 2)
-        if k not in cache:
-            cache[k] = _f(0, u, mb % 2)
-        return cache[k]
+    # ---- (1a) step 0, eager: keep every output on the device
+    ctx, W, G, grad = make(qe.EAGER)
+    eager = {}
+    tapes = {}
+    for a, m in schedule:
+        for u in (range(n) if a == "F" else range(n - 1, -1, -1)):
+            l, j, K, N = units[u]
+            if a == "F":
+                y = torch.empty((T, N), dtype=torch.bfloat16, device=DEV)
+                tapes[(u, m)] = G[u].forward(m, 0, inputs.activations(name, 0, l, j, m, T, K, device=DEV), y)
+                eager[(u, m, "Y")] = y
+            elif a == "dI":
+                dx = torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+                G[u].backward_dI(tapes[(u, m)], inputs.upstream_grads(name, 0, l, j, m, T, N, device=DEV), dx)
+                eager[(u, m, "dX")] = dx
+            else:
+                G[u].backward_dW(tapes[(u, m)], grad, offsets[u])
+    torch.cuda.synchronize()
+    for L in G:
+        L.optimizer_boundary(M)
+    eager_grad, eager_state = grad, [L.state() for L in G]
+    del G, ctx
+    torch.cuda.empty_cache()
 
-    S.x, S.dy = x, dy
-    rows = lambda u: _rows(T, S.units[u][3], 2, u)
-    sampled = {(0, 0, 0), (0, 2, 1), (1, 3, 15), (2, 1, 8), (2, 3, 0)}  # (step, unit, microbatch)
-    for step in range(3):
-        S.run_step(step, heavy=lambda u, m: (step, u, m) in sampled, rows=rows)
-        S.boundary()
-    for G in S.G:
-        st = G.state()
-        assert st["e_W"] == 3 and st["token"] == 3 * 2 * M and st["device_status"] == 0
+    # ---- the ten replayed steps, with the oracle following the sampled linears
+    ctx, W, G, grad = make(qe.GRAPH)
+    # static buffers: one set per (linear, slot); a forward takes the set of the slot it is about to occupy
+    buf = [[{"x": torch.empty((T, K), dtype=torch.bfloat16, device=DEV), "y": torch.empty((T, N), dtype=torch.bfloat16, device=DEV),
+             "dy": torch.empty((T, N), dtype=torch.bfloat16, device=DEV), "dx": torch.empty((T, K), dtype=torch.bfloat16, device=DEV)}
+            for _ in range(P)] for _, _, K, N in units]
+    rows_T = _one_row_per_tile(T, 37)
+    U = lambda l, j: l * nl + j
+    # sampled linear -> (steps followed, heavy (step, mb) units, (step, mb) after whose dW the gradient rows are compared)
+    all_mb = lambda st: {(st, m) for m in range(M)}
+    plan = {
+        U(0, 0): (steps, {(0, 0), (9, 15)}, {(0, 0)}),                      # qkv, layer 0
+        U(0, 1): (steps, all_mb(0), {(0, M - 1)}),                          # o, every layer: one whole heavy step each
+        U(1, 1): (steps, all_mb(3), {(3, M - 1)}),
+        U(2, 1): (steps, all_mb(6), {(6, M - 1)}),
+        U(3, 1): (steps, all_mb(9), {(9, M - 1)}),
+        U(2, 3): (steps, {(0, 0), (0, 1), (9, 15)}, {(0, 0), (0, 1)}),      # down, layer 2
+        U(3, 2): (1, {(0, 0), (0, 1)}, {(0, 0), (0, 1)}),                   # gate/up, layer 3: first step only
+    }
+    followers = {}
+    for u, (nsteps, heavy, gchk) in plan.items():
+        l, j, K, N = units[u]
+        followers[u] = _OracleFollower(f"layer {l} {cfg['linears'][j][0]}", T, K, N, cfg["H"], P, u, rows_T, _one_row_per_tile(N, 53))
+    bits = lambda t: inputs.bits(t.cpu())
+    compared = 0
+    for step in range(steps):
+        for u, (l, j, K, N) in enumerate(units):
+            if step > 0:
+                W[u] = inputs.optimizer_perturbation(W[u], name, step, l, j)
+                G[u].weight.copy_(W[u])
+            if u in plan and step < plan[u][0]:
+                followers[u].put("W", step, -1, bits(W[u]))
+        tapes = {}
+        for a, m in schedule:
+            for u in (range(n) if a == "F" else range(n - 1, -1, -1)):
+                l, j, K, N = units[u]
+                L = G[u]
+                f = followers[u] if (u in plan and step < plan[u][0]) else None
+                heavy = f is not None and (step, m) in plan[u][1]
+                if a == "F":
+                    b = buf[u][L.next_slot()]
+                    b["x"].copy_(inputs.activations(name, step, l, j, m, T, K, device=DEV))
+                    tapes[(u, m)] = t = L.forward(m, step, b["x"], b["y"])
+                    assert buf[u][t.ref.slot] is b
+                    if step == 0:
+                        assert torch.equal(b["y"].view(torch.int16), eager.pop((u, m, "Y")).view(torch.int16)), ("replay != eager: Y", u, m)
+                        compared += 1
+                    if f:
+                        h = {"Xq": L.read_fp8(0, t.ref.slot), "Wq": L.read_fp8(4), "rows": bits(b["y"][rows_T])} if heavy else None
+                        f.put("F", step, m, bits(b["x"]), t.astuple(), L.state(), h)
+                elif a == "dI":
+                    t = tapes[(u, m)]
+                    b = buf[u][t.ref.slot]
+                    b["dy"].copy_(inputs.upstream_grads(name, step, l, j, m, T, N, device=DEV))
+                    L.backward_dI(t, b["dy"], b["dx"])
+                    if step == 0:
+                        assert torch.equal(b["dx"].view(torch.int16), eager.pop((u, m, "dX")).view(torch.int16)), ("replay != eager: dX", u, m)
+                        compared += 1
+                    if f:
+                        h = {"Gq": L.read_fp8(2, t.ref.slot), "rows": bits(b["dx"][rows_T])} if heavy else None
+                        f.put("dI", step, m, bits(b["dy"]), L.state(), h)
+                else:
+                    L.backward_dW(tapes[(u, m)], grad, offsets[u])
+                    if f:
+                        g_rows = None
+                        if (step, m) in plan[u][2]:
+                            g_rows = grad[offsets[u]: offsets[u] + N * K].view(N, K)[f.rows_N].cpu().numpy()
+                        f.put("dW", step, m, L.state(), g_rows)
+            assert not any(f.error for f in followers.values()), [f.error for f in followers.values() if f.error][0]
+        torch.cuda.synchronize()
+        for u, L in enumerate(G):
+            L.optimizer_boundary(M)
+            if u in plan and step < plan[u][0]:
+                followers[u].put("boundary", step, -1, M, L.state())
+        if step == 0:
+            assert compared == 2 * n * M and not eager
+            assert torch.equal(grad.view(torch.int32), eager_grad.view(torch.int32)), "replay != eager: main_grad"
+            for x, y in zip(eager_state, [L.state() for L in G]):
+                assert state_equal({**x, "slots": []}, {**y, "slots": []}) and x["device_token"] == y["device_token"]
+            del eager_grad
+            torch.cuda.empty_cache()
+    for f in followers.values():
+        f.finish()
+    st = ctx.stats()
+    assert st["graphs_built"] == n * (3 * P + 1) and st["eager_launches"] == 0  # G_r = 3 P L (+ one refresh graph per linear)
+    assert st["graph_replays"] == steps * n * (3 * M + 1)
+    for L in G:
+        s_ = L.state()
+        assert s_["e_W"] == steps and s_["token"] == steps * 2 * M and s_["device_status"] == 0
+    total = {k: sum(f.checked[k] for f in followers.values()) for k in ("state", "bytes", "gemm_rows", "grad_rows")}
+    assert total["state"] == sum((3 * M + 1) * plan[u][0] for u in plan)
+    assert total["bytes"] >= 3 * (4 * M + 7) and total["grad_rows"] > 0

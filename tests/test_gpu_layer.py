@@ -91,11 +91,11 @@ def test_config1_every_action_against_oracle(qe, mode):
         assert np.all(np.abs(gy["window"].astype(np.float64) - oy) <= 4 * bf16.ulp(oy))
 
     gouts = run_gpu_steps(qe, L, s, steps, M, gbuf, 64, get, lambda e: W[e], on_action=check)
-    assert set(gouts) == set(oouts)
-    for k in oouts:
+    assert set(gouts) == {k for k in oouts if k[1] != "mg_abs"}
+    for k in gouts:
         if k[1] == "mg":
             assert np.array_equal(gouts[k][:64], np.full(64, 7.0, np.float32))  # nothing outside the slice
-            rel = assert_grad_close(gouts[k][64:], oouts[k][64:], k)
+            rel = assert_grad_close(gouts[k][64:], oouts[k][64:], k, abs_products=oouts[(k[0], "mg_abs")])
             assert rel < 1e-5, rel
         else:
             assert_gemm_close(gouts[k], oouts[k], k)
@@ -175,9 +175,9 @@ def test_shapes_that_take_the_single_cta_gemm_against_oracle(qe, mode):
     ctx, L = _mk_layer(qe, mode, T, K, N, H, 0, P)
     gbuf = torch.full((N * K,), -1.0, device=DEV)
     got = run_gpu_steps(qe, L, s, 2, M, gbuf, 0, get, lambda e: W[e])
-    for k in want:
+    for k in got:
         if k[1] == "mg":
-            assert assert_grad_close(got[k], want[k], k) < 1e-5
+            assert assert_grad_close(got[k], want[k], k, abs_products=want[(k[0], "mg_abs")]) < 1e-5
         else:
             assert_gemm_close(got[k], want[k], k)
     assert state_equal_except_Y(L.state(), O.state())
@@ -203,6 +203,120 @@ def test_scale_commit_standalone_matches_hand_worked_rollover(qe):
     for a, w in zip([1, 8, 2, 2, 2, 2], [28672, 3584, 3584, 3584, 3584, 14336]):
         L2.scale_commit(qe.CLASS_G, torch.tensor([a], dtype=torch.float32, device=DEV))
         assert L2.state()["classes"]["G"]["scale"] == np.float32(w)
+
+
+def _bits(x):
+    return int(np.float32(x).view(np.uint32))
+
+
+@pytest.mark.parametrize("cls,fmt,margin", [("X", fp8.E4M3, 0), ("G", fp8.E5M2, 1), ("W", fp8.E4M3, -2)])
+def test_scale_commit_edge_cases_against_the_oracle(qe, cls, fmt, margin):
+    # What the scale rule does at the edges of its domain, compared with the oracle's ScaleState bit for bit after
+    # every commit: an amax so small that fp8_max / amax overflows (scale clamps to the largest finite binary32 and its
+    # inverse is a subnormal), +Inf and NaN entries (stored in the window, scale and inverse left alone until they
+    # have rolled out), and a window that becomes all zero (scale left alone again).
+    from oracle.scaling import ScaleState
+
+    H = 4
+    ctx, L = _mk_layer(qe, 0, 256, 256, 256, H, margin, 1)
+    O = ScaleState(fmt, H, margin)
+    seq = [2.0**-133, 0.0, float("inf"), 1.0, float("nan"), 2.0, 0.5, 0.25, 0.125, 0.0, 0.0, 0.0, 0.0, 0.0, 3.0, 2.0**-126, 3.3895314e38]
+    kinds = set()
+    for i, a in enumerate(seq):
+        before = _bits(O.scale)
+        L.scale_commit(getattr(qe, "CLASS_" + cls), torch.tensor([a], dtype=torch.float32, device=DEV))
+        O.commit(np.float32(a))
+        g = L.state()["classes"][cls]
+        assert _bits(g["scale"]) == _bits(O.scale), (i, a, g["scale"], O.scale)
+        assert _bits(g["scale_inv"]) == _bits(O.scale_inv), (i, a)
+        assert np.array_equal(g["window"].view(np.uint32), O.window().view(np.uint32)), (i, a)
+        assert g["count"] == O.count == i + 1
+        if _bits(O.scale) == before:
+            kinds.add("unchanged")
+        if O.scale == np.finfo(np.float32).max:
+            kinds.add("clamped")
+            assert 0 < float(O.scale_inv) < 2.0**-126  # the inverse of the clamp is a subnormal, kept as such
+    assert {"unchanged", "clamped"} <= kinds
+    st = L.state()
+    assert st["device_status"] == 0 and st["device_token"] == 0
+    for other in "XWGY":
+        if other != cls:
+            assert st["classes"][other]["count"] == 0 and st["classes"][other]["scale"] == 1.0
+
+
+@pytest.mark.parametrize("fmt_id,fmt", [(0, fp8.E4M3), (1, fp8.E5M2)])
+def test_cast_of_a_tensor_holding_one_nan_and_the_commit_that_follows(qe, fmt_id, fmt):
+    # One NaN among ordinary values: every other byte as the oracle casts it, the NaN's byte the format's NaN code
+    # whatever its sign, the tensor's amax not finite -- and committing that amax leaves the scale where it was.
+    from oracle.scaling import ScaleState, amax_bf16
+
+    rows, cols = 256, 384
+    x = inputs.normal_bf16((rows, cols), 1.0, "nan-cast", fmt_id)
+    x[17, 101] = float("nan")
+    scale = np.float32(37.25)
+    q = torch.empty((rows, cols), dtype=torch.uint8, device=DEV)
+    amax = torch.zeros(1, dtype=torch.float32, device=DEV)
+    qe.qe_quantize(x.to(DEV), torch.tensor([scale], device=DEV), fmt_id, q, None, amax)
+    got = q.cpu().numpy()
+    want = fp8.quantize(bf16.decode(inputs.bits(x)), scale, fmt)
+    assert want[17, 101] & 0x7F == fmt.nan_code
+    assert np.array_equal(got & 0x7F, want & 0x7F) and np.array_equal(np.delete(got.reshape(-1), 17 * cols + 101), np.delete(want.reshape(-1), 17 * cols + 101))
+    a = amax.cpu().numpy()[0]
+    assert not np.isfinite(a) and not np.isfinite(amax_bf16(bf16.decode(inputs.bits(x))))
+    cls = "X" if fmt_id == 0 else "G"
+    ctx, L = _mk_layer(qe, 0, 256, 256, 256, 4, 0, 1)
+    O = ScaleState(fmt, 4, 0)
+    for v in (2.5, a, 0.75):  # an ordinary commit, the non-finite one, an ordinary one while the NaN is still in the window
+        L.scale_commit(getattr(qe, "CLASS_" + cls), torch.tensor([v], dtype=torch.float32, device=DEV))
+        O.commit(np.float32(v))
+        g = L.state()["classes"][cls]
+        assert _bits(g["scale"]) == _bits(O.scale) == _bits(np.float32(fmt.max_finite) / np.float32(2.5))
+        assert _bits(g["scale_inv"]) == _bits(O.scale_inv)
+        assert np.array_equal(g["window"].view(np.uint32) & 0x7FFFFFFF, O.window().view(np.uint32) & 0x7FFFFFFF)
+
+
+def test_boundary_of_many_layers_in_one_call(qe):
+    # 70 small layers of one context (more than one 64-entry gather launch): a step each, then ONE boundary call.
+    # While one layer still lacks a microbatch the call fails and bumps NO layer; afterwards all move together.
+    T = K = N = 256
+    M, nl = 2, 70
+    ctx = qe.Context(qe.EAGER)
+    Ls = [qe.Layer(ctx, T, K, N, 4, 0, 2, inputs.weights("B", 0, u % 3, N, K).to(DEV), unit=u) for u in range(nl)]
+    x = inputs.activations("B", 0, 0, 0, 0, T, K).to(DEV)
+    dy = inputs.upstream_grads("B", 0, 0, 0, 0, T, N).to(DEV)
+    y, dx = torch.empty((T, N), dtype=torch.bfloat16, device=DEV), torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+    grad = torch.zeros(nl * N * K, device=DEV)
+    held = None
+    for u, L in enumerate(Ls):
+        for m in range(M):
+            t = L.forward(m, 0, x, y)
+            L.backward_dI(t, dy, dx)
+            if u == 67 and m == 1:
+                held = t  # layer 67 keeps its last weight gradient back
+            else:
+                L.backward_dW(t, grad, u * N * K)
+    with pytest.raises(qe.QEError) as e:
+        qe.optimizer_boundary_all(Ls, M)
+    assert e.value.code == "PENDING"
+    assert all(L.state()["e_W"] == 0 for L in Ls)
+    Ls[67].backward_dW(held, grad, 67 * N * K)
+    with pytest.raises(qe.QEError) as e:
+        qe.optimizer_boundary_all(Ls, M + 1)
+    assert e.value.code == "INCOMPLETE" and all(L.state()["e_W"] == 0 for L in Ls)
+    k0 = ctx.stats()["kernels_launched"]
+    qe.optimizer_boundary_all(Ls, M)
+    assert ctx.stats()["kernels_launched"] - k0 == 2  # two gather launches for 70 status words
+    for L in Ls:
+        s_ = L.state()
+        assert s_["e_W"] == 1 and s_["write_mask"] == 0 and s_["fwd_in_epoch"] == 0 and s_["device_status"] == 0
+    # same gradients as layer-by-layer boundaries would have left (the boundary touches no data)
+    g = grad.view(nl, N * K)
+    assert torch.equal(g[0], g[3]) and torch.equal(g[1], g[67]) and not torch.equal(g[0], g[1])
+    other = qe.Context(qe.EAGER)
+    alien = qe.Layer(other, T, K, N, 4, 0, 2, torch.zeros((N, K), dtype=torch.bfloat16, device=DEV))
+    with pytest.raises(qe.QEError) as e:
+        qe.optimizer_boundary_all([Ls[0], alien], M)
+    assert e.value.code == "BAD_ARG"
 
 
 def test_contract_violations_through_the_layer_leave_state_untouched(qe):

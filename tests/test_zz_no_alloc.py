@@ -48,7 +48,13 @@ def test_noalloc_matches_existing_entry_points_on_two_calls_in_a_row(qe):
         if key not in dst_new:
             init = torch.randn((M, Nn), generator=torch.Generator().manual_seed(7)).to(DEV)
             dst_new[key], dst_old[key] = init.clone(), init.clone()
+        if i > 0:  # past the first (warm-up) call on this device: a call must leave the device's free memory as it was
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
         qe.qe_gemm_fp8_staged_noalloc(A, afmt, B, bfmt, sa, sb, dst_new[key], acc, status)
+        if i > 0:
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before, i
         temp = torch.full((M, Nn), float("nan"), device=DEV)
         qe.qe_gemm_fp8(A, afmt, B, bfmt, sa, sb, temp, 1, None, status)
         qe.qe_accumulate(dst_old[key], temp, acc)
@@ -57,6 +63,31 @@ def test_noalloc_matches_existing_entry_points_on_two_calls_in_a_row(qe):
         assert torch.equal(dst_new[key], dst_old[key]), i
         assert torch.isfinite(dst_new[key]).all()
     assert status.item() == 0
+
+
+def test_noalloc_against_the_oracle(qe):
+    # the largest case the staging area holds, against the plain definition: exact products of the decoded FP8 values
+    # times the two factors, rounded once to FP32, then one FP32 addition to what the destination held
+    from oracle import fp8
+
+    M, Nn, Kc = 1024, 1024, 512
+    A, B = _operands(300, M, Nn, Kc)
+    sa, sb = np.float32(2.0**-9), np.float32(3.0 * 2.0**-11)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    init = torch.randn((M, Nn), generator=torch.Generator().manual_seed(9))
+    dst = init.clone().to(DEV)
+    qe.qe_gemm_fp8_staged_noalloc(A, 1, B, 0, torch.tensor([sa], device=DEV), torch.tensor([sb], device=DEV), dst, True, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    a, b = fp8.decode(A.cpu().numpy(), fp8.E5M2), fp8.decode(B.cpu().numpy(), fp8.E4M3)
+    D = ((a @ b.T) * np.float64(sa) * np.float64(sb)).astype(np.float32)
+    want = (init.numpy() + D).astype(np.float32)
+    got = dst.cpu().numpy()
+    # FP32 accumulation of Kc products in the GEMM, one multiply by the factors, one addition: each rounds at 2^-24 of
+    # a magnitude bounded by the sum of the absolute products (plus the old value for the addition)
+    bound = 8 * 2.0**-24 * ((np.abs(a) @ np.abs(b).T) * float(sa) * float(sb) + np.abs(init.numpy()))
+    assert (np.abs(got.astype(np.float64) - want) <= bound).all()
+    assert np.linalg.norm(got.astype(np.float64) - want) / np.linalg.norm(want) < 1e-6
 
 
 def test_noalloc_rejects_sizes_beyond_its_staging_area(qe):
