@@ -124,25 +124,35 @@ def dW_abs_products(slot, rows):
     return (G.T @ X) * float(slot.sinv_G) * float(slot.sinv_X)
 
 
-GRAD_ULPS = 8.0  # per-element FP32 bound, in units of 2^-24 * sum |products| (see assert_grad_close)
+GRAD_ULPS = 8.0  # per-element FP32 bound for ordinary data, in units of 2^-24 * sum |products| (see assert_grad_close)
 
 
-def assert_grad_close(got, want, what="", abs_products=None, rel_tol=1e-3):
+def assert_grad_close(got, want, what="", abs_products=None, rel_tol=1e-3, contraction=None):
     """FP32 gradient against the oracle's (exact products, one rounding per microbatch): relative Frobenius error, and
-    -- given abs_products = sum over the microbatches written so far of dW_abs_products -- every element within
-    GRAD_ULPS * 2^-24 * abs_products.  FP32 accumulation of T products in any order, one multiply by alpha and one
-    addition per microbatch each round with relative error 2^-24 of a magnitude that never exceeds the sum of the
-    absolute products, and on these inputs the errors add up like a random walk, far below the worst case of one
-    2^-24 per operation; 8 leaves that margin while a single wrong, missing or doubled product (each at least
-    sum|p| / T ~ 2^-11 sum|p|) still falls outside it."""
+    -- given abs_products = sum over the microbatches written so far of dW_abs_products, and the contraction length T --
+    an elementwise bound in units of u = 2^-24 * abs_products:
+
+      * no element beyond (2 * T / 32 + 8) u.  The tensor cores add the products of 32 contraction indices to the FP32
+        accumulator per instruction; each such step, the multiply by alpha and the addition to the buffer lose at most
+        one unit in the last place (2^-23, chopping allowed for) of a magnitude that never exceeds the sum of the
+        absolute products.  This is what FP32 accumulation guarantees whatever the data.
+      * at most 1 % of the elements beyond GRAD_ULPS u.  On data without a dominating product the partial sums stay far
+        below sum|p| and the errors add up like a random walk; only where one huge product sits in the accumulator for
+        the rest of the contraction (the 1000x outliers of the rollover stress) does an element approach the first bound.
+
+    A wrong, missing or doubled product of typical size is sum|p| / T = 2^-11..2^-12 of sum|p|, far outside both."""
     g, w = got.astype(np.float64), want.astype(np.float64)
     denom = np.linalg.norm(w)
     rel = np.linalg.norm(g - w) / denom if denom > 0 else np.abs(g).max()
     assert rel <= rel_tol, (what, rel)
     if abs_products is not None:
-        bound = GRAD_ULPS * 2.0**-24 * abs_products + 2.0**-149
-        bad = np.abs(g - w) > bound
-        assert not bad.any(), (what, int(bad.sum()), float((np.abs(g - w) / bound).max()))
+        assert contraction is not None
+        u = 2.0**-24 * abs_products + 2.0**-149
+        err = np.abs(g - w) / u
+        hard = 2.0 * contraction / 32 + 8
+        assert (err <= hard).all(), (what, "beyond the FP32 accumulation bound", int((err > hard).sum()), float(err.max()), hard)
+        frac = float((err > GRAD_ULPS).mean())
+        assert frac <= 0.01, (what, "share of elements beyond GRAD_ULPS", frac, float(err.max()))
     return rel
 
 

@@ -221,7 +221,7 @@ def test_chain_layer_by_layer_against_a_teacher_forced_oracle(qe, mode):
         # the gradients: the oracle's tapes hold the same FP8 bytes and snapshots as the GPU's, so this is one GEMM's error
         for j, (K, N) in enumerate(CHAIN):
             assert_grad_close(chain["mg"][step][offs[j]: offs[j] + N * K], buf[offs[j]: offs[j] + N * K], ("mg", step, j),
-                              abs_products=absp[j].reshape(-1), rel_tol=1e-5)
+                              abs_products=absp[j].reshape(-1), rel_tol=1e-5, contraction=T)
         for j, L in enumerate(orc):
             assert state_equal_except_Y(chain["state"][step][j], L.state()), ("state after the boundary", step, j)
 

@@ -139,7 +139,7 @@ class Stage:
         l, j, K, N = self.units[u]
         got = self.grad[self.offsets[u]: self.offsets[u] + N * K].view(N, K)[rows_n].cpu().numpy()
         want = self.ograd[self.offsets[u]: self.offsets[u] + N * K].reshape(N, K)[rows_n]
-        assert_grad_close(got, want, (what, u), abs_products=self.oabs[u], rel_tol=1e-5)
+        assert_grad_close(got, want, (what, u), abs_products=self.oabs[u], rel_tol=1e-5, contraction=self.T)
 
     def boundary(self):
         for G in self.G:
@@ -329,7 +329,7 @@ class _OracleFollower:
             self._state(g, what)
             if grad_rows is not None:  # every microbatch up to this one was heavy: the slice's rows so far
                 want = self.buf.reshape(O.N, O.K)[self.rows_N]
-                assert_grad_close(grad_rows, want, ("main_grad",) + what, abs_products=self.absp, rel_tol=1e-5)
+                assert_grad_close(grad_rows, want, ("main_grad",) + what, abs_products=self.absp, rel_tol=1e-5, contraction=O.T)
                 self.checked["grad_rows"] += len(self.rows_N)
         elif kind == "boundary":
             O.optimizer_boundary(a[0])

@@ -95,7 +95,7 @@ def test_config1_every_action_against_oracle(qe, mode):
     for k in gouts:
         if k[1] == "mg":
             assert np.array_equal(gouts[k][:64], np.full(64, 7.0, np.float32))  # nothing outside the slice
-            rel = assert_grad_close(gouts[k][64:], oouts[k][64:], k, abs_products=oouts[(k[0], "mg_abs")])
+            rel = assert_grad_close(gouts[k][64:], oouts[k][64:], k, abs_products=oouts[(k[0], "mg_abs")], contraction=T)
             assert rel < 1e-5, rel
         else:
             assert_gemm_close(gouts[k], oouts[k], k)
@@ -177,7 +177,7 @@ def test_shapes_that_take_the_single_cta_gemm_against_oracle(qe, mode):
     got = run_gpu_steps(qe, L, s, 2, M, gbuf, 0, get, lambda e: W[e])
     for k in got:
         if k[1] == "mg":
-            assert assert_grad_close(got[k], want[k], k, abs_products=want[(k[0], "mg_abs")]) < 1e-5
+            assert assert_grad_close(got[k], want[k], k, abs_products=want[(k[0], "mg_abs")], contraction=T) < 1e-5
         else:
             assert_gemm_close(got[k], want[k], k)
     assert state_equal_except_Y(L.state(), O.state())
@@ -309,9 +309,9 @@ def test_boundary_of_many_layers_in_one_call(qe):
     for L in Ls:
         s_ = L.state()
         assert s_["e_W"] == 1 and s_["write_mask"] == 0 and s_["fwd_in_epoch"] == 0 and s_["device_status"] == 0
-    # same gradients as layer-by-layer boundaries would have left (the boundary touches no data)
+    # the boundary touches no data: every layer saw the same X and dY, so every slice holds the same gradient
     g = grad.view(nl, N * K)
-    assert torch.equal(g[0], g[3]) and torch.equal(g[1], g[67]) and not torch.equal(g[0], g[1])
+    assert torch.equal(g[0], g[67]) and torch.equal(g[1], g[69]) and torch.count_nonzero(g[0]).item() > 0
     other = qe.Context(qe.EAGER)
     alien = qe.Layer(other, T, K, N, 4, 0, 2, torch.zeros((N, K), dtype=torch.bfloat16, device=DEV))
     with pytest.raises(qe.QEError) as e:
