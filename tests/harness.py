@@ -97,9 +97,16 @@ def run_gpu_steps(qe, layer, schedule, steps, M, grad_buf, off, get_inputs, weig
     return res
 
 
+FLOOR_ONLY = {"elements": 0, "floor_only": 0}  # running count over a test session (see assert_gemm_close)
+
+
 def assert_gemm_close(got_bits, want_bits, what=""):
-    """bf16 outputs: relative Frobenius <= 1e-3 and <= 4 bf16 ulp elementwise, the ulp taken at
-    max(|oracle|, 2^-6 rms) (FP32 accumulation error scales with the sum of |products|)."""
+    """bf16 outputs: relative Frobenius <= 1e-3 and <= 4 bf16 ulp elementwise.  The ulp is taken at the oracle's
+    magnitude, except that it is never taken below 2^-6 of the tensor's rms: an output that is small because large
+    products cancelled carries the FP32 accumulation error of those products (which scales with the sum of their
+    magnitudes, not with the result), so 4 ulp of its own tiny magnitude is not a bound the arithmetic can meet.
+    Elements that pass only thanks to that floor are counted; they must stay under 0.5 % of the tensor (for Gaussian
+    outputs 1.2 % of the elements lie below the floor at all, and few of those need it)."""
     from oracle import bf16
 
     g = bf16.decode(got_bits).astype(np.float64)
@@ -108,8 +115,13 @@ def assert_gemm_close(got_bits, want_bits, what=""):
     rel = np.linalg.norm(g - w) / denom if denom > 0 else np.abs(g).max()
     assert rel <= 1e-3, (what, rel)
     floor = 2.0**-6 * np.sqrt(np.mean(w**2))
-    ok = np.abs(g - w) <= 4 * bf16.ulp(np.maximum(np.abs(w), floor))
-    assert ok.all(), (what, int((~ok).sum()), np.abs(g - w).max())
+    err = np.abs(g - w)
+    ok = err <= 4 * bf16.ulp(np.maximum(np.abs(w), floor))
+    assert ok.all(), (what, int((~ok).sum()), err.max())
+    floor_only = int((err > 4 * bf16.ulp(np.abs(w))).sum())
+    FLOOR_ONLY["elements"] += g.size
+    FLOOR_ONLY["floor_only"] += floor_only
+    assert floor_only <= max(2, 0.005 * g.size), (what, "elements within 4 ulp only at the floored magnitude", floor_only, g.size)
     return rel
 
 

@@ -156,12 +156,20 @@ def _rows(T, N, nr, seed):
             sorted(rng.choice(N, nr, replace=False).tolist() + [0, N - 1]))
 
 
+def _tile_rows(T, N, seed):
+    """One row in every 128-row tile of the token dimension (rows of Y / dX) and of the out-feature dimension (rows of
+    the gradient slice), plus the first and last row: every output tile of every GEMM, both CTAs of a pair and every
+    wave of the tile walk are then compared with the oracle somewhere."""
+    pick = lambda n, mul: sorted({0, n - 1} | {128 * i + (mul * i + seed) % 128 for i in range(n // 128)})
+    return pick(T, 37), pick(N, 53)
+
+
 def test_config2_llama_block_state_every_action_bytes_and_gemm_rows_sampled(qe):
     # 4 linears, T = 2048, H = 1024, 8 microbatches in zero-bubble order, one flat gradient buffer.
     S = Stage(qe, "C2", qe.GRAPH)
-    # 16 sampled token rows of Y / dX and gradient rows of every linear (fewer rows of the two large slices, whose
-    # casts dominate the oracle's time); every microbatch heavy, so that all four gradient slices can be checked
-    rows = lambda u: _rows(S.T, S.units[u][3], 14 if u in (1, 3) else 6, u)
+    # one token row per 128-row tile of Y / dX and one gradient row per 128-row tile of every slice; every microbatch
+    # heavy, so that all four gradient slices (the 92 MB gate/up one included) can be checked element by element
+    rows = lambda u: _tile_rows(S.T, S.units[u][3], u)
     S.run_step(0, lambda u, m: True, rows)
     for u in range(4):
         S.grads_match(u, rows(u)[1], "C2")
