@@ -422,8 +422,13 @@ def block_summary(blocks, steps, flop_per_step, world):
 # `python profile_case.py gemm_step` (config-2 shapes with --small); each entry names the capture's summary and the
 # commit of the kernel it was taken with, so that a stale figure shows
 QE_TRAFFIC = {
-    # config: (bytes per launch, launches per step, summary under profiles/, kernel source commit)
-    "C2": (287.6e6, 19, "gemm_fp8_pair_dram_traffic_config2_microbatch.md", "c7e58e5"),
+    # config: (bytes per launch, launches per step, summary under profiles/, commit of the kernel source captured)
+    "C2": (287.3e6, 19, "gemm_fp8_pair_dram_traffic_config2_microbatch.md", "3398557"),
+    # config 3 holds 59 GB of GEMM operands and outputs per step, too much to capture: the five launches of ONE
+    # layer-microbatch (12 GEMMs, 3770.3 MB read + written, 1.9 GB on the device) were captured and scaled by the 64
+    # layer-microbatches of a step over its 135 launches; every operand and output of a step is distinct data that is
+    # streamed once, so the traffic grows in proportion to the layer-microbatches processed
+    "C3": (3770.3e6 * 64 / 135, 135, "gemm_fp8_pair_dram_traffic_config3_layer_microbatch.md", "3398557"),
 }
 
 
