@@ -110,6 +110,7 @@ class Stage:
         import torch
 
         self.qe, self.cfg, self.dev = qe, cfg, device
+        self.boundary_per_layer = False
         self.group_dw = group_dw and not staged and not arena
         self.chain = chain
         self.pair_f_di = pair_f_di and not chain and not host_io
@@ -184,6 +185,14 @@ class Stage:
         self.h2d = self.d2h = 0
         self.issue_s = 0.0
 
+    def boundary(self):
+        """The optimizer boundary of the whole stage: one drain and one gathered status read (default), or layer by layer."""
+        if self.boundary_per_layer:
+            for L in self.layers:
+                L.optimizer_boundary(self.cfg["M"])
+        else:
+            self.qe.optimizer_boundary_all(self.layers, self.cfg["M"])
+
     def make_plan(self):
         """The whole step as one qe_step_run call (native host loop; one graph for the step in graph mode)."""
         n = len(self.layers)
@@ -196,7 +205,7 @@ class Stage:
             t_issue = time.perf_counter()
             self.plan.run()
             self.issue_s += time.perf_counter() - t_issue
-            self.qe.optimizer_boundary_all(self.layers, self.cfg["M"])
+            self.boundary()
             self.epoch += 1
             return
         tapes = {}
@@ -225,7 +234,7 @@ class Stage:
                 for key, t in zip(keys, self.qe.run_together(self.ctx, acts, self.grad, host=host_io)):
                     tapes[key] = t
             self.issue_s += time.perf_counter() - t_issue
-            self.qe.optimizer_boundary_all(self.layers, self.cfg["M"])
+            self.boundary()
             if host_io:  # the step's result: the accumulated gradients, complete after the boundary
                 self.grad_host.copy_(self.grad, non_blocking=True)
                 self.d2h += self.grad.numel() * 4
@@ -337,7 +346,7 @@ class Stage:
             for i, L in enumerate(self.layers):
                 L.arena_finalize(self.arena, self.cfg["M"] * self.offsets[i], self.cfg["M"], self.grad, self.offsets[i])
         self.issue_s += time.perf_counter() - t_issue  # host time to enqueue the step (before the boundary's sync)
-        self.qe.optimizer_boundary_all(self.layers, self.cfg["M"])  # one drain and one status read for the whole stage
+        self.boundary()
         if host_io:  # the step's result: the accumulated gradients, complete after the boundary
             self.grad_host.copy_(self.grad, non_blocking=True)
             self.d2h += self.grad.numel() * 4
@@ -484,11 +493,13 @@ def gemm_roofline(qe, cfg_name, cfg, peaks, device):
     torch.cuda.synchronize()
     reps = 3
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        step_gemms.run(qe, launches, status)
-    e1.record()
-    torch.cuda.synchronize()
+    with ClockSampler(device.index or 0) as gclk:  # which regime the launches were timed in (burst or power-capped)
+        e0.record()
+        for _ in range(reps):
+            step_gemms.run(qe, launches, status)
+        e1.record()
+        torch.cuda.synchronize()
+    g_clocks = gclk.summary()
     g_ms = e0.elapsed_time(e1) / reps
     g_launches = len(launches)
     del launches
@@ -519,7 +530,12 @@ def gemm_roofline(qe, cfg_name, cfg, peaks, device):
     tr = QE_TRAFFIC.get(cfg_name)
     if tr is not None and tr[1] != g_launches:
         tr = None  # the issue plan changed since the capture
-    peak = 2.0 * peaks["bf16_burst"]  # FP8 dense = 2 x the bf16 peak (nominal ratio), kernels timed alone -> burst figure
+    # FP8 dense = 2 x the bf16 peak (nominal ratio).  Which measured bf16 figure: the burst one for launches timed in a
+    # short loop; the sustained one when the loop is long enough for the power cap to engage and the sampled clocks
+    # say it did (config 3: 0.5 s at ~1.2 GHz) -- the regime the sustained figure was itself measured in
+    sustained = g_ms * reps >= 250.0 and "sw_power_cap" in g_clocks.get("reasons", [])
+    peak = 2.0 * (peaks["bf16_sustained"] if sustained else peaks["bf16_burst"])
+    burst_peak = 2.0 * peaks["bf16_burst"]
     # the weight-gradient launches are bound by the tensor pipe AND by the FP32 read-modify-write of the gradient slice:
     # both fractions, one problem per launch over rotating operand sets
     dw_fl, dw_ms = per["dW"]
@@ -531,13 +547,19 @@ def gemm_roofline(qe, cfg_name, cfg, peaks, device):
         "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": tr[0] if tr else None,
         "traffic_source": ("ncu capture summarised in profiles/%s, kernel as of commit %s" % (tr[2], tr[3])) if tr else None,
         "algorithmic_bytes_per_launch": round(g_bytes / g_launches),
-        "flop_per_launch": round(g_flops / g_launches), "launches_timed": g_launches, "peak_source": peaks["source"] + " bf16 burst x2",
+        "flop_per_launch": round(g_flops / g_launches), "launches_timed": g_launches,
+        "peak_source": peaks["source"] + (" bf16 sustained x2 (launches timed in a %.2f s loop under sw_power_cap)" % (g_ms * reps * 1e-3) if sustained else " bf16 burst x2"),
+        "frac_of_bf16_burst_x2": round(achieved / burst_peak, 4),
         "frac_of_nominal_4500": round(achieved / 4500.0, 4),
+        # the same launches against the figure for a kernel timed inside a long step, with the clock they ran at: the
+        # loop above lasts 0.4 s at config 3 (the power cap engages within it), 6 ms at config 2 (it does not)
+        "frac_of_bf16_sustained_x2": round(achieved / (2.0 * peaks["bf16_sustained"]), 4),
+        "clocks_while_timed": g_clocks,
         "one_problem_per_launch_tflops": round(single, 1),
         "per_action_tflops": {k: round(v[0] / (v[1] * 1e-3) / 1e12, 1) for k, v in per.items()},
-        "dw": {"tflops": round(dw_tf, 1), "frac_tensor": round(dw_tf / peak, 4), "frac_tensor_of_nominal_4500": round(dw_tf / 4500.0, 4),
+        "dw": {"tflops": round(dw_tf, 1), "frac_tensor": round(dw_tf / burst_peak, 4), "frac_tensor_of_nominal_4500": round(dw_tf / 4500.0, 4),
                "GB/s": round(dw_gbs, 1), "frac_hbm": round(dw_gbs / peaks["hbm_gbs"], 4),
-               "what": "weight-gradient GEMMs of one microbatch, one problem per launch: 2TNK flop and T(N+K) + 8NK bytes each"},
+               "what": "weight-gradient GEMMs of one microbatch, one problem per launch in a short loop (tensor fraction of bf16 burst x2): 2TNK flop and T(N+K) + 8NK bytes each"},
         "gemm_ms_per_step": round(g_ms, 4),
         "vendor_library_fp8_forward_tflops_same_shapes": lib,
     }
@@ -692,6 +714,8 @@ def main():
     ap.add_argument("--arena", action="store_true",
                     help="per-microbatch arena variant: dW writes one bf16 view per linear and microbatch, summed into the FP32 buffer before the boundary")
     ap.add_argument("--staged", action="store_true", help="copied-gradient comparison path: dW into a temporary, then a copy-add kernel")
+    ap.add_argument("--boundary-per-layer", action="store_true",
+                    help="one qe_optimizer_boundary call per layer (a drain and a blocking status read each) instead of qe_optimizer_boundary_all")
     ap.add_argument("--own-stream", action="store_true", help="let the context create its own execution stream (event handoff on every action)")
     args = ap.parse_args()
     cfg_name, cfg = args.config, inputs.CONFIGS[args.config]
@@ -729,6 +753,7 @@ def main():
         stage = Stage(qe, name, c, args.mode, device, same_stream=not own_stream,
                       overlap_dw=args.overlap_dw and not use_step, staged=args.staged, group_dw=args.group_dw, arena=args.arena,
                       chain=args.chain, pair_f_di=args.pair_f_di, together=args.together, plan_window=window)
+        stage.boundary_per_layer = args.boundary_per_layer
         if use_step:
             stage.make_plan()
         with ClockSampler(local) as clk:
