@@ -60,6 +60,47 @@ __device__ __forceinline__ void commit_classes(const CommitParams& p, int tid, u
   if (tid == 0 && p.bump_token) st->token += 1ull;
 }
 
+// The same commit done by ONE warp: eight lanes per tensor class (the rare ring scan strides by eight).  A grouped GEMM
+// launch ends with up to eight commits, one per problem; its last CTA gives each of them to an epilogue warp of its
+// own instead of running them one after the other (each is a chain of dependent global accesses, ~1.5 us: at launches
+// of 20 us that was half the launch).  Same values as commit_classes; the token is bumped atomically because two
+// problems of one launch may belong to the same layer (its forward and its input gradient of different microbatches).
+__device__ __forceinline__ void commit_classes_warp(const CommitParams& p, int lane) {
+  DevState* st = p.st;
+  const int c = lane >> 3, g = lane & 7;
+  const bool active = (p.class_mask >> c) & 1u;
+  uint32_t m = 0, newest = 0, cnt = 0, pos = 0;
+  uint32_t* h = reinterpret_cast<uint32_t*>(p.hist + (size_t)c * p.H);
+  if (active) {
+    cnt = __ldcg(&st->count[c]);
+    newest = p.amax_override ? (__float_as_uint(__ldcg(p.amax_override)) & 0x7fffffffu) : __ldcg(&st->pending_amax[c]);
+    const uint32_t wmax = __ldcg(&st->wmax[c]);
+    pos = cnt % p.H;
+    const uint32_t evicted = __ldcg(h + pos);
+    if (newest >= wmax) m = newest;
+    else if (evicted < wmax) m = wmax;
+    else
+      for (uint32_t i = g; i < p.H; i += 8) m = max(m, i == pos ? newest : __ldcg(h + i));
+  }
+  m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
+  m = max(m, __shfl_xor_sync(0xffffffffu, m, 4));
+  if (active && g == 0) {
+    h[pos] = newest;
+    st->count[c] = cnt + 1;
+    st->pending_amax[c] = 0;
+    st->wmax[c] = m;
+    if (m != 0 && m < 0x7f800000u) {
+      const float fp8_max = c == 2 ? 57344.0f : 448.0f;
+      float s = __fmul_rn(__fdiv_rn(fp8_max, __uint_as_float(m)), p.pow2_neg_margin);
+      if (isinf(s)) s = FLT_MAX;
+      st->scale[c] = s;
+      st->scale_inv[c] = __fdiv_rn(1.0f, s);
+    }
+  }
+  if (lane == 0 && p.bump_token) atomicAdd(&st->token, 1ull);
+}
+
 // Returns true in every thread of exactly one block of the grid: the last one to get here.  Stores and atomics the
 // grid made before this call are visible to that block afterwards.
 template <class Sync>

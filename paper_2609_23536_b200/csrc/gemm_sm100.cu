@@ -591,10 +591,12 @@ __device__ __forceinline__ void gemm_body(const PS& ps) {
     for (uint32_t i = 0; i < ps.count(); ++i)
       if (!ticket && ps.commit(i).st) ticket = &ps.commit(i).st->ticket;
     if (ticket && last_block(ticket, gridDim.x, etid, last_flag, epi_bar_sync)) {
-      for (uint32_t i = 0; i < ps.count(); ++i) {
-        if (!ps.commit(i).st) continue;
-        commit_classes(ps.commit(i), etid, red, epi_bar_sync);
-        epi_bar_sync();  // the reduction words are reused by the next problem's commit
+      if (ps.count() == 1) {
+        if (ps.commit(0).st) commit_classes(ps.commit(0), etid, red, epi_bar_sync);
+      } else {
+        // one epilogue warp per problem, side by side
+        for (uint32_t i = (uint32_t)warp - 2u; i < ps.count(); i += EPI_WARPS)
+          if (ps.commit(i).st) commit_classes_warp(ps.commit(i), lane);
       }
     }
     if (lane == 0) tma_store_wait_all();  // this warp's bulk stores have reached global memory
