@@ -59,3 +59,26 @@ def test_step_flops_and_gradient_offsets_of_the_configurations():
     assert bench.step_flops(inputs.CONFIGS["C3"]) == pytest.approx(343e12, rel=2e-3)
     offs, total = inputs.grad_offsets(inputs.CONFIGS["C2"]["linears"])
     assert (offs, total) == ([0, 12582912, 16777216, 39845888], 51380224)
+
+
+def test_block_summary_and_oracle_sample_choice():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2609_23536_b200 import inputs
+
+    blocks = [{"ms": 30.0, "sm_mhz": 1965.0}, {"ms": 40.0, "sm_mhz": 1500.0}, {"ms": 35.0, "sm_mhz": 1600.0}]
+    s = bench.block_summary(blocks, steps=10, flop_per_step=1e12, world=2)
+    assert s["blocks"] == 3 and s["timed_region_s"] == pytest.approx(0.105)
+    assert s["ms_per_step_median"] == 3.5 and s["ms_per_step_min"] == 3.0 and s["ms_per_step_max"] == 4.0
+    assert s["value_median"] == pytest.approx(1e12 * 10 * 2 / 35e-3 / 1e12, rel=1e-3)  # the median block, whole job
+    assert s["value_first_block"] > s["value_last_block"] and s["sm_mhz_first_block"] == 1965.0 and s["sm_mhz_last_block"] == 1600.0
+    # the oracle's bounded sample: the whole block for config 2, the smallest linear for config 3 or for many samples
+    only, text = bench.oracle_sample_choice("C2", inputs.CONFIGS["C2"])
+    assert only is None and "all 4 linears" in text
+    only, text = bench.oracle_sample_choice("C3", inputs.CONFIGS["C3"])
+    assert inputs.CONFIGS["C3"]["linears"][only][0] == "o" and "1/832 of a step" in text
+    only, _ = bench.oracle_sample_choice("C2", inputs.CONFIGS["C2"], many=True)
+    assert inputs.CONFIGS["C2"]["linears"][only][0] == "o"
+    # the stamped DRAM traffic figures name a summary that exists and the launch count they were taken for
+    for cfg, (nbytes, launches, summary, commit) in bench.QE_TRAFFIC.items():
+        assert os.path.exists(os.path.join(ROOT, "profiles", summary)) and nbytes > 0 and launches > 0 and len(commit) >= 7
