@@ -435,6 +435,71 @@ def test_resume_from_checkpoint_equals_uninterrupted_run(qe, mode):
         F.state_load(payload)
 
 
+_RESUME_CHILD = r"""
+import sys, numpy as np, torch
+sys.path.insert(0, {root!r}); sys.path.insert(0, {root!r} + "/tests")
+from harness import c1_inputs, run_gpu_steps
+from paper_2609_23536_b200 import binding as qe, inputs
+from paper_2609_23536_b200.schedules import peak_live, sched
+T, K, N, M, H, mode = 256, 256, 384, 4, 4, {mode}
+s = sched(M, 2, 1)
+W = [inputs.weights("R", 0, 0, N, K)]
+for e in range(1, 8):
+    W.append(inputs.optimizer_perturbation(W[-1], "R", e, 0, 0))
+ctx = qe.Context(mode)
+L = qe.Layer(ctx, T, K, N, H, 0, peak_live(s), torch.zeros((N, K), dtype=torch.bfloat16, device="cuda:0"))
+L.state_load(open({ckpt!r}, "rb").read())
+assert L.state()["e_W"] == 3 and L.state()["token"] == 0
+buf = torch.zeros(N * K, device="cuda:0")
+out = {{}}
+for step in range(3, 8):
+    o = run_gpu_steps(qe, L, s, 1, M, buf, 0, lambda _s, mb: c1_inputs(step, mb, T, K, N, "R"), lambda _e: inputs.bits(W[step]))
+    out.update({{"%d_%s_%s" % ((step,) + (k[1], k[2] if len(k) > 2 else "")): v for k, v in o.items()}})
+st = L.state()
+out["final_scales"] = np.array([st["classes"][c]["scale"] for c in "XWGY"], np.float32)
+out["final_windows"] = np.stack([st["classes"][c]["window"] for c in "XWGY"])
+np.savez({result!r}, **out)
+"""
+
+
+@pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
+def test_resume_in_a_fresh_process_equals_the_uninterrupted_run(qe, mode, tmp_path):
+    # Sec. 5.2's restart check as the paper runs it: the persistent state saved at the boundary after step 3 goes to a
+    # file; a NEW process (new CUDA context, new layer, new graphs, new tape generations) loads it and runs steps 4-8;
+    # its outputs, gradients and final scaling state equal the uninterrupted run's bit for bit.
+    import os
+    import subprocess
+    import sys
+
+    T, K, N, M, H = 256, 256, 384, 4, 4
+    s = sched(M, 2, 1)
+    P = peak_live(s)
+    W = _weights("R", N, K, 8)
+    get = lambda step, mb: c1_inputs(step, mb, T, K, N, "R")
+    ctx, A = _mk_layer(qe, mode, T, K, N, H, 0, P)
+    buf = torch.zeros(N * K, device=DEV)
+    full = {}
+    for step in range(8):
+        o = run_gpu_steps(qe, A, s, 1, M, buf, 0, lambda _s, mb: get(step, mb), lambda _e: W[step])
+        full.update({"%d_%s_%s" % ((step,) + (k[1], k[2] if len(k) > 2 else "")): v for k, v in o.items()})
+        if step == 2:
+            ckpt = tmp_path / "state_after_step_3.bin"
+            ckpt.write_bytes(A.state_save())
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    result = str(tmp_path / "resumed.npz")
+    code = _RESUME_CHILD.format(root=root, mode=mode, ckpt=str(ckpt), result=result)
+    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    got = np.load(result)
+    keys = [k for k in got.files if not k.startswith("final")]
+    assert len(keys) == 5 * (2 * M + 1)
+    for k in keys:
+        assert np.array_equal(full[k].view(np.uint8), got[k].view(np.uint8)), k
+    st = A.state()
+    assert np.array_equal(got["final_scales"].view(np.uint32), np.array([st["classes"][c]["scale"] for c in "XWGY"], np.float32).view(np.uint32))
+    assert np.array_equal(got["final_windows"].view(np.uint32), np.stack([st["classes"][c]["window"] for c in "XWGY"]).view(np.uint32))
+
+
 @pytest.mark.parametrize("mode", [0, 1], ids=["eager", "graph"])
 def test_one_way_handoff_reads_stale_outputs_two_way_never_does(qe, mode):
     # Sec. 2.3: fixed producer/consumer pairs, 200 checks per protocol.  The producer is a forward on the context's
